@@ -1,0 +1,330 @@
+"""Pins for the fp64 oracle: closed forms, invariants, library special cases and
+brute force on tiny inputs.  None of these re-type the oracle's formulas with
+numpy; they use pure-Python loops, torch's library attention, or facts the
+paper and the mathematics fix."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import CitrusOracle, SHARED, INDIVIDUAL
+from paper_2406_12018_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rand(rng, *shape):
+    return rng.standard_normal(shape)
+
+
+# ---------------------------------------------------------------- brute force
+def brute_attention_row(q, keys, vals, visible):
+    """One query row, pure Python floats."""
+    D = len(q)
+    logit = []
+    for j in range(len(keys)):
+        if not visible[j]:
+            logit.append(None)
+            continue
+        acc = 0.0
+        for d in range(D):
+            acc += q[d] * keys[j][d]
+        logit.append(acc / math.sqrt(D))
+    mx = max(x for x in logit if x is not None)
+    e = [0.0 if x is None else math.exp(x - mx) for x in logit]
+    z = sum(e)
+    p = [x / z for x in e]
+    o = [sum(p[j] * vals[j][d] for j in range(len(keys))) for d in range(len(vals[0]))]
+    return p, o
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,m,L", [(2, 1, 4, 3, 5), (4, 2, 4, 0, 6), (2, 2, 8, 7, 1)])
+def test_a1_brute_force(Hq, Hkv, D, m, L):
+    rng = np.random.default_rng(10 + m)
+    Qc, Kc, Vc = rand(rng, L, Hq, D), rand(rng, L, Hkv, D), rand(rng, L, Hkv, D)
+    Kcache, Vcache = rand(rng, Hkv, m, D), rand(rng, Hkv, m, D)
+    w = min(2, L)
+    out, s_lm = oracle.chunk_attention(Qc, Kcache, Vcache, Kc, Vc, lm_window=w)
+    G = Hq // Hkv
+    ref_lm = [[0.0] * (m + L) for _ in range(Hkv)]
+    for h in range(Hq):
+        g = h // G
+        keys = [list(Kcache[g, j]) for j in range(m)] + [list(Kc[u, g]) for u in range(L)]
+        vals = [list(Vcache[g, j]) for j in range(m)] + [list(Vc[u, g]) for u in range(L)]
+        for t in range(L):
+            visible = [True] * m + [u <= t for u in range(L)]
+            p, o = brute_attention_row(list(Qc[t, h]), keys, vals, visible)
+            assert np.allclose(out[t, h], o, rtol=0, atol=1e-12)
+            if t >= L - w:
+                for j in range(m + L):
+                    ref_lm[g][j] += p[j]
+    assert np.allclose(s_lm, np.array(ref_lm), rtol=0, atol=1e-12)
+
+
+def test_a2_brute_force_and_rowsum():
+    rng = np.random.default_rng(3)
+    Hq, Hkv, D, m, L, nI = 4, 2, 4, 5, 3, 3
+    Qi, Kc, Kcache = rand(rng, nI, Hq, D), rand(rng, L, Hkv, D), rand(rng, Hkv, m, D)
+    S = oracle.importance_sum(Qi, Kcache, Kc)
+    G = Hq // Hkv
+    ref = [[0.0] * (m + L) for _ in range(Hkv)]
+    for h in range(Hq):
+        g = h // G
+        keys = [list(Kcache[g, j]) for j in range(m)] + [list(Kc[u, g]) for u in range(L)]
+        for i in range(nI):
+            p, _ = brute_attention_row(list(Qi[i, h]), keys, keys, [True] * (m + L))
+            assert abs(sum(p) - 1.0) < 1e-12
+            for j in range(m + L):
+                ref[g][j] += p[j]
+    assert np.allclose(S, np.array(ref), rtol=0, atol=1e-12)
+    # every (instruction token, head) distributes exactly one unit of attention
+    assert np.allclose(S.sum(axis=1), nI * G, rtol=0, atol=1e-12)
+
+
+# ------------------------------------------------------------- closed forms
+def test_a2_zero_query_uniform_and_dominant_key():
+    rng = np.random.default_rng(4)
+    Hq, Hkv, D, m, L = 2, 1, 8, 6, 4
+    Kc, Kcache = rand(rng, L, Hkv, D), rand(rng, Hkv, m, D)
+    S = oracle.importance_sum(np.zeros((1, Hq, D)), Kcache, Kc)
+    assert np.allclose(S, Hq / (m + L), atol=1e-15)             # q = 0 -> uniform 1/n per head
+    # a key aligned with every query and 200x longer takes all of the mass
+    Qi = np.abs(rand(rng, 5, Hq, D)) + 0.5
+    Kc2 = Kc.copy()
+    Kc2[2, 0] = 200.0 * np.ones(D)
+    S2 = oracle.importance_sum(Qi, Kcache, Kc2)
+    assert abs(S2[0, m + 2] - 5 * Hq) < 1e-9
+    assert S2[0].sum() == pytest.approx(5 * Hq, abs=1e-12)
+
+
+def test_a2_scale_is_inverse_sqrt_d():
+    # two keys, one query: p0/p1 = exp((q.k0 - q.k1)/sqrt(D)) exactly
+    D = 16
+    q = np.zeros((1, 1, D)); q[0, 0, 0] = 2.0
+    Kc = np.zeros((2, 1, D)); Kc[0, 0, 0] = 3.0; Kc[1, 0, 0] = 1.0
+    S = oracle.importance_sum(q, np.zeros((1, 0, D)), Kc)
+    assert S[0, 0] / S[0, 1] == pytest.approx(math.exp((6.0 - 2.0) / 4.0), rel=1e-13)
+
+
+# ------------------------------------------------ library special case (a1)
+def sdpa_full_causal(Q, K, V):
+    """torch's library attention over the whole document, fp64, GQA by head repetition."""
+    G = Q.shape[1] // K.shape[1]
+    q = torch.from_numpy(Q).permute(1, 0, 2)[None]
+    k = torch.from_numpy(np.repeat(K, G, axis=1)).permute(1, 0, 2)[None]
+    v = torch.from_numpy(np.repeat(V, G, axis=1)).permute(1, 0, 2)[None]
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True)
+    return o[0].permute(1, 0, 2).numpy()
+
+
+@pytest.mark.parametrize("mode", [SHARED, INDIVIDUAL])
+def test_no_eviction_equals_full_causal_attention(mode):
+    rng = np.random.default_rng(5)
+    N, Hq, Hkv, D, ls = 50, 4, 2, 8, 16
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, 3, Hq, D)
+    orc = CitrusOracle(Hq, Hkv, D, budget_k=N, mode=mode)
+    outs = []
+    for s in range(0, N, ls):
+        outs.append(orc.process_chunk(Q[s:s + ls], K[s:s + ls], V[s:s + ls], Qi).out)
+    got = np.concatenate(outs, axis=0)
+    assert np.allclose(got, sdpa_full_causal(Q, K, V), rtol=0, atol=1e-12)
+    for c in orc.caches:                                  # nothing evicted, order kept
+        assert c.K.shape[1] == N
+        assert np.array_equal(c.pos, np.broadcast_to(np.arange(N), (Hkv, N)))
+        assert np.array_equal(c.K, K.transpose(1, 0, 2))
+        assert np.array_equal(c.V, V.transpose(1, 0, 2))
+
+
+def test_gqa_equals_mha_with_repeated_kv_heads():
+    rng = np.random.default_rng(6)
+    L, Hq, Hkv, D, m = 7, 4, 2, 8, 5
+    G = Hq // Hkv
+    Qc, Kc, Vc = rand(rng, L, Hq, D), rand(rng, L, Hkv, D), rand(rng, L, Hkv, D)
+    Kca, Vca = rand(rng, Hkv, m, D), rand(rng, Hkv, m, D)
+    o1, _ = oracle.chunk_attention(Qc, Kca, Vca, Kc, Vc)
+    o2, _ = oracle.chunk_attention(Qc, np.repeat(Kca, G, 0), np.repeat(Vca, G, 0),
+                                   np.repeat(Kc, G, 1), np.repeat(Vc, G, 1))
+    assert np.array_equal(o1, o2)
+
+
+# ------------------------------------------------------------- a2-L / TOVA
+def test_lm_scores_window_one_is_last_row_and_tova():
+    rng = np.random.default_rng(7)
+    Hq, Hkv, D, m = 2, 2, 8, 6
+    Kca, Vca = rand(rng, Hkv, m, D), rand(rng, Hkv, m, D)
+    Qc, Kc, Vc = rand(rng, 1, Hq, D), rand(rng, 1, Hkv, D), rand(rng, 1, Hkv, D)
+    _, s_lm = oracle.chunk_attention(Qc, Kca, Vca, Kc, Vc, lm_window=1)
+    for g in range(Hkv):
+        keys = [list(Kca[g, j]) for j in range(m)] + [list(Kc[0, g])]
+        p, _ = brute_attention_row(list(Qc[0, g]), keys, keys, [True] * (m + 1))
+        assert np.allclose(s_lm[g], p, atol=1e-13)
+        # chunk of one token and budget n-1: the state dropped is the one the
+        # last token attends to least (the token-by-token policy the paper
+        # names as the l_s = 1 case of chunked eviction)
+        kept = oracle.select_topk(s_lm[g], m)
+        dropped = set(range(m + 1)) - set(kept.tolist())
+        assert dropped == {int(np.argmin(p))}
+
+
+def test_lm_scores_mass():
+    rng = np.random.default_rng(8)
+    L, Hq, Hkv, D, m, w = 9, 4, 2, 4, 3, 4
+    _, s_lm = oracle.chunk_attention(rand(rng, L, Hq, D), rand(rng, Hkv, m, D), rand(rng, Hkv, m, D),
+                                     rand(rng, L, Hkv, D), rand(rng, L, Hkv, D), lm_window=w)
+    assert np.allclose(s_lm.sum(axis=1), w * (Hq // Hkv), atol=1e-12)
+    # causal: the last chunk row is seen only by the last query, row L-w-1.. by all w voters
+    assert np.all(s_lm[:, -1] <= (Hq // Hkv) + 1e-12)
+
+
+# -------------------------------------------------------------------- a3
+def test_select_bruteforce_and_ties():
+    rng = np.random.default_rng(9)
+    for n, k in [(1, 1), (5, 5), (5, 7), (17, 4), (64, 63), (200, 64)]:
+        score = rng.integers(0, 6, size=n).astype(np.float64)          # many exact ties
+        got = oracle.select_topk(score, k).tolist()
+        ref = sorted(sorted(range(n), key=lambda j: (-score[j], j))[:k])
+        assert got == ref
+    s = np.array([0.5, 0.9, 0.5, 0.5, 0.1])
+    assert oracle.select_topk(s, 3).tolist() == [0, 1, 2]              # lower index wins the tie
+    assert oracle.kth_gap(s, 3) == (0.5, 0.5)
+    assert oracle.kth_gap(s, 5) == (None, None)
+
+
+def test_single_chunk_selection_is_direct_topk():
+    rng = np.random.default_rng(11)
+    N, Hq, Hkv, D, k, nI = 40, 4, 2, 8, 10, 5
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, nI, Hq, D)
+    orc = CitrusOracle(Hq, Hkv, D, k, SHARED)
+    res = orc.process_chunk(Q, K, V, Qi)
+    # direct definition over the whole document, written with scipy-free torch softmax
+    G = Hq // Hkv
+    for g in range(Hkv):
+        tot = torch.zeros(N, dtype=torch.float64)
+        for h in range(g * G, (g + 1) * G):
+            logits = torch.from_numpy(Qi[:, h]) @ torch.from_numpy(K[:, g]).T / math.sqrt(D)
+            tot += torch.softmax(logits, dim=1).sum(0)
+        ref = torch.topk(tot, k).indices.sort().values.numpy()
+        assert np.array_equal(res.idx[0][g], ref)
+        assert np.array_equal(orc.caches[0].pos[g], ref)
+
+
+def test_duplicate_keys_keep_lower_positions():
+    rng = np.random.default_rng(12)
+    N, Hq, Hkv, D, k = 12, 2, 1, 4, 5
+    K = np.tile(rand(rng, 1, Hkv, D), (N, 1, 1))                       # all keys identical -> all scores tie
+    orc = CitrusOracle(Hq, Hkv, D, k, SHARED)
+    orc.process_chunk(rand(rng, N, Hq, D), K, rand(rng, N, Hkv, D), rand(rng, 3, Hq, D))
+    assert orc.caches[0].pos[0].tolist() == [0, 1, 2, 3, 4]
+
+
+# -------------------------------------------------------------------- a4
+def test_compact_is_plain_gather():
+    rng = np.random.default_rng(13)
+    Kg, Vg, Kc, Vc = rand(rng, 4, 3), rand(rng, 4, 3), rand(rng, 2, 3), rand(rng, 2, 3)
+    pos = np.array([1, 5, 6, 9]); cpos = np.array([10, 11])
+    k2, v2, p2 = oracle.compact(Kg, Vg, pos, Kc, Vc, cpos, np.array([0, 3, 5]))
+    assert p2.tolist() == [1, 9, 11]
+    assert k2[0].tolist() == Kg[0].tolist() and k2[1].tolist() == Kg[3].tolist() and k2[2].tolist() == Kc[1].tolist()
+    assert v2[2].tolist() == Vc[1].tolist()
+
+
+# ----------------------------------------------------------- whole loop
+def _run(orc, doc, ls):
+    Q, K, V, Qi = (wl.to_f64(t) for t in (doc.Q, doc.K, doc.V, doc.Q_instr))
+    res = []
+    for s in range(0, Q.shape[0], ls):
+        res.append(orc.process_chunk(Q[s:s + ls], K[s:s + ls], V[s:s + ls], Qi))
+    return res
+
+
+def test_rotated_loop_equals_paper_order():
+    w = wl.scaled(wl.CONFIGS["tiny_fp32"], doc_tokens=300, chunk_s=64, budget_k=48, n_planted=4)
+    doc = wl.make_document(w)
+    orc = CitrusOracle(w.q_heads, w.kv_heads, w.head_dim, w.budget_k, SHARED)
+    res = _run(orc, doc, w.chunk_s)
+    outs, cache = oracle.run_paper_order_shared(wl.to_f64(doc.Q), wl.to_f64(doc.K), wl.to_f64(doc.V),
+                                                wl.to_f64(doc.Q_instr), w.budget_k, w.chunk_s)
+    assert np.array_equal(cache.pos, orc.caches[0].pos)
+    assert np.array_equal(cache.K, orc.caches[0].K) and np.array_equal(cache.V, orc.caches[0].V)
+    for a, b in zip(outs, res):
+        assert np.allclose(a, b.out, rtol=0, atol=1e-13)
+
+
+def test_cache_size_arithmetic_from_paper():
+    # golden: the paper's main setting and its footnote on resident states
+    vals = {}
+    with open(os.path.join(GOLDEN, "cache_sizes.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            key, v = line.split("=")
+            vals[key.strip()] = int(v)
+    k, ls = vals["k"], vals["l_s"]
+    assert k + ls == vals["resident_shared"] and 2 * (k + ls) == vals["resident_individual"]
+    rng = np.random.default_rng(14)
+    Hq, Hkv, D = 2, 1, 4
+    for mode, expect in [(SHARED, vals["resident_shared"]), (INDIVIDUAL, vals["resident_individual"])]:
+        orc = CitrusOracle(Hq, Hkv, D, k, mode, lm_window=8)
+        peak = 0
+        for c in range(5):
+            resident_before = sum(cs.K.shape[1] + ls for cs in orc.caches)   # cache rows + the chunk's states
+            peak = max(peak, resident_before)
+            orc.process_chunk(rand(rng, ls, Hq, D), rand(rng, ls, Hkv, D), rand(rng, ls, Hkv, D), rand(rng, 2, Hq, D))
+            for cs in orc.caches:
+                assert cs.K.shape[1] == min(k, orc.tokens_seen) == vals["k_generation"] or orc.tokens_seen < k
+                assert np.all(np.diff(cs.pos, axis=1) > 0)
+        assert peak == expect
+
+
+@pytest.mark.parametrize("mode", [SHARED, INDIVIDUAL])
+def test_planted_keys_and_sinks_survive(mode):
+    w = wl.scaled(wl.CONFIGS["mistral7b_layer"], q_heads=4, kv_heads=2, head_dim=32, budget_k=48, chunk_s=32,
+                  doc_tokens=400, n_instr=8, n_planted=6, n_sinks=1, mode=mode)
+    doc = wl.make_document(w)
+    orc = CitrusOracle(w.q_heads, w.kv_heads, w.head_dim, w.budget_k, mode, lm_window=8)
+    _run(orc, doc, w.chunk_s)
+    inst = orc.caches[-1]                       # the instruction-aware cache
+    for g in range(w.kv_heads):
+        kept = set(inst.pos[g].tolist())
+        assert set(doc.planted.tolist()) <= kept
+        assert set(doc.sinks.tolist()) <= kept
+    if mode == INDIVIDUAL:                      # sinks also survive in the LM cache
+        for g in range(w.kv_heads):
+            assert set(doc.sinks.tolist()) <= set(orc.caches[0].pos[g].tolist())
+
+
+def test_selection_invariant_to_positive_rescaling_and_layerwise():
+    rng = np.random.default_rng(15)
+    s = rng.random(50)
+    assert np.array_equal(oracle.select_topk(s, 7), oracle.select_topk(s / 37.0, 7))   # mean vs sum form
+    # layer-wise granularity: every head gets the index set of the head-summed score
+    N, Hq, Hkv, D, k = 30, 4, 2, 4, 6
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, 3, Hq, D)
+    orc = CitrusOracle(Hq, Hkv, D, k, SHARED, layerwise=True)
+    res = orc.process_chunk(Q, K, V, Qi)
+    tot = res.scores[0].sum(axis=0)
+    ref = sorted(sorted(range(N), key=lambda j: (-tot[j], j))[:k])
+    assert res.idx[0][0].tolist() == ref and res.idx[0][1].tolist() == ref
+
+
+def test_forced_selection_is_adopted():
+    rng = np.random.default_rng(16)
+    N, Hq, Hkv, D, k = 10, 2, 1, 4, 3
+    orc = CitrusOracle(Hq, Hkv, D, k, SHARED)
+    forced = {0: np.array([[1, 4, 7]])}
+    res = orc.process_chunk(rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, 2, Hq, D), forced)
+    assert orc.caches[0].pos[0].tolist() == [1, 4, 7]
+    assert res.applied[0].tolist() == [[1, 4, 7]]
+
+
+def test_workload_generator_is_deterministic_and_shaped():
+    w = wl.scaled(wl.CONFIGS["long_doc_stress"], doc_tokens=600, n_planted=5)
+    a, b = wl.make_document(w), wl.make_document(w)
+    assert torch.equal(a.K, b.K) and torch.equal(a.Q_instr, b.Q_instr)
+    assert a.Q.shape == (600, 32, 128) and a.K.dtype == torch.bfloat16
+    assert a.sinks.tolist() == [0, 1, 2, 3] and len(set(a.planted.tolist())) == 5
+    lens = wl.sequence_lengths(wl.CONFIGS["serving_mix"])
+    assert len(lens) == 16 and all(4096 <= x <= 32768 for x in lens) and lens == wl.sequence_lengths(wl.CONFIGS["serving_mix"])
