@@ -1,0 +1,163 @@
+/*
+ * citrus.h -- C ABI of the chunked instruction-aware state eviction library
+ * (CItruS, arXiv 2406.12018) for NVIDIA B200 (sm_100a).
+ *
+ * One call of citrus_process_chunk performs, for one decoder layer and one
+ * document chunk s of L <= l_s tokens, the four steps of the eviction loop:
+ *
+ *   a1  attention of the chunk's queries over [retained cache ; chunk], causal
+ *       inside the chunk (Section 4.1, step 1 of the chunked eviction process);
+ *   a2  importance of every candidate state c in [cache ; chunk]:
+ *       Imp(s', c) of Eq. 1 -- the softmax attention c receives, summed over the
+ *       scoring tokens s' and over the query heads of c's KV group.  The scoring
+ *       tokens are the instruction text I for the instruction-aware cache
+ *       (Section 4.2) and the chunk's own last w queries for the language-
+ *       modelling cache of the individual design (Section 4.1, Eq. 1 with s = chunk);
+ *   a3  top-k selection (Eq. 2-3; Eq. 4-5 for the instruction cache): keep the
+ *       budget_k candidates with the highest score, the lower position winning
+ *       exact ties, kept indices in ascending order;
+ *   a4  compaction of K, V and original positions of the kept candidates into
+ *       the new cache (the cache C-hat of Eq. 3 with the chunk's states put in).
+ *
+ * Scores are the SUM form of Eq. 1 (|s'| * G times the printed mean), which
+ * selects the same states.  The softmax of a2 runs over exactly the n = m + L
+ * candidates (m = rows currently retained).
+ *
+ * Conventions
+ *   - All tensor arguments are DEVICE pointers unless a function says "host".
+ *   - Token-major, densely packed: Q [tokens, q_heads, head_dim],
+ *     K/V [tokens, kv_heads, head_dim]; query head h uses KV head h / (q_heads/kv_heads).
+ *   - Element type is bf16 (default) or fp32 (CITRUS_MODE_FP32).
+ *   - Pointers must be 16-byte aligned.  The library never retains caller
+ *     pointers after the stream work of the call has completed.
+ *   - Every function returns 0 on success or a negative CITRUS_ERR_* code; none
+ *     aborts, throws, traps or prints.  A call that fails leaves all cache state
+ *     as it was.
+ *   - Work is enqueued on the caller's stream; no call synchronises the device
+ *     except citrus_create / citrus_destroy / citrus_poll_status and the *_host
+ *     variant (which waits for its own copies).
+ */
+#ifndef CITRUS_H_
+#define CITRUS_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct citrus_ctx* citrus_handle;
+/* Same object as the CUDA runtime's cudaStream_t (NULL = legacy default stream). */
+typedef struct CUstream_st* citrus_stream_t;
+
+/* mode bit-field of citrus_create */
+#define CITRUS_MODE_SHARED      0u        /* one cache, evicted by Imp(I, c)         (Section 4.2, shared cache)   */
+#define CITRUS_MODE_INDIVIDUAL  1u        /* LM cache C + instruction cache C^I       (Section 4.2, Eq. 4-5)        */
+#define CITRUS_MODE_FP32        2u        /* tensors are fp32 (default bf16)                                         */
+#define CITRUS_MODE_LAYERWISE   4u        /* one index set per layer from head-summed scores (Section 4.1, last par.) */
+#define CITRUS_MODE_LM_WINDOW(w) (((unsigned)(w) & 0xFFFFu) << 8)   /* w scoring queries for C; 0 = whole chunk */
+
+#define CITRUS_OK                 0
+#define CITRUS_ERR_INVALID_ARG   -1
+#define CITRUS_ERR_SHAPE         -2
+#define CITRUS_ERR_ALIGN         -3
+#define CITRUS_ERR_LAYER         -4
+#define CITRUS_ERR_STATE         -5
+#define CITRUS_ERR_NOMEM         -6
+#define CITRUS_ERR_CUDA          -7
+#define CITRUS_ERR_TIMEOUT       -8
+#define CITRUS_ERR_UNSUPPORTED   -9
+
+#define CITRUS_MAX_INSTR       4096       /* largest n_instr accepted */
+#define CITRUS_MAX_CANDIDATES 49152       /* largest budget_k + chunk_s accepted */
+
+/*
+ * Allocate a context on the current CUDA device (Sections 4.1-4.3; cache sizes
+ * follow the footnote of Section 4.3: budget_k retained rows per cache, plus the
+ * caller's chunk of up to chunk_s rows while a call runs).
+ * Per layer and per cache (1 shared, 2 individual) it owns two ping-pong buffers
+ * K,V [kv_heads, budget_k, head_dim] and positions [kv_heads, budget_k] (int32),
+ * plus score / index / log-sum-exp scratch.  Requirements: layers >= 1,
+ * q_heads % kv_heads == 0, head_dim in {64, 128} (bf16 needs 128),
+ * budget_k >= 1, chunk_s >= 1, budget_k + chunk_s <= CITRUS_MAX_CANDIDATES.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, NOMEM, CUDA.
+ */
+int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int head_dim,
+                  int budget_k, int chunk_s, unsigned mode);
+
+/* Number of independent sequence slots sharing the geometry (ragged serving
+ * batches); must be called before the first process call. Default 1. */
+int citrus_set_batch(citrus_handle h, int n_seq);
+
+/* Forget every cache of every layer and slot (start a new document). Host-only
+ * bookkeeping; enqueues nothing. */
+int citrus_reset(citrus_handle h);
+
+/*
+ * Steps a1-a4 for (layer, sequence slot 0) on `stream`.
+ *   Q_chunk [n_tokens, q_heads, D], K_chunk / V_chunk [n_tokens, kv_heads, D],
+ *   Q_instr [n_instr, q_heads, D] (queries of the instruction text I for this
+ *   layer), out [n_tokens, q_heads, D] receives the attention output of a1 in the
+ *   element type.  1 <= n_tokens <= chunk_s (a shorter chunk is allowed anywhere,
+ *   cf. "except for the final chunk", Section 4.1); 1 <= n_instr <= CITRUS_MAX_INSTR.
+ * Chunks of one (layer, slot) must be submitted in document order on one stream.
+ * The caller's K_chunk / V_chunk must stay valid until the stream work is done
+ * (the new cache is gathered straight from them).
+ * Errors: INVALID_ARG (NULL), LAYER, SHAPE, ALIGN, CUDA (launch failure).
+ */
+int citrus_process_chunk(citrus_handle h, int layer,
+                         const void* Q_chunk, const void* K_chunk, const void* V_chunk, int n_tokens,
+                         const void* Q_instr, int n_instr, void* out, citrus_stream_t stream);
+
+/* Same, for sequence slot `seq_slot` (ragged batches submit one call per active
+ * sequence; slots are independent and may use different streams). */
+int citrus_process_chunk_slot(citrus_handle h, int layer, int seq_slot,
+                              const void* Q_chunk, const void* K_chunk, const void* V_chunk, int n_tokens,
+                              const void* Q_instr, int n_instr, void* out, citrus_stream_t stream);
+
+/*
+ * End-to-end variant with HOST buffers (pinned memory recommended): copies the
+ * four inputs to device staging owned by the context, runs a1-a4, copies `out`
+ * back and waits for that copy.  Same argument rules otherwise.
+ */
+int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,
+                              const void* Q_chunk_host, const void* K_chunk_host, const void* V_chunk_host,
+                              int n_tokens, const void* Q_instr_host, int n_instr, void* out_host,
+                              citrus_stream_t stream);
+
+/*
+ * Borrowed device pointers into the current cache of (layer, which, seq_slot);
+ * which = 0 the language-modelling / shared cache, 1 the instruction cache C^I
+ * (individual mode only).  K, V are [kv_heads, budget_k, D] with rows
+ * [0, *n_rows) valid; positions [kv_heads, budget_k] int32 are the original
+ * token positions, strictly ascending per head (the order a position-shift
+ * caller needs).  *n_rows = min(budget_k, tokens seen) is host bookkeeping, so
+ * the call does not synchronise; the contents are final once the stream work of
+ * the last process call is done.  Valid until the next process / reset / destroy.
+ */
+int citrus_cache_view(citrus_handle h, int layer, int which, int seq_slot,
+                      const void** K, const void** V, const int** positions, int* n_rows);
+
+/*
+ * Borrowed device pointers to what the last process call on (layer, which,
+ * seq_slot) computed in a2-a3: scores [kv_heads, *n_candidates] fp32 (row stride
+ * *score_stride elements) and kept candidate indices [kv_heads, *n_kept] int32
+ * ascending (row stride budget_k).  Candidate j < m_before is old cache row j,
+ * otherwise chunk row j - m_before.
+ */
+int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
+                     const float** scores, int* score_stride, const int** idx,
+                     int* n_candidates, int* n_kept, int* m_before);
+
+/* Reads the device status word (0, or CITRUS_ERR_TIMEOUT if a bounded wait in a
+ * kernel gave up). Synchronises the device. */
+int citrus_poll_status(citrus_handle h);
+
+/* Frees everything. NULL is a no-op; a handle that was already destroyed
+ * returns CITRUS_ERR_STATE. */
+int citrus_destroy(citrus_handle h);
+
+const char* citrus_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CITRUS_H_ */

@@ -1,0 +1,186 @@
+"""Thin ctypes binding over the C ABI of include/citrus.h.
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+There is no CPU fallback; if libcitrus.so is missing or a call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcitrus.so")
+
+MODE_SHARED = 0
+MODE_INDIVIDUAL = 1
+MODE_FP32 = 2
+MODE_LAYERWISE = 4
+MAX_INSTR = 4096
+MAX_CANDIDATES = 49152
+
+EXPORTS = [
+    "citrus_create", "citrus_set_batch", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
+    "citrus_process_chunk_host", "citrus_cache_view", "citrus_step_view", "citrus_poll_status",
+    "citrus_destroy", "citrus_strerror",
+]
+
+_lib = None
+
+
+class CitrusError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {code} ({strerror(code)})")
+
+
+def load() -> C.CDLL:
+    """Load libcitrus.so (built by paper_2406_12018_b200.build); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2406_12018_b200.build`; "
+                           "there is no fallback path")
+    lib = C.CDLL(LIB_PATH)
+    vp, i = C.c_void_p, C.c_int
+    lib.citrus_create.argtypes = [C.POINTER(vp), i, i, i, i, i, i, C.c_uint]
+    lib.citrus_set_batch.argtypes = [vp, i]
+    lib.citrus_reset.argtypes = [vp]
+    lib.citrus_process_chunk.argtypes = [vp, i, vp, vp, vp, i, vp, i, vp, vp]
+    lib.citrus_process_chunk_slot.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, vp]
+    lib.citrus_process_chunk_host.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, vp]
+    lib.citrus_cache_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(i)]
+    lib.citrus_step_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(i), C.POINTER(vp),
+                                     C.POINTER(i), C.POINTER(i), C.POINTER(i)]
+    lib.citrus_poll_status.argtypes = [vp]
+    lib.citrus_destroy.argtypes = [vp]
+    lib.citrus_strerror.argtypes = [i]
+    lib.citrus_strerror.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "citrus_strerror":
+            getattr(lib, name).restype = i
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().citrus_strerror(code).decode()
+
+
+class _DevView:
+    """Zero-copy torch view of library-owned device memory."""
+
+    def __init__(self, ptr: int, shape, typestr: str, strides=None):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr, "data": (ptr, False),
+                                         "version": 2, "strides": strides}
+
+
+def _view(ptr, shape, typestr, itemsize, strides_elems=None):
+    strides = None if strides_elems is None else tuple(s * itemsize for s in strides_elems)
+    return torch.as_tensor(_DevView(ptr, shape, typestr, strides), device="cuda")
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+class Citrus:
+    """One eviction context (all layers and sequence slots of one geometry)."""
+
+    def __init__(self, layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, mode="shared", dtype="bf16",
+                 lm_window=0, layerwise=False, n_seqs=1):
+        lib = load()
+        bits = (MODE_INDIVIDUAL if mode == "individual" else MODE_SHARED)
+        bits |= MODE_FP32 if dtype == "fp32" else 0
+        bits |= MODE_LAYERWISE if layerwise else 0
+        bits |= (int(lm_window) & 0xFFFF) << 8
+        self._h = C.c_void_p()
+        rc = lib.citrus_create(C.byref(self._h), layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, bits)
+        if rc != 0:
+            self._h = None
+            raise CitrusError(rc, "citrus_create")
+        self.layers, self.q_heads, self.kv_heads, self.head_dim = layers, q_heads, kv_heads, head_dim
+        self.budget_k, self.chunk_s = budget_k, chunk_s
+        self.individual = mode == "individual"
+        self.torch_dtype = torch.float32 if dtype == "fp32" else torch.bfloat16
+        if n_seqs != 1:
+            rc = lib.citrus_set_batch(self._h, n_seqs)
+            if rc != 0:
+                self.close()
+                raise CitrusError(rc, "citrus_set_batch")
+
+    # -- calls -------------------------------------------------------------
+    def _check(self, t: torch.Tensor, cuda: bool):
+        assert t.dtype == self.torch_dtype and t.is_contiguous() and t.is_cuda == cuda
+
+    def process_chunk(self, layer, Qc, Kc, Vc, Qi, out: Optional[torch.Tensor] = None, slot=0, stream=None):
+        for t in (Qc, Kc, Vc, Qi):
+            self._check(t, True)
+        if out is None:
+            out = torch.empty_like(Qc)
+        rc = load().citrus_process_chunk_slot(self._h, layer, slot, Qc.data_ptr(), Kc.data_ptr(), Vc.data_ptr(),
+                                              Qc.shape[0], Qi.data_ptr(), Qi.shape[0], out.data_ptr(),
+                                              _stream_ptr(stream))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_process_chunk")
+        return out
+
+    def process_chunk_host(self, layer, Qc, Kc, Vc, Qi, out, slot=0, stream=None):
+        for t in (Qc, Kc, Vc, Qi, out):
+            self._check(t, False)
+        rc = load().citrus_process_chunk_host(self._h, layer, slot, Qc.data_ptr(), Kc.data_ptr(), Vc.data_ptr(),
+                                              Qc.shape[0], Qi.data_ptr(), Qi.shape[0], out.data_ptr(),
+                                              _stream_ptr(stream))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_process_chunk_host")
+        return out
+
+    def cache_view(self, layer, which=0, slot=0) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+        """(K [H_kv, n_rows, D], V, positions [H_kv, n_rows]) views of the current cache."""
+        K, V, P, n = C.c_void_p(), C.c_void_p(), C.c_void_p(), C.c_int()
+        rc = load().citrus_cache_view(self._h, layer, which, slot, C.byref(K), C.byref(V), C.byref(P), C.byref(n))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_cache_view")
+        H, k, D = self.kv_heads, self.budget_k, self.head_dim
+        if self.torch_dtype == torch.float32:
+            Kt, Vt = (_view(p.value, (H, k, D), "<f4", 4) for p in (K, V))
+        else:
+            Kt, Vt = (_view(p.value, (H, k, D), "<i2", 2).view(torch.bfloat16) for p in (K, V))
+        Pt = _view(P.value, (H, k), "<i4", 4)
+        return Kt[:, :n.value], Vt[:, :n.value], Pt[:, :n.value]
+
+    def step_view(self, layer, which=0, slot=0):
+        """(scores [H_kv, n] fp32, idx [H_kv, kept] int32, m_before) of the last call."""
+        S, I = C.c_void_p(), C.c_void_p()
+        stride, n, kept, m = C.c_int(), C.c_int(), C.c_int(), C.c_int()
+        rc = load().citrus_step_view(self._h, layer, which, slot, C.byref(S), C.byref(stride), C.byref(I),
+                                     C.byref(n), C.byref(kept), C.byref(m))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_step_view")
+        St = _view(S.value, (self.kv_heads, stride.value), "<f4", 4)[:, :n.value]
+        It = _view(I.value, (self.kv_heads, self.budget_k), "<i4", 4)[:, :kept.value]
+        return St, It, m.value
+
+    def reset(self):
+        rc = load().citrus_reset(self._h)
+        if rc != 0:
+            raise CitrusError(rc, "citrus_reset")
+
+    def poll_status(self) -> int:
+        return load().citrus_poll_status(self._h)
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value is not None:
+            load().citrus_destroy(self._h)
+        self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

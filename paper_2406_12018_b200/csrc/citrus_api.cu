@@ -1,0 +1,383 @@
+// Host side of the C ABI declared in include/citrus.h: context state, argument
+// checks, ping-pong cache bookkeeping and the launch sequence of one chunk step.
+#include "../../include/citrus.h"
+#include "citrus_internal.h"
+
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <set>
+#include <vector>
+
+namespace {
+
+using namespace citrus;
+
+struct CacheBufs {
+    void* K[2] = {nullptr, nullptr};
+    void* V[2] = {nullptr, nullptr};
+    int* pos[2] = {nullptr, nullptr};
+    int cur = 0;
+};
+
+struct Unit {                       // one (layer, sequence slot)
+    CacheBufs cache[2];
+    float* scores = nullptr;        // [n_caches, kv_heads, score_stride]
+    int* idx = nullptr;             // [n_caches, kv_heads, budget_k]
+    float* lse_chunk = nullptr;     // [q_heads, chunk_s]
+    float* lse_instr = nullptr;     // [q_heads, CITRUS_MAX_INSTR]
+    float* part = nullptr;          // tensor-core score pass partials
+    int m = 0;                      // rows retained in every cache
+    long long tokens_seen = 0;
+    int last_n = 0, last_kept = 0, last_m = 0;
+    bool has_step = false;
+};
+
+}  // namespace
+
+struct citrus_ctx {
+    int device = 0;
+    int layers = 0, Hq = 0, Hkv = 0, D = 0, k = 0, ls = 0;
+    bool individual = false, fp32 = false, layerwise = false, use_tc = false;
+    int lm_window = 0;
+    int elt = 2;
+    int n_caches = 1;
+    int n_slots = 1;
+    int score_stride = 0;
+    bool used = false;
+    std::vector<Unit> units;        // [layers * n_slots]
+    std::vector<void*> allocs;      // cache buffers and per-unit scratch
+    std::vector<void*> misc;        // status word, host-variant staging
+    int* status = nullptr;
+    // staging of the host-buffer variant
+    void *stQ = nullptr, *stK = nullptr, *stV = nullptr, *stQi = nullptr, *stOut = nullptr;
+};
+
+namespace {
+
+std::mutex g_mu;
+std::set<citrus_ctx*> g_live;
+std::set<citrus_ctx*> g_dead;
+
+bool is_live(citrus_ctx* h) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_live.count(h) != 0;
+}
+
+int dev_alloc(citrus_ctx* c, void** p, size_t bytes, bool zero, bool misc = false) {
+    cudaError_t e = cudaMalloc(p, bytes);
+    if (e != cudaSuccess) { cudaGetLastError(); return e == cudaErrorMemoryAllocation ? CITRUS_ERR_NOMEM : CITRUS_ERR_CUDA; }
+    (misc ? c->misc : c->allocs).push_back(*p);
+    if (zero) {
+        e = cudaMemset(*p, 0, bytes);
+        if (e != cudaSuccess) return CITRUS_ERR_CUDA;
+    }
+    return CITRUS_OK;
+}
+
+void free_units(citrus_ctx* c) {
+    for (void* p : c->allocs) cudaFree(p);
+    c->allocs.clear();
+    c->units.clear();
+}
+void free_all(citrus_ctx* c) {
+    free_units(c);
+    for (void* p : c->misc) cudaFree(p);
+    c->misc.clear();
+}
+
+int alloc_units(citrus_ctx* c) {
+    const size_t row = (size_t)c->D * c->elt;
+    const size_t kv_bytes = (size_t)c->Hkv * c->k * row;
+    c->units.assign((size_t)c->layers * c->n_slots, Unit());
+    for (Unit& u : c->units) {
+        int rc;
+        for (int ci = 0; ci < c->n_caches; ++ci)
+            for (int b = 0; b < 2; ++b) {
+                if ((rc = dev_alloc(c, &u.cache[ci].K[b], kv_bytes, true))) return rc;
+                if ((rc = dev_alloc(c, &u.cache[ci].V[b], kv_bytes, true))) return rc;
+                if ((rc = dev_alloc(c, (void**)&u.cache[ci].pos[b], (size_t)c->Hkv * c->k * sizeof(int), true))) return rc;
+            }
+        if ((rc = dev_alloc(c, (void**)&u.scores, (size_t)c->n_caches * c->Hkv * c->score_stride * sizeof(float), true))) return rc;
+        if ((rc = dev_alloc(c, (void**)&u.idx, (size_t)c->n_caches * c->Hkv * c->k * sizeof(int), true))) return rc;
+        if ((rc = dev_alloc(c, (void**)&u.lse_chunk, (size_t)c->Hq * c->ls * sizeof(float), true))) return rc;
+        if ((rc = dev_alloc(c, (void**)&u.lse_instr, (size_t)c->Hq * CITRUS_MAX_INSTR * sizeof(float), true))) return rc;
+    }
+    return CITRUS_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_rc(cudaError_t e) {
+    if (e == cudaSuccess) return CITRUS_OK;
+    cudaGetLastError();
+    return CITRUS_ERR_CUDA;
+}
+
+int check_process_args(citrus_ctx* h, int layer, int slot, const void* Q, const void* K, const void* V, int L,
+                       const void* Qi, int nI, const void* out) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    if (!Q || !K || !V || !Qi || !out) return CITRUS_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= h->layers) return CITRUS_ERR_LAYER;
+    if (slot < 0 || slot >= h->n_slots) return CITRUS_ERR_INVALID_ARG;
+    if (L < 1 || L > h->ls || nI < 1 || nI > CITRUS_MAX_INSTR) return CITRUS_ERR_SHAPE;
+    return CITRUS_OK;
+}
+
+// The launch sequence of one chunk step; all pointers are device pointers.
+int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc, const void* Vc, int L,
+             const void* Qi, int nI, void* out, cudaStream_t st) {
+    c->used = true;
+    Unit& u = c->units[(size_t)layer * c->n_slots + slot];
+    const int m = u.m, n = m + L;
+    const int kept = n < c->k ? n : c->k;
+    if (u.tokens_seen + L > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
+
+    Candidates cand[2];
+    for (int ci = 0; ci < c->n_caches; ++ci) {
+        const CacheBufs& cb = u.cache[ci];
+        cand[ci] = Candidates{cb.K[cb.cur], cb.V[cb.cur], Kc, Vc, m, L, c->k, c->Hkv};
+    }
+    QueryRows q_chunk{Qc, L, c->Hq, 1, 0};
+    QueryRows q_instr{Qi, nI, c->Hq, 0, 0};
+    float* scores[2] = {u.scores, u.scores + (size_t)c->Hkv * c->score_stride};
+    const int ic = c->individual ? 1 : 0;     // the cache scored by the instruction text
+
+    cudaError_t e;
+    // a1: attention of the chunk over [cache 0 ; chunk], row log-sum-exp kept for a2-L
+    if (c->use_tc) e = tc_attention(q_chunk, cand[0], out, u.lse_chunk, c->ls, c->status, st);
+    else e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, u.lse_chunk, c->ls, st);
+    if (e != cudaSuccess) return cuda_rc(e);
+
+    // a2-L (individual design): votes of the chunk's last w queries on cache 0's candidates
+    if (c->individual) {
+        int w = c->lm_window > 0 && c->lm_window < L ? c->lm_window : L;
+        const char* q0 = reinterpret_cast<const char*>(Qc) + (size_t)(L - w) * c->Hq * c->D * c->elt;
+        QueryRows q_lm{q0, w, c->Hq, 1, L - w};
+        if (c->use_tc) e = tc_colsum(q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, c->status, st);
+        else e = simt_colsum(c->fp32, c->D, q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, st);
+        if (e != cudaSuccess) return cuda_rc(e);
+    }
+    // a2-I: Eq. 1 with the instruction queries over the instruction-side cache's candidates
+    if (c->use_tc) {
+        e = tc_score_lse(q_instr, cand[ic], u.part, u.part, u.lse_instr, CITRUS_MAX_INSTR, c->status, st);
+        if (e == cudaSuccess)
+            e = tc_colsum(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, c->status, st);
+    } else {
+        e = simt_attention(c->fp32, c->D, q_instr, cand[ic], nullptr, u.lse_instr, CITRUS_MAX_INSTR, st);
+        if (e == cudaSuccess)
+            e = simt_colsum(c->fp32, c->D, q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, st);
+    }
+    if (e != cudaSuccess) return cuda_rc(e);
+
+    // a3 + a4 for every cache in one launch each
+    SelectJob sj[2];
+    CompactJob cj[2];
+    for (int ci = 0; ci < c->n_caches; ++ci) {
+        CacheBufs& cb = u.cache[ci];
+        int* idx = u.idx + (size_t)ci * c->Hkv * c->k;
+        sj[ci] = SelectJob{scores[ci], idx, c->score_stride};
+        cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
+                            cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, m};
+    }
+    e = select_topk(sj, c->n_caches, c->Hkv, n, c->k, c->layerwise ? 1 : 0, st);
+    if (e != cudaSuccess) return cuda_rc(e);
+    e = compact_kv(cj, c->n_caches, Kc, Vc, c->Hkv, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
+    if (e != cudaSuccess) return cuda_rc(e);
+
+    for (int ci = 0; ci < c->n_caches; ++ci) u.cache[ci].cur ^= 1;
+    u.last_n = n; u.last_kept = kept; u.last_m = m; u.has_step = true;
+    u.m = kept;
+    u.tokens_seen += L;
+    return CITRUS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int head_dim,
+                  int budget_k, int chunk_s, unsigned mode) {
+    if (out == nullptr) return CITRUS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (layers < 1 || q_heads < 1 || kv_heads < 1 || budget_k < 1 || chunk_s < 1) return CITRUS_ERR_INVALID_ARG;
+    if (mode & ~(0x7u | 0xFFFF00u)) return CITRUS_ERR_INVALID_ARG;
+    if (q_heads % kv_heads != 0) return CITRUS_ERR_SHAPE;
+    if (head_dim != 64 && head_dim != 128) return CITRUS_ERR_UNSUPPORTED;
+    const bool fp32 = (mode & CITRUS_MODE_FP32) != 0;
+    if (!fp32 && head_dim != 128) return CITRUS_ERR_UNSUPPORTED;
+    if ((long long)budget_k + chunk_s > CITRUS_MAX_CANDIDATES) return CITRUS_ERR_UNSUPPORTED;
+
+    citrus_ctx* c = new (std::nothrow) citrus_ctx();
+    if (c == nullptr) return CITRUS_ERR_NOMEM;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { cudaGetLastError(); delete c; return CITRUS_ERR_CUDA; }
+    c->layers = layers; c->Hq = q_heads; c->Hkv = kv_heads; c->D = head_dim; c->k = budget_k; c->ls = chunk_s;
+    c->individual = (mode & CITRUS_MODE_INDIVIDUAL) != 0;
+    c->fp32 = fp32;
+    c->layerwise = (mode & CITRUS_MODE_LAYERWISE) != 0;
+    c->lm_window = (int)((mode >> 8) & 0xFFFFu);
+    c->elt = fp32 ? 4 : 2;
+    c->n_caches = c->individual ? 2 : 1;
+    c->score_stride = (budget_k + chunk_s + 3) & ~3;
+    c->use_tc = !fp32 && head_dim == 128;
+    if (c->use_tc) {
+        const char* dbg = std::getenv("CITRUS_DEBUG_SIMT");
+        if (dbg != nullptr && dbg[0] == '1') c->use_tc = false;
+    }
+    int rc = dev_alloc(c, (void**)&c->status, sizeof(int), true, true);
+    if (rc == CITRUS_OK && c->use_tc && tc_init() != cudaSuccess) rc = CITRUS_ERR_UNSUPPORTED;
+    if (rc == CITRUS_OK) rc = alloc_units(c);
+    if (rc != CITRUS_OK) { free_all(c); delete c; return rc; }
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_live.insert(c);
+        g_dead.erase(c);
+    }
+    *out = c;
+    return CITRUS_OK;
+}
+
+int citrus_set_batch(citrus_handle h, int n_seq) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    if (n_seq < 1) return CITRUS_ERR_INVALID_ARG;
+    if (h->used) return CITRUS_ERR_STATE;
+    if (n_seq != h->n_slots) {
+        const int old = h->n_slots;
+        free_units(h);
+        h->n_slots = n_seq;
+        int rc = alloc_units(h);
+        if (rc != CITRUS_OK) {           // fall back to the geometry that worked before
+            free_units(h);
+            h->n_slots = old;
+            if (alloc_units(h) != CITRUS_OK) free_units(h);
+            return rc;
+        }
+    }
+    return CITRUS_OK;
+}
+
+int citrus_reset(citrus_handle h) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    for (Unit& u : h->units) {
+        u.m = 0; u.tokens_seen = 0; u.has_step = false;
+        u.last_n = u.last_kept = u.last_m = 0;
+    }
+    return CITRUS_OK;
+}
+
+int citrus_process_chunk_slot(citrus_handle h, int layer, int seq_slot,
+                              const void* Q_chunk, const void* K_chunk, const void* V_chunk, int n_tokens,
+                              const void* Q_instr, int n_instr, void* out, citrus_stream_t stream) {
+    int rc = check_process_args(h, layer, seq_slot, Q_chunk, K_chunk, V_chunk, n_tokens, Q_instr, n_instr, out);
+    if (rc) return rc;
+    if (!aligned16(Q_chunk) || !aligned16(K_chunk) || !aligned16(V_chunk) || !aligned16(Q_instr) || !aligned16(out))
+        return CITRUS_ERR_ALIGN;
+    return run_step(h, layer, seq_slot, Q_chunk, K_chunk, V_chunk, n_tokens, Q_instr, n_instr, out,
+                    reinterpret_cast<cudaStream_t>(stream));
+}
+
+int citrus_process_chunk(citrus_handle h, int layer,
+                         const void* Q_chunk, const void* K_chunk, const void* V_chunk, int n_tokens,
+                         const void* Q_instr, int n_instr, void* out, citrus_stream_t stream) {
+    return citrus_process_chunk_slot(h, layer, 0, Q_chunk, K_chunk, V_chunk, n_tokens, Q_instr, n_instr, out, stream);
+}
+
+int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,
+                              const void* Qh, const void* Kh, const void* Vh, int n_tokens,
+                              const void* Qih, int n_instr, void* out_h, citrus_stream_t stream) {
+    int rc = check_process_args(h, layer, seq_slot, Qh, Kh, Vh, n_tokens, Qih, n_instr, out_h);
+    if (rc) return rc;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t qrow = (size_t)h->Hq * h->D * h->elt, krow = (size_t)h->Hkv * h->D * h->elt;
+    if (h->stQ == nullptr) {
+        if ((rc = dev_alloc(h, &h->stQ, qrow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->stOut, qrow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->stK, krow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->stV, krow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->stQi, qrow * CITRUS_MAX_INSTR, false, true))) return rc;
+    }
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(h->stQ, Qh, qrow * n_tokens, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
+    if ((e = cudaMemcpyAsync(h->stK, Kh, krow * n_tokens, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
+    if ((e = cudaMemcpyAsync(h->stV, Vh, krow * n_tokens, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
+    if ((e = cudaMemcpyAsync(h->stQi, Qih, qrow * n_instr, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
+    rc = run_step(h, layer, seq_slot, h->stQ, h->stK, h->stV, n_tokens, h->stQi, n_instr, h->stOut, st);
+    if (rc) return rc;
+    if ((e = cudaMemcpyAsync(out_h, h->stOut, qrow * n_tokens, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_rc(e);
+    return cuda_rc(cudaStreamSynchronize(st));
+}
+
+int citrus_cache_view(citrus_handle h, int layer, int which, int seq_slot,
+                      const void** K, const void** V, const int** positions, int* n_rows) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= h->layers) return CITRUS_ERR_LAYER;
+    if (which < 0 || which >= h->n_caches || seq_slot < 0 || seq_slot >= h->n_slots) return CITRUS_ERR_INVALID_ARG;
+    if (h->units.empty()) return CITRUS_ERR_STATE;
+    const Unit& u = h->units[(size_t)layer * h->n_slots + seq_slot];
+    const CacheBufs& cb = u.cache[which];
+    if (K) *K = cb.K[cb.cur];
+    if (V) *V = cb.V[cb.cur];
+    if (positions) *positions = cb.pos[cb.cur];
+    if (n_rows) *n_rows = u.m;
+    return CITRUS_OK;
+}
+
+int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
+                     const float** scores, int* score_stride, const int** idx,
+                     int* n_candidates, int* n_kept, int* m_before) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= h->layers) return CITRUS_ERR_LAYER;
+    if (which < 0 || which >= h->n_caches || seq_slot < 0 || seq_slot >= h->n_slots) return CITRUS_ERR_INVALID_ARG;
+    if (h->units.empty()) return CITRUS_ERR_STATE;
+    const Unit& u = h->units[(size_t)layer * h->n_slots + seq_slot];
+    if (!u.has_step) return CITRUS_ERR_STATE;
+    if (scores) *scores = u.scores + (size_t)which * h->Hkv * h->score_stride;
+    if (score_stride) *score_stride = h->score_stride;
+    if (idx) *idx = u.idx + (size_t)which * h->Hkv * h->k;
+    if (n_candidates) *n_candidates = u.last_n;
+    if (n_kept) *n_kept = u.last_kept;
+    if (m_before) *m_before = u.last_m;
+    return CITRUS_OK;
+}
+
+int citrus_poll_status(citrus_handle h) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    int v = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
+    if (cudaMemcpy(&v, h->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
+    return v == 0 ? CITRUS_OK : CITRUS_ERR_TIMEOUT;
+}
+
+int citrus_destroy(citrus_handle h) {
+    if (h == nullptr) return CITRUS_OK;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (g_live.count(h) == 0) return g_dead.count(h) ? CITRUS_ERR_STATE : CITRUS_ERR_INVALID_ARG;
+        g_live.erase(h);
+        g_dead.insert(h);
+    }
+    cudaDeviceSynchronize();
+    free_all(h);
+    cudaGetLastError();
+    delete h;
+    return CITRUS_OK;
+}
+
+const char* citrus_strerror(int code) {
+    switch (code) {
+        case CITRUS_OK: return "ok";
+        case CITRUS_ERR_INVALID_ARG: return "invalid argument";
+        case CITRUS_ERR_SHAPE: return "size out of range";
+        case CITRUS_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case CITRUS_ERR_LAYER: return "layer index out of range";
+        case CITRUS_ERR_STATE: return "call not valid in this state";
+        case CITRUS_ERR_NOMEM: return "out of device memory";
+        case CITRUS_ERR_CUDA: return "CUDA runtime error";
+        case CITRUS_ERR_TIMEOUT: return "a bounded device wait expired";
+        case CITRUS_ERR_UNSUPPORTED: return "configuration not supported";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,190 @@
+// Step a3 (exact top-k with lower-index tie-break, ascending output) and step a4
+// (ordered gather of K, V and positions into the other ping-pong buffer).
+#include "citrus_internal.h"
+
+namespace citrus {
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kMaxJobs = 2;
+
+struct SelectArgs { SelectJob job[kMaxJobs]; };
+struct CompactArgs { CompactJob job[kMaxJobs]; };
+
+// Order-preserving map from fp32 to uint32 (larger float <=> larger key).
+__device__ __forceinline__ uint32_t order_key(float f) {
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// One CTA per (cache, KV head) -- or per cache when layerwise.  The score vector is
+// staged once in shared memory as order keys; a 4-pass most-significant-digit radix
+// select finds the k-th largest key T and how many candidates equal to T are kept;
+// a flagged block scan in index order then emits kept indices ascending, taking the
+// lowest-index candidates among those equal to T.
+__global__ void __launch_bounds__(kSelThreads)
+select_topk_kernel(SelectArgs args, int kv_heads, int n, int k, int layerwise) {
+    extern __shared__ uint32_t keys[];            // [n]
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t s_prefix, s_remaining;
+    __shared__ uint32_t warp_gt[32], warp_eq[32];
+
+    const SelectJob job = args.job[blockIdx.y];
+    const int g = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int heads_out = layerwise ? kv_heads : 1;
+    int* idx0 = job.idx + (size_t)g * k;
+
+    if (n <= k) {                                  // nothing to evict: identity
+        for (int j = tid; j < n; j += kSelThreads)
+            for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * k + j] = j;
+        return;
+    }
+    for (int j = tid; j < n; j += kSelThreads) {
+        float v;
+        if (layerwise) {
+            v = 0.f;
+            for (int gg = 0; gg < kv_heads; ++gg) v += job.scores[(size_t)gg * job.score_stride + j];
+        } else {
+            v = job.scores[(size_t)g * job.score_stride + j];
+        }
+        keys[j] = order_key(v);
+    }
+    if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; }
+    __syncthreads();
+
+    uint32_t mask = 0u;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        for (int j = tid; j < n; j += kSelThreads) {
+            uint32_t key = keys[j];
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t remaining = s_remaining, cum = 0u;
+            int b = 255;
+            for (; b > 0; --b) {
+                if (cum + hist[b] >= remaining) break;
+                cum += hist[b];
+            }
+            s_remaining = remaining - cum;          // still to take inside bin b
+            s_prefix = prefix | ((uint32_t)b << shift);
+        }
+        mask |= 255u << shift;
+        __syncthreads();
+    }
+    const uint32_t T = s_prefix;                   // k-th largest key
+    const uint32_t take_eq = s_remaining;          // candidates equal to T that are kept (lowest indices)
+
+    // ordered emission: thread t owns the contiguous index range [t*per, (t+1)*per)
+    const int per = (n + kSelThreads - 1) / kSelThreads;
+    const int lo = min(n, tid * per), hi = min(n, lo + per);
+    uint32_t gt = 0u, eq = 0u;
+    for (int j = lo; j < hi; ++j) { uint32_t key = keys[j]; gt += key > T; eq += key == T; }
+    // block exclusive scan of (gt, eq)
+    const int lane = tid & 31, warp = tid >> 5;
+    uint32_t sgt = gt, seq = eq;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t a = __shfl_up_sync(0xffffffffu, sgt, o), b = __shfl_up_sync(0xffffffffu, seq, o);
+        if (lane >= o) { sgt += a; seq += b; }
+    }
+    if (lane == 31) { warp_gt[warp] = sgt; warp_eq[warp] = seq; }
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t a = warp_gt[lane], b = warp_eq[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            uint32_t x = __shfl_up_sync(0xffffffffu, a, o), y = __shfl_up_sync(0xffffffffu, b, o);
+            if (lane >= o) { a += x; b += y; }
+        }
+        warp_gt[lane] = a; warp_eq[lane] = b;      // inclusive over warps
+    }
+    __syncthreads();
+    uint32_t gt_before = sgt - gt + (warp ? warp_gt[warp - 1] : 0u);
+    uint32_t eq_before = seq - eq + (warp ? warp_eq[warp - 1] : 0u);
+    for (int j = lo; j < hi; ++j) {
+        uint32_t key = keys[j];
+        bool keep = key > T || (key == T && eq_before < take_eq);
+        if (keep) {
+            uint32_t p = gt_before + min(eq_before, take_eq);
+            for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * k + p] = j;
+        }
+        gt_before += key > T;
+        eq_before += key == T;
+    }
+}
+
+// Rows are copied with 128-bit accesses, row_bytes/16 lanes per row.
+// grid: (row tiles, KV heads, caches)
+constexpr int kCompactThreads = 256;
+constexpr int kCompactRowsPerCta = 64;
+
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kv_kernel(CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
+                  int kv_heads, int cap, int row_vecs, int kept, int chunk_pos0) {
+    const CompactJob job = args.job[blockIdx.z];
+    const int g = blockIdx.y;
+    const int r_base = blockIdx.x * kCompactRowsPerCta;
+    const int rows_per_pass = kCompactThreads / row_vecs;
+    const int sub = threadIdx.x / row_vecs, v = threadIdx.x % row_vecs;
+    const int* idx = job.idx + (size_t)g * cap;
+    const uint4* srcK = reinterpret_cast<const uint4*>(job.srcK);
+    const uint4* srcV = reinterpret_cast<const uint4*>(job.srcV);
+    uint4* dstK = reinterpret_cast<uint4*>(job.dstK);
+    uint4* dstV = reinterpret_cast<uint4*>(job.dstV);
+    for (int rr = sub; rr < kCompactRowsPerCta; rr += rows_per_pass) {
+        const int r = r_base + rr;
+        if (r >= kept) break;
+        const int j = idx[r];
+        const uint4 *pk, *pv;
+        if (j < job.m) {
+            size_t off = ((size_t)g * cap + j) * row_vecs + v;
+            pk = srcK + off; pv = srcV + off;
+        } else {
+            size_t off = ((size_t)(j - job.m) * kv_heads + g) * row_vecs + v;
+            pk = chunkK + off; pv = chunkV + off;
+        }
+        uint4 a = __ldg(pk), b = __ldg(pv);
+        size_t doff = ((size_t)g * cap + r) * row_vecs + v;
+        dstK[doff] = a;
+        dstV[doff] = b;
+        if (v == 0) job.dstPos[(size_t)g * cap + r] = j < job.m ? job.srcPos[(size_t)g * cap + j] : chunk_pos0 + (j - job.m);
+    }
+}
+
+}  // namespace
+
+cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, int k, int layerwise, cudaStream_t s) {
+    if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
+    SelectArgs a;
+    for (int i = 0; i < n_jobs; ++i) a.job[i] = jobs[i];
+    static bool attr_set = false;
+    size_t smem = (size_t)n * sizeof(uint32_t);
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    dim3 grid(layerwise ? 1 : kv_heads, n_jobs);
+    select_topk_kernel<<<grid, kSelThreads, smem, s>>>(a, kv_heads, n, k, layerwise);
+    return cudaGetLastError();
+}
+
+cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
+                       int kv_heads, int cap, int row_bytes, int kept, int chunk_pos0, cudaStream_t s) {
+    if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
+    CompactArgs a;
+    for (int i = 0; i < n_jobs; ++i) a.job[i] = jobs[i];
+    int row_vecs = row_bytes / 16;
+    dim3 grid((kept + kCompactRowsPerCta - 1) / kCompactRowsPerCta, kv_heads, n_jobs);
+    compact_kv_kernel<<<grid, kCompactThreads, 0, s>>>(a, reinterpret_cast<const uint4*>(chunkK),
+                                                       reinterpret_cast<const uint4*>(chunkV),
+                                                       kv_heads, cap, row_vecs, kept, chunk_pos0);
+    return cudaGetLastError();
+}
+
+}  // namespace citrus

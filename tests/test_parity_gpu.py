@@ -1,0 +1,166 @@
+"""Parity of the CUDA path against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2406_12018_b200 import workloads as wl
+from paper_2406_12018_b200.binding import Citrus, CitrusError
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+C = wl.CONFIGS
+
+
+def _report(name, st):
+    print(f"\n[parity] {name}: chunks checked {st['checked_chunks']}, max |out err| {st['max_out_err']:.3e}, "
+          f"max normalised score err {st['max_score_err']:.3e}, max rel score err {st['max_score_rel']:.3e}, "
+          f"permitted near-tie flips {st['flips']}")
+
+
+def test_config1_tiny_fp32_full():
+    w = C["tiny_fp32"]
+    ctx = pu.make_pair(w)
+    doc, st = pu.run_document(w, ctx)
+    _report("tiny_fp32", st)
+    K, V, P = ctx.cache_view(0)
+    for g in range(w.kv_heads):
+        assert set(doc.planted.tolist()) <= set(P[g].tolist())
+    ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["shared", "individual"])
+@pytest.mark.parametrize("dtype,D", [("fp32", 64), ("fp32", 128), ("bf16", 128)])
+def test_small_ragged_shapes(mode, dtype, D):
+    # several tiles plus ragged tails; chunk lengths that are not multiples of any tile
+    w = wl.scaled(C["tiny_fp32"], q_heads=4, kv_heads=2, head_dim=D, budget_k=150, chunk_s=200, doc_tokens=777,
+                  n_instr=37, dtype=dtype, mode=mode, lm_window=19, n_planted=5, n_sinks=1)
+    ctx = pu.make_pair(w)
+    _, st = pu.run_document(w, ctx, chunk_lengths=[200, 1, 137, 200, 39, 200])
+    _report(f"ragged {mode} {dtype} D{D}", st)
+    ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_budget_not_reached_and_window_whole_chunk(dtype):
+    # budget larger than the document: nothing is ever evicted; LM window 0 = whole chunk
+    w = wl.scaled(C["tiny_fp32"], q_heads=4, kv_heads=4, head_dim=128, budget_k=600, chunk_s=128, doc_tokens=500,
+                  n_instr=5, dtype=dtype, mode="individual", lm_window=0)
+    ctx = pu.make_pair(w)
+    _, st = pu.run_document(w, ctx)
+    K, V, P = ctx.cache_view(0, 1)
+    assert P.shape[1] == 500 and torch.equal(P[0].cpu(), torch.arange(500, dtype=torch.int32))
+    ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_layerwise_granularity(dtype):
+    w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=4, head_dim=128, budget_k=96, chunk_s=160, doc_tokens=640,
+                  n_instr=12, dtype=dtype, mode="shared", n_planted=4)
+    ctx = pu.make_pair(w, layerwise=True)
+    _, st = pu.run_document(w, ctx, layerwise=True)
+    K, V, P = ctx.cache_view(0)
+    assert all(torch.equal(P[0], P[g]) for g in range(1, w.kv_heads))
+    ctx.close()
+
+
+def test_exact_ties_keep_lower_positions():
+    # identical keys -> identical scores: the kept set is the lowest positions
+    for dtype in ("fp32", "bf16"):
+        td = torch.float32 if dtype == "fp32" else torch.bfloat16
+        Hq, Hkv, D, k, N = 4, 2, 128, 40, 100
+        ctx = Citrus(1, Hq, Hkv, D, k, N, dtype=dtype)
+        g = torch.Generator().manual_seed(1)
+        Q = torch.randn(N, Hq, D, generator=g).to(td).cuda()
+        K = torch.randn(1, Hkv, D, generator=g).to(td).repeat(N, 1, 1).contiguous().cuda()
+        V = torch.randn(N, Hkv, D, generator=g).to(td).cuda()
+        Qi = torch.randn(3, Hq, D, generator=g).to(td).cuda()
+        ctx.process_chunk(0, Q, K, V, Qi)
+        torch.cuda.synchronize()
+        _, _, P = ctx.cache_view(0)
+        assert P.cpu().tolist() == [list(range(k))] * Hkv
+        ctx.close()
+
+
+def test_config2_mistral_layer_full_document():
+    w = C["mistral7b_layer"]
+    ctx = pu.make_pair(w)
+    doc, st = pu.run_document(w, ctx)
+    _report("mistral7b_layer", st)
+    K, V, P = ctx.cache_view(0)
+    for g in range(w.kv_heads):
+        kept = set(P[g].tolist())
+        assert set(doc.planted.tolist()) <= kept and set(doc.sinks.tolist()) <= kept
+    ctx.close()
+
+
+def test_config3_llama_stack_sampled():
+    w = C["llama2_7b_stack"]
+    layers = [0, 17, 31]
+    ctx = pu.make_pair(w, layers=w.layers)
+    st = {}
+    for layer in layers:
+        pu.run_document(w, ctx, layer=layer, oracle_chunks={0, 1, 15, 31} if layer == 0 else {31}, stats=st)
+    _report("llama2_7b_stack", st)
+    ctx.close()
+
+
+def test_config4_serving_mix_sampled():
+    w = C["serving_mix"]
+    lens = wl.sequence_lengths(w)
+    ctx = pu.make_pair(w)
+    st = {}
+    order = np.argsort(lens)
+    for seq in (int(order[0]), int(order[-1]), int(order[len(order) // 2])):
+        n_chunks = -(-lens[seq] // w.chunk_s)
+        pu.run_document(w, ctx, slot=seq, seq=seq, oracle_chunks={0, 1, n_chunks - 1}, stats=st)
+    _report("serving_mix", st)
+    ctx.close()
+
+
+def test_config5_long_document_sampled():
+    w = C["long_doc_stress"]
+    ctx = pu.make_pair(w)
+    doc, st = pu.run_document(w, ctx, oracle_chunks={0, 1, 31})
+    _report("long_doc_stress", st)
+    K, V, P = ctx.cache_view(0, 1)
+    for g in range(w.kv_heads):
+        kept = set(P[g].tolist())
+        assert set(doc.planted.tolist()) <= kept and set(doc.sinks.tolist()) <= kept
+    ctx.close()
+
+
+def test_host_buffer_variant_matches_device_variant():
+    w = wl.scaled(C["mistral7b_layer"], doc_tokens=2048)
+    doc = wl.make_document(w)
+    a, b = pu.make_pair(w), pu.make_pair(w)
+    for s in range(0, 2048, w.chunk_s):
+        sl = slice(s, s + w.chunk_s)
+        o1 = a.process_chunk(0, doc.Q[sl].cuda(), doc.K[sl].cuda(), doc.V[sl].cuda(), doc.Q_instr.cuda())
+        oh = torch.empty_like(doc.Q[sl]).pin_memory()
+        b.process_chunk_host(0, doc.Q[sl].pin_memory(), doc.K[sl].pin_memory(), doc.V[sl].pin_memory(),
+                             doc.Q_instr.pin_memory(), oh)
+        torch.cuda.synchronize()
+        assert torch.equal(o1.cpu(), oh)
+    Pa, Pb = a.cache_view(0)[2], b.cache_view(0)[2]
+    assert torch.equal(Pa, Pb)
+    a.close(); b.close()
+
+
+def test_reset_and_rerun_is_deterministic():
+    w = wl.scaled(C["mistral7b_layer"], doc_tokens=3000)
+    doc = wl.make_document(w)
+    ctx = pu.make_pair(w)
+    runs = []
+    for _ in range(2):
+        ctx.reset()
+        outs = []
+        for s in range(0, 3000, w.chunk_s):
+            sl = slice(s, min(3000, s + w.chunk_s))
+            outs.append(ctx.process_chunk(0, doc.Q[sl].cuda(), doc.K[sl].cuda(), doc.V[sl].cuda(), doc.Q_instr.cuda()))
+        torch.cuda.synchronize()
+        S, I, _ = ctx.step_view(0)
+        runs.append((torch.cat(outs).clone(), S.clone(), I.clone(), ctx.cache_view(0)[2].clone()))
+    for x, y in zip(*runs):
+        assert torch.equal(x, y)
+    assert ctx.poll_status() == 0
+    ctx.close()
