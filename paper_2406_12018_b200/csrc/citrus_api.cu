@@ -27,7 +27,6 @@ struct Unit {                       // one (layer, sequence slot)
     int* idx = nullptr;             // [n_caches, kv_heads, budget_k]
     float* lse_chunk = nullptr;     // [q_heads, chunk_s]
     float* lse_instr = nullptr;     // [q_heads, CITRUS_MAX_INSTR]
-    float* part = nullptr;          // tensor-core score pass partials
     int m = 0;                      // rows retained in every cache
     long long tokens_seen = 0;
     int last_n = 0, last_kept = 0, last_m = 0;
@@ -161,7 +160,7 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     }
     // a2-I: Eq. 1 with the instruction queries over the instruction-side cache's candidates
     if (c->use_tc) {
-        e = tc_score_lse(q_instr, cand[ic], u.part, u.part, u.lse_instr, CITRUS_MAX_INSTR, c->status, st);
+        e = tc_score_lse(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, c->status, st);
         if (e == cudaSuccess)
             e = tc_colsum(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, c->status, st);
     } else {

@@ -39,12 +39,11 @@ cudaError_t simt_colsum(bool is_fp32, int D, const QueryRows& q, const Candidate
                         const float* lse2, int lse_stride, float* scores, int score_stride, cudaStream_t s);
 
 // ---- tensor-core (tcgen05 / TMEM / TMA) path: bf16, D = 128 ----------------
-struct TcPlan;   // opaque per-call tensor maps, defined in tc_kernels.cu
 cudaError_t tc_init();   // resolves the driver entry point for tensor-map encoding
 cudaError_t tc_attention(const QueryRows& q, const Candidates& c, void* out, float* lse2, int lse_stride,
                          int* status, cudaStream_t s);
-cudaError_t tc_score_lse(const QueryRows& q, const Candidates& c, float* part_max, float* part_sum,
-                         float* lse2, int lse_stride, int* status, cudaStream_t s);
+cudaError_t tc_score_lse(const QueryRows& q, const Candidates& c, float* lse2, int lse_stride,
+                         int* status, cudaStream_t s);
 cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse2, int lse_stride,
                       float* scores, int score_stride, int* status, cudaStream_t s);
 

@@ -1,8 +1,670 @@
-// placeholder until the tcgen05 kernels land
+// Tensor-core path (bf16, head_dim 128) for steps a1 and a2 on sm_100a:
+// TMA (cp.async.bulk.tensor) stages 128-byte-swizzled tiles in shared memory,
+// tcgen05.mma accumulates in tensor memory, and the softmax / column-sum warps read
+// the accumulators back with tcgen05.ld.  Three kernels share the machinery:
+//
+//   attn_kernel<true>   a1: causal attention of the chunk over [cache ; chunk] (+ row LSE)
+//   attn_kernel<false>  a2 pass 1: row log-sum-exp of the scoring queries over all candidates
+//   colsum_kernel       a2 pass 2: S^T = K Q^T with the candidates on the accumulator's rows,
+//                       so the column sum of Eq. 1 over scoring rows is a per-thread sum
+//
+// Every wait on an mbarrier is bounded; a wait that expires raises the status word,
+// the CTA drains and returns (tensor memory is always released).
 #include "citrus_internal.h"
+
+#include <cuda.h>
+
 namespace citrus {
-cudaError_t tc_init() { return cudaErrorNotSupported; }
-cudaError_t tc_attention(const QueryRows&, const Candidates&, void*, float*, int, int*, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t tc_score_lse(const QueryRows&, const Candidates&, float*, float*, float*, int, int*, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t tc_colsum(const QueryRows&, const Candidates&, const float*, int, float*, int, int*, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kTile = 128;              // rows of every staged tile (queries, keys)
+constexpr int kD = 128;                 // head dimension
+constexpr int kHalfBytes = kTile * 128; // one [128 rows][64 bf16] swizzle-128B sub-tile
+constexpr int kTileBytes = 2 * kHalfBytes;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint64_t kWaitLimitNs = 1000000000ull;   // a bounded wait gives up after about one second
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false (and the status word raised) if the phase never completes.
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status) {
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < kWaitLimitNs) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity)) return true;
+        __nanosleep(128);
+    }
+    atomicExch(status, 1);
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+    for (int i = 0; i < 512; ++i)
+        if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, status);
+}
+// Same, with one outcome for the whole warp (the callers go on to warp-collective instructions).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, status));
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (base + i).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+          "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Shared-memory matrix descriptors (sm_100 format: version 1 at bit 46, 128-byte swizzle = 2 at bit 61).
+// K-major operand tile [rows][64 bf16]: 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// MN-major operand (V as B of P.V): [keys][64 bf16] sub-tiles; 8-key groups 1024 B apart (stride offset),
+// the two 64-wide halves of the head dimension kHalfBytes apart (leading offset).
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(kHalfBytes >> 4) << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ parameters
+struct TcParams {
+    int rows;        // query rows in the block
+    int row0;        // row offset of the block inside the Q tensor map
+    int q_heads, kv_heads;
+    int m, L;        // retained rows, chunk rows
+    int causal, t0;  // row r sees chunk keys u <= t0 + r
+    void* out;       // [rows, q_heads, 128] bf16 or null
+    float* lse2;     // [q_heads, lse_stride]
+    int lse_stride;
+    const float* lse_in;   // colsum: log-sum-exp of the scoring rows
+    float* scores;   // colsum: [kv_heads, score_stride]
+    int score_stride;
+    int* status;
+};
+
+// Load one 128x128 bf16 tile as two swizzled halves.  token_major: coordinates (d, head, row);
+// otherwise (cache layout) (d, row, head).
+__device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row, int head, bool token_major) {
+    if (token_major) {
+        tma_load_3d(dst, map, bar, 0, head, row);
+        tma_load_3d(dst + kHalfBytes, map, bar, 64, head, row);
+    } else {
+        tma_load_3d(dst, map, bar, 0, row, head);
+        tma_load_3d(dst + kHalfBytes, map, bar, 64, row, head);
+    }
+}
+
+// S[128 x n_cols] = A_tile . B_tile^T over the 128-wide head dimension (8 steps of 16).
+__device__ __forceinline__ void issue_qk(uint32_t tmem_d, uint32_t a_smem, uint32_t b_smem, uint32_t idesc) {
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+        uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+        mma_ss(tmem_d, desc_kmajor(a_smem + off), desc_kmajor(b_smem + off), idesc, kk > 0);
+    }
+}
+
+constexpr int kStages = 2;
+constexpr int kAttnThreads = 192;       // 4 softmax warps, 1 TMA warp, 1 MMA warp
+constexpr int kTmemCols = 512;
+constexpr float kRescaleTau = 8.f;      // rescale O only when the row max grows by more than 2^8
+
+struct AttnSmem {
+    uint64_t q_full, k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+    uint64_t s_full[2], p_full[2], o_done, drain;
+    uint32_t tmem_base;
+};
+constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + 2 * kStages) + 1024;
+
+// grid: (ceil(rows / 128), q_heads).  One CTA = 128 query rows of one head.
+template <bool WITH_PV>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
+            const __grid_constant__ CUtensorMap mapCV, const __grid_constant__ CUtensorMap mapSK,
+            const __grid_constant__ CUtensorMap mapSV, const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = base;
+    const uint32_t sK = sQ + kTileBytes;
+    const uint32_t sV = sK + kStages * kTileBytes;
+    AttnSmem* bars = reinterpret_cast<AttnSmem*>(smem_raw + (sV + kStages * kTileBytes - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int qt = blockIdx.x, h = blockIdx.y;
+    const int g = h / (p.q_heads / p.kv_heads);
+    const int q_row0 = qt * kTile;                                  // first row of this tile inside the block
+    const int n_cache_tiles = (p.m + kTile - 1) / kTile;
+    // chunk key tiles this query tile may see
+    int n_chunk_tiles = (p.L + kTile - 1) / kTile;
+    if (p.causal) {
+        int last_t = p.t0 + min(q_row0 + kTile, p.rows) - 1;         // highest chunk index among the rows
+        n_chunk_tiles = min(n_chunk_tiles, last_t / kTile + 1);
+    }
+    const int nt = n_cache_tiles + n_chunk_tiles;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars->q_full), 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1);
+            mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->p_full[b]), 128); }
+        mbar_init(smem_u32(&bars->o_done), 1);
+        mbar_init(smem_u32(&bars->drain), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 5) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+    auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
+    const uint32_t tmO = tmem + 256u;
+
+    if (warp == 4) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(smem_u32(&bars->q_full), kTileBytes);
+            load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
+            bool ok = true;
+            for (int j = 0; j < nt && ok; ++j) {
+                const int s = j % kStages;
+                const uint32_t ph = ((j / kStages) & 1) ^ 1;
+                const bool from_cache = j < n_cache_tiles;
+                const int row = from_cache ? j * kTile : (j - n_cache_tiles) * kTile;
+                ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph, p.status);
+                if (!ok) break;
+                mbar_expect_tx(smem_u32(&bars->k_full[s]), kTileBytes);
+                load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, g, !from_cache);
+                if (WITH_PV) {
+                    ok = mbar_wait(smem_u32(&bars->v_empty[s]), ph, p.status);
+                    if (!ok) break;
+                    mbar_expect_tx(smem_u32(&bars->v_full[s]), kTileBytes);
+                    load_tile(sV + s * kTileBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc(128, 0);
+            constexpr uint32_t idesc_pv = make_idesc(128, 1);
+            bool ok = mbar_wait(smem_u32(&bars->q_full), 0, p.status);
+            auto qk = [&](int j) -> bool {
+                const int s = j % kStages;
+                if (!mbar_wait(smem_u32(&bars->k_full[s]), (j / kStages) & 1, p.status)) return false;
+                tc_fence_after();
+                issue_qk(tmS(j & 1), sQ, sK + s * kTileBytes, idesc_qk);
+                mma_commit(smem_u32(&bars->s_full[j & 1]));
+                mma_commit(smem_u32(&bars->k_empty[s]));
+                return true;
+            };
+            if (ok && nt > 0) ok = qk(0);
+            if (ok && nt > 1) ok = qk(1);
+            for (int j = 0; j < nt && ok; ++j) {
+                // softmax has consumed S_j (and, with PV, written P_j over it)
+                ok = mbar_wait(smem_u32(&bars->p_full[j & 1]), (j >> 1) & 1, p.status);
+                if (!ok) break;
+                if (WITH_PV) {
+                    const int s = j % kStages;
+                    ok = mbar_wait(smem_u32(&bars->v_full[s]), (j / kStages) & 1, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t v_smem = sV + s * kTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)     // 16 keys per step: P columns 8*kk.., V rows 16*kk..
+                        mma_ts(tmO, tmS(j & 1) + kk * 8, desc_mnmajor(v_smem + kk * 2048), idesc_pv, (j > 0 || kk > 0));
+                    mma_commit(smem_u32(&bars->v_empty[s]));
+                    mma_commit(smem_u32(&bars->o_done));
+                }
+                if (j + 2 < nt) ok = qk(j + 2);
+            }
+            // all tensor-core work retired before tensor memory is released
+            mma_commit(smem_u32(&bars->drain));
+            mbar_wait(smem_u32(&bars->drain), 0, p.status);
+        }
+    } else {
+        // ---------------------------------------------------------------- softmax / epilogue (warps 0-3)
+        const int row_in_tile = warp * 32 + lane;
+        const int r = q_row0 + row_in_tile;                          // row inside the block
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const float scale2 = kLog2e * rsqrtf((float)kD);
+        float m_ref = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        uint32_t sreg[128];
+        for (int j = 0; j < nt; ++j) {
+            const int b = j & 1;
+            ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (j >> 1) & 1, p.status);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tmS(b) + lane_base + c * 32, sreg + c * 32);
+            tmem_wait_ld();
+            // number of visible columns of this tile for this row
+            int lim = kTile;
+            if (j < n_cache_tiles) {
+                lim = min(kTile, p.m - j * kTile);
+            } else {
+                const int u0 = (j - n_cache_tiles) * kTile;
+                lim = min(kTile, p.L - u0);
+                if (p.causal) lim = min(lim, p.t0 + r - u0 + 1);
+            }
+            float mx = -INFINITY;
+            if (lim >= kTile) {
+#pragma unroll
+                for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sreg[c]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < 128; ++c) {
+                    float v = c < lim ? __uint_as_float(sreg[c]) : -INFINITY;
+                    sreg[c] = __float_as_uint(v);
+                    mx = fmaxf(mx, v);
+                }
+            }
+            const float m_new = fmaxf(m_ref, mx * scale2);
+            if (j == 0) {
+                m_ref = m_new;
+            } else {
+                const bool grow = (m_new - m_ref) > kRescaleTau;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float f = ex2(m_ref - m_new);
+                    l_run *= f;
+                    m_ref = m_new;
+                    if (WITH_PV) {
+                        // O holds tiles 0..j-1 once P.V of tile j-1 has retired
+                        ok = mbar_wait_warp(smem_u32(&bars->o_done), (j - 1) & 1, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        uint32_t oreg[32];
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            tmem_ld32(tmO + lane_base + c * 32, oreg);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * f);
+                            tmem_st32(tmO + lane_base + c * 32, oreg);
+                        }
+                    }
+                }
+            }
+            // rows whose tile is fully masked keep m_ref = -inf only if nothing was visible so far;
+            // the first tile of every row has a visible column, so m_ref is finite here.
+            const float neg_m = -m_ref;
+            float sum = 0.f;
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t packed[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float p0 = ex2(fmaf(__uint_as_float(sreg[c4 * 32 + 2 * i]), scale2, neg_m));
+                    float p1 = ex2(fmaf(__uint_as_float(sreg[c4 * 32 + 2 * i + 1]), scale2, neg_m));
+                    sum += p0 + p1;
+                    packed[i] = pack_bf16(p0, p1);
+                }
+                if (WITH_PV) tmem_st16(tmS(b) + lane_base + c4 * 16, packed);
+            }
+            l_run += sum;
+            if (WITH_PV) tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->p_full[b]));
+        }
+        if (ok && nt > 0) {
+            if (WITH_PV) {
+                ok = mbar_wait_warp(smem_u32(&bars->o_done), (nt - 1) & 1, p.status);
+                if (ok) {
+                    tc_fence_after();
+                    const float inv = 1.f / l_run;
+                    __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + ((size_t)r * p.q_heads + h) * kD;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t oreg[32];
+                        tmem_ld32(tmO + lane_base + c * 32, oreg);
+                        tmem_wait_ld();
+                        if (r < p.rows) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                uint4 v;
+                                v.x = pack_bf16(__uint_as_float(oreg[8 * i + 0]) * inv, __uint_as_float(oreg[8 * i + 1]) * inv);
+                                v.y = pack_bf16(__uint_as_float(oreg[8 * i + 2]) * inv, __uint_as_float(oreg[8 * i + 3]) * inv);
+                                v.z = pack_bf16(__uint_as_float(oreg[8 * i + 4]) * inv, __uint_as_float(oreg[8 * i + 5]) * inv);
+                                v.w = pack_bf16(__uint_as_float(oreg[8 * i + 6]) * inv, __uint_as_float(oreg[8 * i + 7]) * inv);
+                                *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = v;
+                            }
+                        }
+                    }
+                }
+            }
+            if (ok && r < p.rows && p.lse2 != nullptr) p.lse2[(size_t)h * p.lse_stride + r] = m_ref + log2f(l_run);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+}
+
+// ------------------------------------------------------------------ column sums (a2 pass 2)
+constexpr int kColStages = 3;
+constexpr int kColTmemCols = 256;
+struct ColSmem {
+    uint64_t k_full, q_full[kColStages], q_empty[kColStages], s_full[2], s_free[2], drain;
+    uint32_t tmem_base;
+};
+constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 1024;
+
+// grid: (candidate tiles, kv_heads).  Accumulator rows = 128 candidates, columns = scoring rows of one
+// (head, row block); thread i owns candidate i and adds exp2(logit2 - lse2[row]) over its columns.
+__global__ void __launch_bounds__(kAttnThreads, 1)
+colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
+              const __grid_constant__ CUtensorMap mapSK, const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sK = base;
+    const uint32_t sQ = sK + kTileBytes;
+    ColSmem* bars = reinterpret_cast<ColSmem*>(smem_raw + (sQ + kColStages * kTileBytes - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kt = blockIdx.x, g = blockIdx.y;
+    const int G = p.q_heads / p.kv_heads;
+    const int n_cache_tiles = (p.m + kTile - 1) / kTile;
+    const bool from_cache = kt < n_cache_tiles;
+    const int key_row0 = from_cache ? kt * kTile : (kt - n_cache_tiles) * kTile;   // row in its source
+    const int n_rb = (p.rows + kTile - 1) / kTile;
+    // first row block that can see any key of this tile
+    int rb0 = 0;
+    if (p.causal && !from_cache && key_row0 > p.t0) rb0 = (key_row0 - p.t0) / kTile;
+    const int nb = G * (n_rb - rb0);                  // (head, row block) iterations
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars->k_full), 1);
+        for (int s = 0; s < kColStages; ++s) { mbar_init(smem_u32(&bars->q_full[s]), 1); mbar_init(smem_u32(&bars->q_empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 128); }
+        mbar_init(smem_u32(&bars->drain), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 5) tmem_alloc(smem_u32(&bars->tmem_base), kColTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+    auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
+
+    if (warp == 4) {
+        if (lane == 0) {
+            mbar_expect_tx(smem_u32(&bars->k_full), kTileBytes);
+            load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
+            for (int it = 0; it < nb; ++it) {
+                const int s = it % kColStages;
+                const int h = g * G + it / (n_rb - rb0);
+                const int rb = rb0 + it % (n_rb - rb0);
+                if (!mbar_wait(smem_u32(&bars->q_empty[s]), ((it / kColStages) & 1) ^ 1, p.status)) break;
+                mbar_expect_tx(smem_u32(&bars->q_full[s]), kTileBytes);
+                load_tile(sQ + s * kTileBytes, &mapQ, smem_u32(&bars->q_full[s]), p.row0 + rb * kTile, h, true);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            bool ok = mbar_wait(smem_u32(&bars->k_full), 0, p.status);
+            for (int it = 0; it < nb && ok; ++it) {
+                const int s = it % kColStages, b = it & 1;
+                const int rb = rb0 + it % (n_rb - rb0);
+                const int ncols = min(kTile, ((p.rows - rb * kTile) + 15) & ~15);
+                ok = mbar_wait(smem_u32(&bars->q_full[s]), (it / kColStages) & 1, p.status);
+                if (!ok) break;
+                ok = mbar_wait(smem_u32(&bars->s_free[b]), ((it >> 1) & 1) ^ 1, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_qk(tmS(b), sK, sQ + s * kTileBytes, make_idesc(ncols, 0));
+                mma_commit(smem_u32(&bars->s_full[b]));
+                mma_commit(smem_u32(&bars->q_empty[s]));
+            }
+            mma_commit(smem_u32(&bars->drain));
+            mbar_wait(smem_u32(&bars->drain), 0, p.status);
+        }
+    } else {
+        const int key_in_tile = warp * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const float scale2 = kLog2e * rsqrtf((float)kD);
+        const int j = kt < n_cache_tiles ? key_row0 + key_in_tile : p.m + key_row0 + key_in_tile;   // candidate index
+        const int n_src = from_cache ? p.m : p.L;
+        const bool key_ok = key_row0 + key_in_tile < n_src;
+        // first scoring row that may see this candidate
+        int r_first = 0;
+        if (p.causal && !from_cache) r_first = max(0, key_row0 + key_in_tile - p.t0);
+        float acc = 0.f;
+        bool ok = true;
+        uint32_t sreg[128];
+        for (int it = 0; it < nb; ++it) {
+            const int b = it & 1;
+            const int h = g * G + it / (n_rb - rb0);
+            const int rb = rb0 + it % (n_rb - rb0);
+            const int r0 = rb * kTile;
+            const int ncols = min(kTile, p.rows - r0);
+            ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 1) & 1, p.status);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (c * 32 < ncols) tmem_ld32(tmS(b) + lane_base + c * 32, sreg + c * 32);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->s_free[b]));
+            const float* lse = p.lse_in + (size_t)h * p.lse_stride + r0;
+            const int c_lo = max(0, r_first - r0);
+            float part = 0.f;
+#pragma unroll
+            for (int c = 0; c < 128; ++c) {
+                if (c < ncols) {
+                    float e = ex2(fmaf(__uint_as_float(sreg[c]), scale2, -__ldg(lse + c)));
+                    part += c >= c_lo ? e : 0.f;
+                }
+            }
+            acc += part;
+        }
+        if (ok && key_ok) p.scores[(size_t)g * p.score_stride + j] = acc;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem, kColTmemCols);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn g_encode = nullptr;
+
+// Token-major tensor [rows, heads, 128] bf16: coordinates (d, head, row), box 64 x 1 x 128.
+bool map_token_major(CUtensorMap* map, const void* ptr, int rows, int heads) {
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)heads, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)heads * kD * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)kTile};
+    cuuint32_t es[3] = {1, 1, 1};
+    return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// Cache tensor [heads, cap, 128] bf16: coordinates (d, row, head), box 64 x 128 x 1.
+bool map_cache(CUtensorMap* map, const void* ptr, int cap, int heads) {
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)cap, (cuuint64_t)heads};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)cap * kD * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)kTile, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Maps { CUtensorMap Q, CK, CV, SK, SV; };
+
+// The tensor map's row extent is the number of valid rows, so rows past it read as zero.
+bool build_maps(Maps* mp, const void* Qbase, int q_rows_total, const QueryRows& q, const Candidates& c, bool with_v) {
+    if (!map_token_major(&mp->Q, Qbase, q_rows_total, q.q_heads)) return false;
+    if (!map_cache(&mp->CK, c.cacheK, c.cap, c.kv_heads)) return false;
+    if (!map_token_major(&mp->SK, c.chunkK, c.L, c.kv_heads)) return false;
+    if (with_v) {
+        if (!map_cache(&mp->CV, c.cacheV, c.cap, c.kv_heads)) return false;
+        if (!map_token_major(&mp->SV, c.chunkV, c.L, c.kv_heads)) return false;
+    } else {
+        mp->CV = mp->CK; mp->SV = mp->SK;
+    }
+    return true;
+}
+
+TcParams base_params(const QueryRows& q, const Candidates& c, int* status) {
+    TcParams p{};
+    p.rows = q.rows; p.row0 = 0; p.q_heads = q.q_heads; p.kv_heads = c.kv_heads;
+    p.m = c.m; p.L = c.L; p.causal = q.causal; p.t0 = q.t0; p.status = status;
+    return p;
+}
+
+}  // namespace
+
+cudaError_t tc_init() {
+    if (g_encode != nullptr) return cudaSuccess;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+    g_encode = reinterpret_cast<EncodeFn>(fn);
+    e = cudaFuncSetAttribute(attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kColSmemBytes);
+}
+
+cudaError_t tc_attention(const QueryRows& q, const Candidates& c, void* out, float* lse2, int lse_stride,
+                         int* status, cudaStream_t s) {
+    Maps mp;
+    if (!build_maps(&mp, q.Q, q.rows, q, c, true)) return cudaErrorInvalidValue;
+    TcParams p = base_params(q, c, status);
+    p.out = out; p.lse2 = lse2; p.lse_stride = lse_stride;
+    dim3 grid((q.rows + kTile - 1) / kTile, q.q_heads);
+    attn_kernel<true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
+    return cudaGetLastError();
+}
+
+cudaError_t tc_score_lse(const QueryRows& q, const Candidates& c, float* lse2, int lse_stride,
+                         int* status, cudaStream_t s) {
+    Maps mp;
+    if (!build_maps(&mp, q.Q, q.rows, q, c, false)) return cudaErrorInvalidValue;
+    TcParams p = base_params(q, c, status);
+    p.out = nullptr; p.lse2 = lse2; p.lse_stride = lse_stride;
+    dim3 grid((q.rows + kTile - 1) / kTile, q.q_heads);
+    attn_kernel<false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
+    return cudaGetLastError();
+}
+
+cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse2, int lse_stride,
+                      float* scores, int score_stride, int* status, cudaStream_t s) {
+    Maps mp;
+    if (!build_maps(&mp, q.Q, q.rows, q, c, false)) return cudaErrorInvalidValue;
+    TcParams p = base_params(q, c, status);
+    p.lse_in = lse2; p.lse_stride = lse_stride; p.scores = scores; p.score_stride = score_stride;
+    const int n_tiles = (c.m + kTile - 1) / kTile + (c.L + kTile - 1) / kTile;
+    dim3 grid(n_tiles, c.kv_heads);
+    colsum_kernel<<<grid, kAttnThreads, kColSmemBytes, s>>>(mp.Q, mp.CK, mp.SK, p);
+    return cudaGetLastError();
+}
+
+}  // namespace citrus
