@@ -147,6 +147,23 @@ int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
                      const float** scores, int* score_stride, const int** idx,
                      int* n_candidates, int* n_kept, int* m_before);
 
+/*
+ * Measurement aid for the roofline figures (kernel time of a1 / a2 / a3 / a4 taken
+ * separately).  While enabled, every kernel launch of a process call is bracketed by
+ * CUDA events recorded on the call's stream (do not enable during stream capture).
+ * citrus_profile_read synchronises the device, adds up the elapsed milliseconds and
+ * the number of launches per kernel id since the last read into ms[CITRUS_N_KERNELS]
+ * and launches[CITRUS_N_KERNELS] (host arrays), and clears the record.
+ */
+#define CITRUS_KERNEL_ATTENTION 0   /* a1 */
+#define CITRUS_KERNEL_SCORE_LSE 1   /* a2, log-sum-exp pass of the instruction queries */
+#define CITRUS_KERNEL_COLSUM    2   /* a2, column sums (instruction and LM) */
+#define CITRUS_KERNEL_SELECT    3   /* a3 */
+#define CITRUS_KERNEL_COMPACT   4   /* a4 */
+#define CITRUS_N_KERNELS        5
+int citrus_profile(citrus_handle h, int enable);
+int citrus_profile_read(citrus_handle h, double* ms, long long* launches);
+
 /* Reads the device status word (0, or CITRUS_ERR_TIMEOUT if a bounded wait in a
  * kernel gave up). Synchronises the device. */
 int citrus_poll_status(citrus_handle h);

@@ -22,9 +22,12 @@ MODE_LAYERWISE = 4
 MAX_INSTR = 4096
 MAX_CANDIDATES = 49152
 
+KERNEL_NAMES = ["attention", "score_lse", "colsum", "select", "compact"]
+
 EXPORTS = [
     "citrus_create", "citrus_set_batch", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
-    "citrus_process_chunk_host", "citrus_cache_view", "citrus_step_view", "citrus_poll_status",
+    "citrus_process_chunk_host", "citrus_cache_view", "citrus_step_view", "citrus_profile",
+    "citrus_profile_read", "citrus_poll_status",
     "citrus_destroy", "citrus_strerror",
 ]
 
@@ -56,6 +59,8 @@ def load() -> C.CDLL:
     lib.citrus_cache_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(i)]
     lib.citrus_step_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(i), C.POINTER(vp),
                                      C.POINTER(i), C.POINTER(i), C.POINTER(i)]
+    lib.citrus_profile.argtypes = [vp, i]
+    lib.citrus_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     lib.citrus_poll_status.argtypes = [vp]
     lib.citrus_destroy.argtypes = [vp]
     lib.citrus_strerror.argtypes = [i]
@@ -165,6 +170,20 @@ class Citrus:
         St = _view(S.value, (self.kv_heads, stride.value), "<f4", 4)[:, :n.value]
         It = _view(I.value, (self.kv_heads, self.budget_k), "<i4", 4)[:, :kept.value]
         return St, It, m.value
+
+    def profile(self, enable: bool):
+        rc = load().citrus_profile(self._h, 1 if enable else 0)
+        if rc != 0:
+            raise CitrusError(rc, "citrus_profile")
+
+    def profile_read(self):
+        """{kernel name: (total ms, launches)} since the last read."""
+        ms = (C.c_double * len(KERNEL_NAMES))()
+        cnt = (C.c_longlong * len(KERNEL_NAMES))()
+        rc = load().citrus_profile_read(self._h, ms, cnt)
+        if rc != 0:
+            raise CitrusError(rc, "citrus_profile_read")
+        return {n: (ms[i], cnt[i]) for i, n in enumerate(KERNEL_NAMES)}
 
     def reset(self):
         rc = load().citrus_reset(self._h)

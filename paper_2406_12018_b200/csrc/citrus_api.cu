@@ -49,6 +49,10 @@ struct citrus_ctx {
     std::vector<void*> allocs;      // cache buffers and per-unit scratch
     std::vector<void*> misc;        // status word, host-variant staging
     int* status = nullptr;
+    // optional per-launch timing: (kernel id, start, stop) event pairs recorded on the launching stream
+    bool profiling = false;
+    struct Timed { int id; cudaEvent_t a, b; };
+    std::vector<Timed> timed;
     // staging of the host-buffer variant
     void *stQ = nullptr, *stK = nullptr, *stV = nullptr, *stQi = nullptr, *stOut = nullptr;
 };
@@ -124,6 +128,20 @@ int check_process_args(citrus_ctx* h, int layer, int slot, const void* Q, const 
     return CITRUS_OK;
 }
 
+struct LaunchTimer {                 // brackets one kernel launch with events when profiling is on
+    citrus_ctx* c; cudaStream_t st; cudaEvent_t a = nullptr, b = nullptr; int id;
+    LaunchTimer(citrus_ctx* c_, int id_, cudaStream_t st_) : c(c_), st(st_), id(id_) {
+        if (!c->profiling) return;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { a = b = nullptr; cudaGetLastError(); return; }
+        cudaEventRecord(a, st);
+    }
+    ~LaunchTimer() {
+        if (a == nullptr) return;
+        cudaEventRecord(b, st);
+        c->timed.push_back(citrus_ctx::Timed{id, a, b});
+    }
+};
+
 // The launch sequence of one chunk step; all pointers are device pointers.
 int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc, const void* Vc, int L,
              const void* Qi, int nI, void* out, cudaStream_t st) {
@@ -145,8 +163,11 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
 
     cudaError_t e;
     // a1: attention of the chunk over [cache 0 ; chunk], row log-sum-exp kept for a2-L
-    if (c->use_tc) e = tc_attention(q_chunk, cand[0], out, u.lse_chunk, c->ls, c->status, st);
-    else e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, u.lse_chunk, c->ls, st);
+    {
+        LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
+        if (c->use_tc) e = tc_attention(q_chunk, cand[0], out, u.lse_chunk, c->ls, c->status, st);
+        else e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, u.lse_chunk, c->ls, st);
+    }
     if (e != cudaSuccess) return cuda_rc(e);
 
     // a2-L (individual design): votes of the chunk's last w queries on cache 0's candidates
@@ -154,19 +175,22 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         int w = c->lm_window > 0 && c->lm_window < L ? c->lm_window : L;
         const char* q0 = reinterpret_cast<const char*>(Qc) + (size_t)(L - w) * c->Hq * c->D * c->elt;
         QueryRows q_lm{q0, w, c->Hq, 1, L - w};
+        LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
         if (c->use_tc) e = tc_colsum(q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, c->status, st);
         else e = simt_colsum(c->fp32, c->D, q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, st);
         if (e != cudaSuccess) return cuda_rc(e);
     }
     // a2-I: Eq. 1 with the instruction queries over the instruction-side cache's candidates
-    if (c->use_tc) {
-        e = tc_score_lse(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, c->status, st);
-        if (e == cudaSuccess)
-            e = tc_colsum(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, c->status, st);
-    } else {
-        e = simt_attention(c->fp32, c->D, q_instr, cand[ic], nullptr, u.lse_instr, CITRUS_MAX_INSTR, st);
-        if (e == cudaSuccess)
-            e = simt_colsum(c->fp32, c->D, q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, st);
+    {
+        LaunchTimer t(c, CITRUS_KERNEL_SCORE_LSE, st);
+        if (c->use_tc) e = tc_score_lse(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, c->status, st);
+        else e = simt_attention(c->fp32, c->D, q_instr, cand[ic], nullptr, u.lse_instr, CITRUS_MAX_INSTR, st);
+    }
+    if (e != cudaSuccess) return cuda_rc(e);
+    {
+        LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
+        if (c->use_tc) e = tc_colsum(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, c->status, st);
+        else e = simt_colsum(c->fp32, c->D, q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, st);
     }
     if (e != cudaSuccess) return cuda_rc(e);
 
@@ -180,9 +204,15 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
                             cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, m};
     }
-    e = select_topk(sj, c->n_caches, c->Hkv, n, c->k, c->layerwise ? 1 : 0, st);
+    {
+        LaunchTimer t(c, CITRUS_KERNEL_SELECT, st);
+        e = select_topk(sj, c->n_caches, c->Hkv, n, c->k, c->layerwise ? 1 : 0, st);
+    }
     if (e != cudaSuccess) return cuda_rc(e);
-    e = compact_kv(cj, c->n_caches, Kc, Vc, c->Hkv, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
+    {
+        LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
+        e = compact_kv(cj, c->n_caches, Kc, Vc, c->Hkv, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
+    }
     if (e != cudaSuccess) return cuda_rc(e);
 
     for (int ci = 0; ci < c->n_caches; ++ci) u.cache[ci].cur ^= 1;
@@ -340,6 +370,27 @@ int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
     return CITRUS_OK;
 }
 
+int citrus_profile(citrus_handle h, int enable) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    h->profiling = enable != 0;
+    return CITRUS_OK;
+}
+
+int citrus_profile_read(citrus_handle h, double* ms, long long* launches) {
+    if (h == nullptr || !is_live(h) || ms == nullptr || launches == nullptr) return CITRUS_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
+    for (int i = 0; i < CITRUS_N_KERNELS; ++i) { ms[i] = 0.0; launches[i] = 0; }
+    for (const citrus_ctx::Timed& t : h->timed) {
+        float f = 0.f;
+        if (cudaEventElapsedTime(&f, t.a, t.b) == cudaSuccess) { ms[t.id] += f; launches[t.id] += 1; }
+        else cudaGetLastError();
+        cudaEventDestroy(t.a);
+        cudaEventDestroy(t.b);
+    }
+    h->timed.clear();
+    return CITRUS_OK;
+}
+
 int citrus_poll_status(citrus_handle h) {
     if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
     int v = 0;
@@ -357,6 +408,7 @@ int citrus_destroy(citrus_handle h) {
         g_dead.insert(h);
     }
     cudaDeviceSynchronize();
+    for (const citrus_ctx::Timed& t : h->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     free_all(h);
     cudaGetLastError();
     delete h;

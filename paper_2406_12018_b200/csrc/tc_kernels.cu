@@ -327,7 +327,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
         const int r = q_row0 + row_in_tile;                          // row inside the block
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         const float scale2 = kLog2e * rsqrtf((float)kD);
-        float m_ref = -INFINITY, l_run = 0.f;
+        float m_ref = -INFINITY, l_run = 0.f, l_out = 0.f;
         bool ok = true;
         uint32_t sreg[128];
         for (int j = 0; j < nt; ++j) {
@@ -367,6 +367,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                 if (__any_sync(0xffffffffu, grow)) {
                     const float f = ex2(m_ref - m_new);
                     l_run *= f;
+                    l_out *= f;
                     m_ref = m_new;
                     if (WITH_PV) {
                         // O holds tiles 0..j-1 once P.V of tile j-1 has retired
@@ -387,8 +388,11 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
             }
             // rows whose tile is fully masked keep m_ref = -inf only if nothing was visible so far;
             // the first tile of every row has a visible column, so m_ref is finite here.
+            // l_run sums the fp32 probabilities (it feeds the log-sum-exp that a2-L reuses); l_out sums
+            // the bf16-rounded ones that P.V actually multiplies, so that out = sum(p~ v) / sum(p~) stays a
+            // convex combination of V rows even when one key takes nearly all of the mass.
             const float neg_m = -m_ref;
-            float sum = 0.f;
+            float sum = 0.f, sum_r = 0.f;
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
                 uint32_t packed[16];
@@ -398,20 +402,26 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                     float p1 = ex2(fmaf(__uint_as_float(sreg[c4 * 32 + 2 * i + 1]), scale2, neg_m));
                     sum += p0 + p1;
                     packed[i] = pack_bf16(p0, p1);
+                    if (WITH_PV) sum_r += __uint_as_float(packed[i] << 16) + __uint_as_float(packed[i] & 0xffff0000u);
                 }
                 if (WITH_PV) tmem_st16(tmS(b) + lane_base + c4 * 16, packed);
             }
             l_run += sum;
+            l_out += sum_r;
             if (WITH_PV) tmem_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&bars->p_full[b]));
         }
         if (ok && nt > 0) {
             if (WITH_PV) {
-                ok = mbar_wait_warp(smem_u32(&bars->o_done), (nt - 1) & 1, p.status);
+                // o_done completes one phase per tile.  Only tiles 0..nt-3 are known to have retired here
+                // (their P.V precedes the last S tile in issue order), so wait for tile nt-2 first: a
+                // parity wait alone cannot tell "tile nt-1 done" from "tile nt-2 still running".
+                if (nt > 1) ok = mbar_wait_warp(smem_u32(&bars->o_done), (nt - 2) & 1, p.status);
+                if (ok) ok = mbar_wait_warp(smem_u32(&bars->o_done), (nt - 1) & 1, p.status);
                 if (ok) {
                     tc_fence_after();
-                    const float inv = 1.f / l_run;
+                    const float inv = 1.f / l_out;
                     __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + ((size_t)r * p.q_heads + h) * kD;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -437,7 +447,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 5) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
 }
 
 // ------------------------------------------------------------------ column sums (a2 pass 2)
@@ -563,7 +573,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem, kColTmemCols);
+    if (warp == 5) { __syncwarp(); tmem_dealloc(tmem, kColTmemCols); }
 }
 
 // ------------------------------------------------------------------ host side
