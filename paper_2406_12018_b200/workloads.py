@@ -104,7 +104,11 @@ def _orthonormal_pair(rng, D):
 
 def make_document(w: Workload, layer: int = 0, seq: int = 0, n_tokens: Optional[int] = None) -> Document:
     """Draw one (layer, sequence) document of workload w on the CPU."""
-    N = n_tokens if n_tokens is not None else sequence_lengths(w)[seq]
+    if n_tokens is not None:
+        N = n_tokens
+    else:
+        lens = sequence_lengths(w)
+        N = lens[seq] if seq < len(lens) else w.doc_tokens      # further sequences of a fixed-length workload
     Hq, Hkv, D = w.q_heads, w.kv_heads, w.head_dim
     G = Hq // Hkv
     rng = np.random.Generator(np.random.Philox(key=[w.seed * 1000 + layer, seq]))
