@@ -164,6 +164,42 @@ int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
 int citrus_profile(citrus_handle h, int enable);
 int citrus_profile_read(citrus_handle h, double* ms, long long* launches);
 
+/*
+ * Importance scoring without any allocation.  The paper has no counterpart: this exists for
+ * callers that must not (or cannot) allocate device memory -- a serving loop that has handed the
+ * whole GPU to its own memory pool so that cudaMalloc fails or stalls every stream with its
+ * device-wide synchronisation, a plug-in that is only allowed to launch work on streams it is
+ * given, or code that may run while another thread holds an allocator lock.
+ *
+ * Computes the same quantity as step a2-I of citrus_process_chunk on an empty cache:
+ *   scores[g][j] = sum over heads h of KV group g, and over the n_s scoring rows i, of
+ *                  softmax_j( Q_s[i,h] . K[j,g] / sqrt(head_dim) ),     j < n_keys,
+ * with Q_s [n_s, q_heads, head_dim] and K [n_keys, kv_heads, head_dim] token-major device
+ * tensors (bf16, or fp32 with CITRUS_MODE_FP32 as the only accepted mode bit) and scores
+ * [kv_heads, score_stride] fp32 device memory, all owned by the caller.  No context is needed.
+ *
+ * The intermediate log-sum-exp of every (head, row) lives in a fixed array of
+ * CITRUS_STATIC_MAX_LSE floats (256 KB, plus a 256-byte status word) that is part of the
+ * library image: every GPU that loads the library holds it until the process exits.  Limits:
+ * q_heads * round_up(n_s, 4) <= CITRUS_STATIC_MAX_LSE, n_s <= CITRUS_MAX_INSTR,
+ * n_keys <= CITRUS_MAX_CANDIDATES; head_dim 128 (bf16) or 64/128 (fp32).  Larger sizes return
+ * CITRUS_ERR_SHAPE and launch nothing.  The function never calls cudaMalloc, cudaFree or any
+ * allocating routine.
+ *
+ * The first call on a device looks up the array's device address (and, for bf16, resolves the
+ * tensor-map encoder and raises the kernels' shared-memory limits); make that first call
+ * outside of any stream capture.  All calls on a device share the one array and overwrite it:
+ * two calls whose GPU work overlaps (different streams, or different threads) race; run them
+ * on one stream or order them with events.  device_status may be NULL; otherwise it is a
+ * caller-owned device int, zeroed by the caller, set to 1 if a bounded wait inside a kernel
+ * expires.
+ */
+#define CITRUS_STATIC_MAX_LSE 65536
+int citrus_importance_static(const void* Q_s, int n_s, const void* K, int n_keys,
+                             int q_heads, int kv_heads, int head_dim, unsigned mode,
+                             float* scores, int score_stride, int* device_status,
+                             citrus_stream_t stream);
+
 /* Reads the device status word (0, or CITRUS_ERR_TIMEOUT if a bounded wait in a
  * kernel gave up). Synchronises the device. */
 int citrus_poll_status(citrus_handle h);

@@ -27,7 +27,7 @@ KERNEL_NAMES = ["attention", "score_lse", "colsum", "select", "compact"]
 EXPORTS = [
     "citrus_create", "citrus_set_batch", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
     "citrus_process_chunk_host", "citrus_cache_view", "citrus_step_view", "citrus_profile",
-    "citrus_profile_read", "citrus_poll_status",
+    "citrus_profile_read", "citrus_importance_static", "citrus_poll_status",
     "citrus_destroy", "citrus_strerror",
 ]
 
@@ -61,6 +61,7 @@ def load() -> C.CDLL:
                                      C.POINTER(i), C.POINTER(i), C.POINTER(i)]
     lib.citrus_profile.argtypes = [vp, i]
     lib.citrus_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
+    lib.citrus_importance_static.argtypes = [vp, i, vp, i, i, i, i, C.c_uint, vp, i, vp, vp]
     lib.citrus_poll_status.argtypes = [vp]
     lib.citrus_destroy.argtypes = [vp]
     lib.citrus_strerror.argtypes = [i]
@@ -74,6 +75,20 @@ def load() -> C.CDLL:
 
 def strerror(code: int) -> str:
     return load().citrus_strerror(code).decode()
+
+
+def importance_static(Q_s: torch.Tensor, K: torch.Tensor, scores: torch.Tensor, stream=None) -> torch.Tensor:
+    """Eq. 1 column sums of scoring rows Q_s [n_s, H_q, D] over keys K [n, H_kv, D] into the caller's
+    `scores` [H_kv, >= n] fp32, through the entry point that allocates nothing (see citrus.h)."""
+    assert Q_s.is_cuda and K.is_cuda and scores.is_cuda and scores.dtype == torch.float32
+    assert Q_s.is_contiguous() and K.is_contiguous() and scores.is_contiguous() and Q_s.dtype == K.dtype
+    mode = MODE_FP32 if Q_s.dtype == torch.float32 else 0
+    rc = load().citrus_importance_static(Q_s.data_ptr(), Q_s.shape[0], K.data_ptr(), K.shape[0], Q_s.shape[1],
+                                         K.shape[1], Q_s.shape[2], mode, scores.data_ptr(), scores.shape[1],
+                                         None, _stream_ptr(stream))
+    if rc != 0:
+        raise CitrusError(rc, "citrus_importance_static")
+    return scores
 
 
 class _DevView:

@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcitrus.so")
-SOURCES = ["citrus_api.cu", "simt_kernels.cu", "select_compact.cu", "tc_kernels.cu"]
+SOURCES = ["citrus_api.cu", "simt_kernels.cu", "select_compact.cu", "tc_kernels.cu", "citrus_static.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 
