@@ -165,8 +165,9 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     // a1: attention of the chunk over [cache 0 ; chunk], row log-sum-exp kept for a2-L
     {
         LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
-        if (c->use_tc) e = tc_attention(q_chunk, cand[0], out, u.lse_chunk, c->ls, c->status, st);
-        else e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, u.lse_chunk, c->ls, st);
+        float* lse_chunk = c->individual ? u.lse_chunk : nullptr;     // only a2-L reads it
+        if (c->use_tc) e = tc_attention(q_chunk, cand[0], out, lse_chunk, c->ls, c->status, st);
+        else e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, lse_chunk, c->ls, st);
     }
     if (e != cudaSuccess) return cuda_rc(e);
 

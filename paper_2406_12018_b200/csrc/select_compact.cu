@@ -63,15 +63,29 @@ select_topk_kernel(SelectArgs args, int kv_heads, int n, int k, int layerwise) {
             if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
         }
         __syncthreads();
-        if (tid == 0) {
-            uint32_t remaining = s_remaining, cum = 0u;
-            int b = 255;
-            for (; b > 0; --b) {
-                if (cum + hist[b] >= remaining) break;
-                cum += hist[b];
+        if (tid < 32) {
+            // warp 0 walks the 256 bins from the top: lane l owns bins [8l, 8l+8)
+            const uint32_t remaining = s_remaining;
+            uint32_t mine = 0u;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) mine += hist[tid * 8 + i];
+            uint32_t suffix = mine;                              // inclusive sum over lanes >= tid
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                uint32_t v = __shfl_down_sync(0xffffffffu, suffix, o);
+                if (tid + o < 32) suffix += v;
             }
-            s_remaining = remaining - cum;          // still to take inside bin b
-            s_prefix = prefix | ((uint32_t)b << shift);
+            const uint32_t above = suffix - mine;                // candidates in bins of higher lanes
+            if (above < remaining && remaining <= suffix) {      // exactly one lane holds the k-th largest
+                uint32_t cum = above;
+                int b = tid * 8 + 7;
+                for (; b > tid * 8; --b) {
+                    if (cum + hist[b] >= remaining) break;
+                    cum += hist[b];
+                }
+                s_remaining = remaining - cum;                   // still to take inside bin b
+                s_prefix = prefix | ((uint32_t)b << shift);
+            }
         }
         mask |= 255u << shift;
         __syncthreads();

@@ -3,8 +3,8 @@
 // tcgen05.mma accumulates in tensor memory, and the softmax / column-sum warps read
 // the accumulators back with tcgen05.ld.  Three kernels share the machinery:
 //
-//   attn_kernel<true>   a1: causal attention of the chunk over [cache ; chunk] (+ row LSE)
-//   attn_kernel<false>  a2 pass 1: row log-sum-exp of the scoring queries over all candidates
+//   attn_kernel<true,*> a1: causal attention of the chunk over [cache ; chunk] (+ row LSE)
+//   attn_kernel<false,*> a2 pass 1: row log-sum-exp of the scoring queries over all candidates
 //   colsum_kernel       a2 pass 2: S^T = K Q^T with the candidates on the accumulator's rows,
 //                       so the column sum of Eq. 1 over scoring rows is a per-thread sum
 //
@@ -13,6 +13,17 @@
 #include "citrus_internal.h"
 
 #include <cuda.h>
+
+// Optional cycle stamps of one CTA's roles (build with -DCITRUS_TRACE; compiled out otherwise).
+#ifdef CITRUS_TRACE
+__device__ unsigned long long g_citrus_trace[256];
+#define CITRUS_TR(i) do { if (blockIdx.x == gridDim.x - 1 && blockIdx.y == 0 && (threadIdx.x & 31) == 0) \
+                              g_citrus_trace[(i)] = clock64(); } while (0)
+extern "C" int citrus_trace_read(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_citrus_trace, sizeof(g_citrus_trace)); }
+extern "C" int citrus_trace_clear() { static unsigned long long z[256]; return (int)cudaMemcpyToSymbol(g_citrus_trace, z, sizeof(z)); }
+#else
+#define CITRUS_TR(i) do { } while (0)
+#endif
 
 namespace citrus {
 namespace {
@@ -69,6 +80,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
 // Same, with one outcome for the whole warp (the callers go on to warp-collective instructions).
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, status));
+}
+
+// One lane of a converged warp.  Loop control, addresses and descriptors are computed by the whole
+// warp (so they stay warp-uniform); only the issuing instruction itself is predicated on the leader.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
@@ -182,23 +201,45 @@ struct TcParams {
 
 // Load one 128x128 bf16 tile as two swizzled halves.  token_major: coordinates (d, head, row);
 // otherwise (cache layout) (d, row, head).
+// Called by a converged warp; one elected lane arms the barrier and issues the two copies.
 __device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row, int head, bool token_major) {
-    if (token_major) {
-        tma_load_3d(dst, map, bar, 0, head, row);
-        tma_load_3d(dst + kHalfBytes, map, bar, 64, head, row);
-    } else {
-        tma_load_3d(dst, map, bar, 0, row, head);
-        tma_load_3d(dst + kHalfBytes, map, bar, 64, row, head);
+    const int y = token_major ? head : row, z = token_major ? row : head;
+    if (elect_one()) {
+        mbar_expect_tx(bar, kTileBytes);
+        tma_load_3d(dst, map, bar, 0, y, z);
+        tma_load_3d(dst + kHalfBytes, map, bar, 64, y, z);
     }
+    __syncwarp();
 }
 
 // S[128 x n_cols] = A_tile . B_tile^T over the 128-wide head dimension (8 steps of 16).
-__device__ __forceinline__ void issue_qk(uint32_t tmem_d, uint32_t a_smem, uint32_t b_smem, uint32_t idesc) {
+// Called by a converged warp; bar1/bar2 (0 = none) receive a commit after the eight MMAs.
+__device__ __forceinline__ void issue_qk(uint32_t tmem_d, uint32_t a_smem, uint32_t b_smem, uint32_t idesc,
+                                         uint32_t bar1, uint32_t bar2) {
+    const uint64_t a0 = desc_kmajor(a_smem), b0 = desc_kmajor(b_smem);
+    if (elect_one()) {
 #pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-        uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-        mma_ss(tmem_d, desc_kmajor(a_smem + off), desc_kmajor(b_smem + off), idesc, kk > 0);
+        for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);   // start-address field units
+            mma_ss(tmem_d, a0 + off, b0 + off, idesc, kk > 0);
+        }
+        if (bar1) mma_commit(bar1);
+        if (bar2) mma_commit(bar2);
     }
+    __syncwarp();
+}
+// O (+)= P . V for one key tile: P (bf16) in tensor memory, V tile MN-major in shared memory.
+__device__ __forceinline__ void issue_pv(uint32_t tmem_o, uint32_t tmem_p, uint32_t v_smem, uint32_t idesc, bool first,
+                                         uint32_t bar1, uint32_t bar2) {
+    const uint64_t b0 = desc_mnmajor(v_smem);
+    if (elect_one()) {
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)     // 16 keys per step: P columns 8*kk.., V rows 16*kk.. (2048 B apart)
+            mma_ts(tmem_o, tmem_p + kk * 8, b0 + (uint64_t)((kk * 2048) >> 4), idesc, !(first && kk == 0));
+        mma_commit(bar1);
+        mma_commit(bar2);
+    }
+    __syncwarp();
 }
 
 constexpr int kStages = 2;
@@ -214,7 +255,8 @@ struct AttnSmem {
 constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + 2 * kStages) + 1024;
 
 // grid: (ceil(rows / 128), q_heads).  One CTA = 128 query rows of one head.
-template <bool WITH_PV>
+// WITH_PV: accumulate O = P.V and write `out`; NEED_LSE: keep the fp32 row sum and write the row log-sum-exp.
+template <bool WITH_PV, bool NEED_LSE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
             const __grid_constant__ CUtensorMap mapCV, const __grid_constant__ CUtensorMap mapSK,
@@ -229,6 +271,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = blockIdx.x, h = blockIdx.y;
     const int g = h / (p.q_heads / p.kv_heads);
+    if (WITH_PV && warp == 0) CITRUS_TR(0);
     const int q_row0 = qt * kTile;                                  // first row of this tile inside the block
     const int n_cache_tiles = (p.m + kTile - 1) / kTile;
     // chunk key tiles this query tile may see
@@ -258,69 +301,60 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
     const uint32_t tmO = tmem + 256u;
+    if (WITH_PV && warp == 0) CITRUS_TR(1);
 
     if (warp == 4) {
-        // ---------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            mbar_expect_tx(smem_u32(&bars->q_full), kTileBytes);
-            load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
-            bool ok = true;
-            for (int j = 0; j < nt && ok; ++j) {
-                const int s = j % kStages;
-                const uint32_t ph = ((j / kStages) & 1) ^ 1;
-                const bool from_cache = j < n_cache_tiles;
-                const int row = from_cache ? j * kTile : (j - n_cache_tiles) * kTile;
-                ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph, p.status);
-                if (!ok) break;
-                mbar_expect_tx(smem_u32(&bars->k_full[s]), kTileBytes);
-                load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, g, !from_cache);
-                if (WITH_PV) {
-                    ok = mbar_wait(smem_u32(&bars->v_empty[s]), ph, p.status);
-                    if (!ok) break;
-                    mbar_expect_tx(smem_u32(&bars->v_full[s]), kTileBytes);
-                    load_tile(sV + s * kTileBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
-                }
+        // ---------------------------------------------------------------- TMA producer (converged warp)
+        load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
+        for (int j = 0; j < nt; ++j) {
+            const int s = j % kStages;
+            const uint32_t ph = ((j / kStages) & 1) ^ 1;
+            const bool from_cache = j < n_cache_tiles;
+            const int row = from_cache ? j * kTile : (j - n_cache_tiles) * kTile;
+            if (!mbar_wait_warp(smem_u32(&bars->k_empty[s]), ph, p.status)) break;
+            load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, g, !from_cache);
+            if (WITH_PV) {
+                if (!mbar_wait_warp(smem_u32(&bars->v_empty[s]), ph, p.status)) break;
+                load_tile(sV + s * kTileBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
             }
         }
     } else if (warp == 5) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_qk = make_idesc(128, 0);
-            constexpr uint32_t idesc_pv = make_idesc(128, 1);
-            bool ok = mbar_wait(smem_u32(&bars->q_full), 0, p.status);
-            auto qk = [&](int j) -> bool {
+        // ---------------------------------------------------------------- MMA issuer (converged warp)
+        constexpr uint32_t idesc_qk = make_idesc(128, 0);
+        constexpr uint32_t idesc_pv = make_idesc(128, 1);
+        bool ok = mbar_wait_warp(smem_u32(&bars->q_full), 0, p.status);
+        if (WITH_PV) CITRUS_TR(2);
+        auto qk = [&](int j) -> bool {
+            const int s = j % kStages;
+            if (!mbar_wait_warp(smem_u32(&bars->k_full[s]), (j / kStages) & 1, p.status)) return false;
+            tc_fence_after();
+            if (WITH_PV) CITRUS_TR(70 + j);
+            issue_qk(tmS(j & 1), sQ, sK + s * kTileBytes, idesc_qk, smem_u32(&bars->s_full[j & 1]), smem_u32(&bars->k_empty[s]));
+            if (WITH_PV) CITRUS_TR(10 + j);
+            return true;
+        };
+        if (ok && nt > 0) ok = qk(0);
+        if (ok && nt > 1) ok = qk(1);
+        for (int j = 0; j < nt && ok; ++j) {
+            // softmax has consumed S_j (and, with PV, written P_j over it)
+            ok = mbar_wait_warp(smem_u32(&bars->p_full[j & 1]), (j >> 1) & 1, p.status);
+            if (!ok) break;
+            if (WITH_PV) {
                 const int s = j % kStages;
-                if (!mbar_wait(smem_u32(&bars->k_full[s]), (j / kStages) & 1, p.status)) return false;
-                tc_fence_after();
-                issue_qk(tmS(j & 1), sQ, sK + s * kTileBytes, idesc_qk);
-                mma_commit(smem_u32(&bars->s_full[j & 1]));
-                mma_commit(smem_u32(&bars->k_empty[s]));
-                return true;
-            };
-            if (ok && nt > 0) ok = qk(0);
-            if (ok && nt > 1) ok = qk(1);
-            for (int j = 0; j < nt && ok; ++j) {
-                // softmax has consumed S_j (and, with PV, written P_j over it)
-                ok = mbar_wait(smem_u32(&bars->p_full[j & 1]), (j >> 1) & 1, p.status);
+                ok = mbar_wait_warp(smem_u32(&bars->v_full[s]), (j / kStages) & 1, p.status);
                 if (!ok) break;
-                if (WITH_PV) {
-                    const int s = j % kStages;
-                    ok = mbar_wait(smem_u32(&bars->v_full[s]), (j / kStages) & 1, p.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t v_smem = sV + s * kTileBytes;
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)     // 16 keys per step: P columns 8*kk.., V rows 16*kk..
-                        mma_ts(tmO, tmS(j & 1) + kk * 8, desc_mnmajor(v_smem + kk * 2048), idesc_pv, (j > 0 || kk > 0));
-                    mma_commit(smem_u32(&bars->v_empty[s]));
-                    mma_commit(smem_u32(&bars->o_done));
-                }
-                if (j + 2 < nt) ok = qk(j + 2);
+                tc_fence_after();
+                CITRUS_TR(90 + j);
+                issue_pv(tmO, tmS(j & 1), sV + s * kTileBytes, idesc_pv, j == 0,
+                         smem_u32(&bars->v_empty[s]), smem_u32(&bars->o_done));
+                CITRUS_TR(30 + j);
             }
-            // all tensor-core work retired before tensor memory is released
-            mma_commit(smem_u32(&bars->drain));
-            mbar_wait(smem_u32(&bars->drain), 0, p.status);
+            if (j + 2 < nt) ok = qk(j + 2);
         }
+        // all tensor-core work retired before tensor memory is released
+        if (elect_one()) mma_commit(smem_u32(&bars->drain));
+        __syncwarp();
+        mbar_wait_warp(smem_u32(&bars->drain), 0, p.status);
     } else {
         // ---------------------------------------------------------------- softmax / epilogue (warps 0-3)
         const int row_in_tile = warp * 32 + lane;
@@ -334,6 +368,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
             const int b = j & 1;
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (j >> 1) & 1, p.status);
             if (!ok) break;
+            if (WITH_PV && warp == 0) CITRUS_TR(50 + 2 * j);
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tmS(b) + lane_base + c * 32, sreg + c * 32);
@@ -347,18 +382,19 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                 lim = min(kTile, p.L - u0);
                 if (p.causal) lim = min(lim, p.t0 + r - u0 + 1);
             }
-            float mx = -INFINITY;
-            if (lim >= kTile) {
+            if (lim < kTile) {
 #pragma unroll
-                for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sreg[c]));
-            } else {
-#pragma unroll
-                for (int c = 0; c < 128; ++c) {
-                    float v = c < lim ? __uint_as_float(sreg[c]) : -INFINITY;
-                    sreg[c] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
-                }
+                for (int c = 0; c < 128; ++c)
+                    if (c >= lim) sreg[c] = 0xff800000u;             // -inf
             }
+            // four independent chains keep the single warp of this scheduler from stalling on itself
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int c = 0; c < 128; c += 4) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) mx4[i] = fmaxf(mx4[i], __uint_as_float(sreg[c + i]));
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             const float m_new = fmaxf(m_ref, mx * scale2);
             if (j == 0) {
                 m_ref = m_new;
@@ -392,7 +428,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
             // the bf16-rounded ones that P.V actually multiplies, so that out = sum(p~ v) / sum(p~) stays a
             // convex combination of V rows even when one key takes nearly all of the mass.
             const float neg_m = -m_ref;
-            float sum = 0.f, sum_r = 0.f;
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f}, sumr4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
                 uint32_t packed[16];
@@ -400,17 +436,21 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                 for (int i = 0; i < 16; ++i) {
                     float p0 = ex2(fmaf(__uint_as_float(sreg[c4 * 32 + 2 * i]), scale2, neg_m));
                     float p1 = ex2(fmaf(__uint_as_float(sreg[c4 * 32 + 2 * i + 1]), scale2, neg_m));
-                    sum += p0 + p1;
+                    if (NEED_LSE) { sum4[i & 3] += p0; sum4[(i + 2) & 3] += p1; }
                     packed[i] = pack_bf16(p0, p1);
-                    if (WITH_PV) sum_r += __uint_as_float(packed[i] << 16) + __uint_as_float(packed[i] & 0xffff0000u);
+                    if (WITH_PV) {
+                        sumr4[i & 3] += __uint_as_float(packed[i] << 16);
+                        sumr4[(i + 2) & 3] += __uint_as_float(packed[i] & 0xffff0000u);
+                    }
                 }
                 if (WITH_PV) tmem_st16(tmS(b) + lane_base + c4 * 16, packed);
             }
-            l_run += sum;
-            l_out += sum_r;
+            l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+            l_out += (sumr4[0] + sumr4[1]) + (sumr4[2] + sumr4[3]);
             if (WITH_PV) tmem_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&bars->p_full[b]));
+            if (WITH_PV && warp == 0) CITRUS_TR(51 + 2 * j);
         }
         if (ok && nt > 0) {
             if (WITH_PV) {
@@ -420,6 +460,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                 if (nt > 1) ok = mbar_wait_warp(smem_u32(&bars->o_done), (nt - 2) & 1, p.status);
                 if (ok) ok = mbar_wait_warp(smem_u32(&bars->o_done), (nt - 1) & 1, p.status);
                 if (ok) {
+                    if (warp == 0) CITRUS_TR(110);
                     tc_fence_after();
                     const float inv = 1.f / l_out;
                     __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + ((size_t)r * p.q_heads + h) * kD;
@@ -442,11 +483,13 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                     }
                 }
             }
-            if (ok && r < p.rows && p.lse2 != nullptr) p.lse2[(size_t)h * p.lse_stride + r] = m_ref + log2f(l_run);
+            if (NEED_LSE && ok && r < p.rows && p.lse2 != nullptr) p.lse2[(size_t)h * p.lse_stride + r] = m_ref + log2f(l_run);
         }
     }
+    if (WITH_PV && warp == 0) CITRUS_TR(111);
     tc_fence_before();
     __syncthreads();
+    if (WITH_PV && warp == 0) CITRUS_TR(112);
     if (warp == 5) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
 }
 
@@ -454,10 +497,11 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
 constexpr int kColStages = 3;
 constexpr int kColTmemCols = 256;
 struct ColSmem {
-    uint64_t k_full, q_full[kColStages], q_empty[kColStages], s_full[2], s_free[2], drain;
+    uint64_t k_full, q_full[kColStages], q_empty[kColStages], s_full[2], s_free[2], lse_full[4], drain;
     uint32_t tmem_base;
+    alignas(16) float lse[4][kTile];          // log-sum-exp of the scoring rows of four consecutive (head, row block)s
 };
-constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 1024;
+constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 2048;
 
 // grid: (candidate tiles, kv_heads).  Accumulator rows = 128 candidates, columns = scoring rows of one
 // (head, row block); thread i owns candidate i and adds exp2(logit2 - lse2[row]) over its columns.
@@ -475,17 +519,22 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int G = p.q_heads / p.kv_heads;
     const int n_cache_tiles = (p.m + kTile - 1) / kTile;
     const bool from_cache = kt < n_cache_tiles;
+    if (warp == 0) CITRUS_TR(128);
     const int key_row0 = from_cache ? kt * kTile : (kt - n_cache_tiles) * kTile;   // row in its source
     const int n_rb = (p.rows + kTile - 1) / kTile;
     // first row block that can see any key of this tile
     int rb0 = 0;
     if (p.causal && !from_cache && key_row0 > p.t0) rb0 = (key_row0 - p.t0) / kTile;
-    const int nb = G * (n_rb - rb0);                  // (head, row block) iterations
+    const int rb_per_head = n_rb - rb0;
+    const int nb = G * rb_per_head;                   // (head, row block) iterations
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars->k_full), 1);
         for (int s = 0; s < kColStages; ++s) { mbar_init(smem_u32(&bars->q_full[s]), 1); mbar_init(smem_u32(&bars->q_empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 128); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 128);
+        }
+        for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&bars->lse_full[b]), 128);
         mbar_init(smem_u32(&bars->drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -498,37 +547,35 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
 
     if (warp == 4) {
-        if (lane == 0) {
-            mbar_expect_tx(smem_u32(&bars->k_full), kTileBytes);
-            load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
-            for (int it = 0; it < nb; ++it) {
-                const int s = it % kColStages;
-                const int h = g * G + it / (n_rb - rb0);
-                const int rb = rb0 + it % (n_rb - rb0);
-                if (!mbar_wait(smem_u32(&bars->q_empty[s]), ((it / kColStages) & 1) ^ 1, p.status)) break;
-                mbar_expect_tx(smem_u32(&bars->q_full[s]), kTileBytes);
-                load_tile(sQ + s * kTileBytes, &mapQ, smem_u32(&bars->q_full[s]), p.row0 + rb * kTile, h, true);
-            }
+        // TMA producer (converged warp)
+        load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
+        for (int it = 0; it < nb; ++it) {
+            const int s = it % kColStages;
+            const int h = g * G + it / rb_per_head;
+            const int rb = rb0 + it % rb_per_head;
+            if (!mbar_wait_warp(smem_u32(&bars->q_empty[s]), ((it / kColStages) & 1) ^ 1, p.status)) break;
+            load_tile(sQ + s * kTileBytes, &mapQ, smem_u32(&bars->q_full[s]), p.row0 + rb * kTile, h, true);
         }
     } else if (warp == 5) {
-        if (lane == 0) {
-            bool ok = mbar_wait(smem_u32(&bars->k_full), 0, p.status);
-            for (int it = 0; it < nb && ok; ++it) {
-                const int s = it % kColStages, b = it & 1;
-                const int rb = rb0 + it % (n_rb - rb0);
-                const int ncols = min(kTile, ((p.rows - rb * kTile) + 15) & ~15);
-                ok = mbar_wait(smem_u32(&bars->q_full[s]), (it / kColStages) & 1, p.status);
-                if (!ok) break;
-                ok = mbar_wait(smem_u32(&bars->s_free[b]), ((it >> 1) & 1) ^ 1, p.status);
-                if (!ok) break;
-                tc_fence_after();
-                issue_qk(tmS(b), sK, sQ + s * kTileBytes, make_idesc(ncols, 0));
-                mma_commit(smem_u32(&bars->s_full[b]));
-                mma_commit(smem_u32(&bars->q_empty[s]));
-            }
-            mma_commit(smem_u32(&bars->drain));
-            mbar_wait(smem_u32(&bars->drain), 0, p.status);
+        // MMA issuer (converged warp)
+        bool ok = mbar_wait_warp(smem_u32(&bars->k_full), 0, p.status);
+        for (int it = 0; it < nb && ok; ++it) {
+            const int s = it % kColStages, b = it & 1;
+            const int rb = rb0 + it % rb_per_head;
+            const int ncols = min(kTile, ((p.rows - rb * kTile) + 15) & ~15);
+            ok = mbar_wait_warp(smem_u32(&bars->q_full[s]), (it / kColStages) & 1, p.status);
+            if (!ok) break;
+            ok = mbar_wait_warp(smem_u32(&bars->s_free[b]), ((it >> 1) & 1) ^ 1, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            CITRUS_TR(140 + 2 * (it & 7));
+            issue_qk(tmS(b), sK, sQ + s * kTileBytes, make_idesc(ncols, 0),
+                     smem_u32(&bars->s_full[b]), smem_u32(&bars->q_empty[s]));
+            CITRUS_TR(141 + 2 * (it & 7));
         }
+        if (elect_one()) mma_commit(smem_u32(&bars->drain));
+        __syncwarp();
+        mbar_wait_warp(smem_u32(&bars->drain), 0, p.status);
     } else {
         const int key_in_tile = warp * 32 + lane;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
@@ -544,10 +591,19 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         uint32_t sreg[128];
         for (int it = 0; it < nb; ++it) {
             const int b = it & 1;
-            const int h = g * G + it / (n_rb - rb0);
-            const int rb = rb0 + it % (n_rb - rb0);
+            const int h = g * G + it / rb_per_head;
+            const int rb = rb0 + it % rb_per_head;
             const int r0 = rb * kTile;
             const int ncols = min(kTile, p.rows - r0);
+            // stage this block's log-sum-exp values (thread i brings row r0 + i).  A thread can run at most
+            // three iterations ahead of the slowest one (the MMA of it-1 needs everybody's s_free of it-3),
+            // so with four buffers nobody is still reading the one written here.
+            const int lb = it & 3;
+            {
+                const int rr = r0 + key_in_tile;
+                bars->lse[lb][key_in_tile] = rr < p.rows ? __ldg(p.lse_in + (size_t)h * p.lse_stride + rr) : INFINITY;
+                mbar_arrive(smem_u32(&bars->lse_full[lb]));
+            }
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 1) & 1, p.status);
             if (!ok) break;
             tc_fence_after();
@@ -557,22 +613,35 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive(smem_u32(&bars->s_free[b]));
-            const float* lse = p.lse_in + (size_t)h * p.lse_stride + r0;
+            if (warp == 0) CITRUS_TR(160 + 3 * (it & 7));
+            ok = mbar_wait_warp(smem_u32(&bars->lse_full[lb]), (it >> 2) & 1, p.status);
+            if (!ok) break;
+            if (warp == 0) CITRUS_TR(161 + 3 * (it & 7));
+            const float4* lse4 = reinterpret_cast<const float4*>(bars->lse[lb]);
             const int c_lo = max(0, r_first - r0);
-            float part = 0.f;
+            float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < 128; ++c) {
-                if (c < ncols) {
-                    float e = ex2(fmaf(__uint_as_float(sreg[c]), scale2, -__ldg(lse + c)));
-                    part += c >= c_lo ? e : 0.f;
+            for (int c = 0; c < 128; c += 4) {
+                if (c < ncols) {                               // rows past the block end carry lse = +inf -> exp2 = 0
+                    const float4 l = lse4[c >> 2];
+                    float e0 = ex2(fmaf(__uint_as_float(sreg[c + 0]), scale2, -l.x));
+                    float e1 = ex2(fmaf(__uint_as_float(sreg[c + 1]), scale2, -l.y));
+                    float e2 = ex2(fmaf(__uint_as_float(sreg[c + 2]), scale2, -l.z));
+                    float e3 = ex2(fmaf(__uint_as_float(sreg[c + 3]), scale2, -l.w));
+                    part[0] += c + 0 >= c_lo ? e0 : 0.f;
+                    part[1] += c + 1 >= c_lo ? e1 : 0.f;
+                    part[2] += c + 2 >= c_lo ? e2 : 0.f;
+                    part[3] += c + 3 >= c_lo ? e3 : 0.f;
                 }
             }
-            acc += part;
+            acc += (part[0] + part[1]) + (part[2] + part[3]);
+            if (warp == 0) CITRUS_TR(162 + 3 * (it & 7));
         }
         if (ok && key_ok) p.scores[(size_t)g * p.score_stride + j] = acc;
     }
     tc_fence_before();
     __syncthreads();
+    if (warp == 0) CITRUS_TR(190);
     if (warp == 5) { __syncwarp(); tmem_dealloc(tmem, kColTmemCols); }
 }
 
@@ -636,9 +705,11 @@ cudaError_t tc_init() {
     if (e != cudaSuccess) return e;
     if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
     g_encode = reinterpret_cast<EncodeFn>(fn);
-    e = cudaFuncSetAttribute(attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    e = cudaFuncSetAttribute(attn_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    e = cudaFuncSetAttribute(attn_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kColSmemBytes);
 }
@@ -650,7 +721,8 @@ cudaError_t tc_attention(const QueryRows& q, const Candidates& c, void* out, flo
     TcParams p = base_params(q, c, status);
     p.out = out; p.lse2 = lse2; p.lse_stride = lse_stride;
     dim3 grid((q.rows + kTile - 1) / kTile, q.q_heads);
-    attn_kernel<true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
+    if (lse2 != nullptr) attn_kernel<true, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
+    else attn_kernel<true, false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
     return cudaGetLastError();
 }
 
@@ -661,7 +733,7 @@ cudaError_t tc_score_lse(const QueryRows& q, const Candidates& c, float* lse2, i
     TcParams p = base_params(q, c, status);
     p.out = nullptr; p.lse2 = lse2; p.lse_stride = lse_stride;
     dim3 grid((q.rows + kTile - 1) / kTile, q.q_heads);
-    attn_kernel<false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
+    attn_kernel<false, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
     return cudaGetLastError();
 }
 
