@@ -242,31 +242,50 @@ __device__ __forceinline__ void issue_pv(uint32_t tmem_o, uint32_t tmem_p, uint3
     __syncwarp();
 }
 
-constexpr int kStages = 2;
-constexpr int kAttnThreads = 192;       // 4 softmax warps, 1 TMA warp, 1 MMA warp
+constexpr int kStagesK = 3;             // K ring
+constexpr int kStagesV = 2;             // V ring
+constexpr int kAttnThreads = 352;       // 2 softmax warpgroups (8 warps), K-TMA warp, MMA warp, V-TMA warp
+constexpr int kColThreads = 192;        // 4 column-sum warps, 1 TMA warp, 1 MMA warp
 constexpr int kTmemCols = 512;
 constexpr float kRescaleTau = 8.f;      // rescale O only when the row max grows by more than 2^8
 
+// Bulk tensor store shared -> global (rows past the tensor map's extent are clipped).
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
+struct RowState { float m, l, lo; };    // exponent reference, fp32 sum, sum of bf16-rounded probabilities
+
 struct AttnSmem {
-    uint64_t q_full, k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-    uint64_t s_full[2], p_full[2], o_done, drain;
+    uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
+    uint64_t s_full[2], p_full[2], o_done[2], xch, out_ready[2], drain;
     uint32_t tmem_base;
+    RowState rows[2][kTile];            // final per-row state of each warpgroup, exchanged once at the end
 };
-constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + 2 * kStages) + 1024;
+constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + kStagesK + kStagesV) + 4096;
 
 // grid: (ceil(rows / 128), q_heads).  One CTA = 128 query rows of one head.
 // WITH_PV: accumulate O = P.V and write `out`; NEED_LSE: keep the fp32 row sum and write the row log-sum-exp.
+//
+// Key tiles alternate between two softmax warpgroups: warpgroup b takes tiles b, b+2, ... with its own
+// exponent reference, its own S/P buffer S[b] and its own accumulator O[b], so the two never exchange
+// anything inside the loop and each scheduler always has a second warp to run.  The two partial results
+// are merged once, in the epilogue:  out = (w0 O[0] + w1 O[1]) / (w0 l0 + w1 l1),  w_b = 2^(m_b - max m).
 template <bool WITH_PV, bool NEED_LSE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
             const __grid_constant__ CUtensorMap mapCV, const __grid_constant__ CUtensorMap mapSK,
-            const __grid_constant__ CUtensorMap mapSV, const TcParams p) {
+            const __grid_constant__ CUtensorMap mapSV, const __grid_constant__ CUtensorMap mapO, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = base;
     const uint32_t sK = sQ + kTileBytes;
-    const uint32_t sV = sK + kStages * kTileBytes;
-    AttnSmem* bars = reinterpret_cast<AttnSmem*>(smem_raw + (sV + kStages * kTileBytes - smem_u32(smem_raw)));
+    const uint32_t sV = sK + kStagesK * kTileBytes;
+    uint8_t* const gQ = smem_raw + (sQ - smem_u32(smem_raw));         // generic pointer to the Q tile / output staging
+    AttnSmem* bars = reinterpret_cast<AttnSmem*>(smem_raw + (sV + kStagesV * kTileBytes - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = blockIdx.x, h = blockIdx.y;
@@ -284,95 +303,104 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars->q_full), 1);
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1);
-            mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1);
+        for (int s = 0; s < kStagesK; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
+        for (int s = 0; s < kStagesV; ++s) { mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->p_full[b]), 128);
+            mbar_init(smem_u32(&bars->o_done[b]), 1); mbar_init(smem_u32(&bars->out_ready[b]), 128);
         }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->p_full[b]), 128); }
-        mbar_init(smem_u32(&bars->o_done), 1);
+        mbar_init(smem_u32(&bars->xch), 256);
         mbar_init(smem_u32(&bars->drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 5) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
+    if (warp == 9) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
-    const uint32_t tmO = tmem + 256u;
+    auto tmO = [tmem](int b) { return tmem + 256u + (uint32_t)b * 128u; };
     if (WITH_PV && warp == 0) CITRUS_TR(1);
 
-    if (warp == 4) {
-        // ---------------------------------------------------------------- TMA producer (converged warp)
+    if (warp == 8) {
+        // ---------------------------------------------------------------- K (and Q) TMA producer (converged warp)
         load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
         for (int j = 0; j < nt; ++j) {
-            const int s = j % kStages;
-            const uint32_t ph = ((j / kStages) & 1) ^ 1;
+            const int s = j % kStagesK;
             const bool from_cache = j < n_cache_tiles;
             const int row = from_cache ? j * kTile : (j - n_cache_tiles) * kTile;
-            if (!mbar_wait_warp(smem_u32(&bars->k_empty[s]), ph, p.status)) break;
+            if (!mbar_wait_warp(smem_u32(&bars->k_empty[s]), ((j / kStagesK) & 1) ^ 1, p.status)) break;
             load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, g, !from_cache);
-            if (WITH_PV) {
-                if (!mbar_wait_warp(smem_u32(&bars->v_empty[s]), ph, p.status)) break;
+        }
+    } else if (warp == 10) {
+        // ---------------------------------------------------------------- V TMA producer (converged warp)
+        if (WITH_PV) {
+            for (int j = 0; j < nt; ++j) {
+                const int s = j % kStagesV;
+                const bool from_cache = j < n_cache_tiles;
+                const int row = from_cache ? j * kTile : (j - n_cache_tiles) * kTile;
+                if (!mbar_wait_warp(smem_u32(&bars->v_empty[s]), ((j / kStagesV) & 1) ^ 1, p.status)) break;
                 load_tile(sV + s * kTileBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ---------------------------------------------------------------- MMA issuer (converged warp)
         constexpr uint32_t idesc_qk = make_idesc(128, 0);
         constexpr uint32_t idesc_pv = make_idesc(128, 1);
         bool ok = mbar_wait_warp(smem_u32(&bars->q_full), 0, p.status);
         if (WITH_PV) CITRUS_TR(2);
-        auto qk = [&](int j) -> bool {
-            const int s = j % kStages;
-            if (!mbar_wait_warp(smem_u32(&bars->k_full[s]), (j / kStages) & 1, p.status)) return false;
-            tc_fence_after();
-            if (WITH_PV) CITRUS_TR(70 + j);
+        auto k_ready = [&](int j) { return mbar_wait_warp(smem_u32(&bars->k_full[j % kStagesK]), (j / kStagesK) & 1, p.status); };
+        auto qk = [&](int j) {
+            const int s = j % kStagesK;
             issue_qk(tmS(j & 1), sQ, sK + s * kTileBytes, idesc_qk, smem_u32(&bars->s_full[j & 1]), smem_u32(&bars->k_empty[s]));
-            if (WITH_PV) CITRUS_TR(10 + j);
-            return true;
         };
-        if (ok && nt > 0) ok = qk(0);
-        if (ok && nt > 1) ok = qk(1);
+        for (int j = 0; j < 2 && j < nt && ok; ++j) {
+            ok = k_ready(j);
+            if (ok) { tc_fence_after(); qk(j); }
+        }
         for (int j = 0; j < nt && ok; ++j) {
-            // softmax has consumed S_j (and, with PV, written P_j over it)
+            // operands of the next two MMA groups are checked while the softmax of tile j is still running,
+            // so only the p_full wait sits between its arrival and the tensor pipe
+            if (WITH_PV) {
+                ok = mbar_wait_warp(smem_u32(&bars->v_full[j % kStagesV]), (j / kStagesV) & 1, p.status);
+                if (!ok) break;
+            }
+            if (j + 2 < nt) { ok = k_ready(j + 2); if (!ok) break; }
+            // warpgroup j&1 has consumed S_j (and, with PV, written P_j over it)
             ok = mbar_wait_warp(smem_u32(&bars->p_full[j & 1]), (j >> 1) & 1, p.status);
             if (!ok) break;
+            tc_fence_after();
             if (WITH_PV) {
-                const int s = j % kStages;
-                ok = mbar_wait_warp(smem_u32(&bars->v_full[s]), (j / kStages) & 1, p.status);
-                if (!ok) break;
-                tc_fence_after();
+                const int s = j % kStagesV;
                 CITRUS_TR(90 + j);
-                issue_pv(tmO, tmS(j & 1), sV + s * kTileBytes, idesc_pv, j == 0,
-                         smem_u32(&bars->v_empty[s]), smem_u32(&bars->o_done));
+                issue_pv(tmO(j & 1), tmS(j & 1), sV + s * kTileBytes, idesc_pv, j < 2,
+                         smem_u32(&bars->v_empty[s]), smem_u32(&bars->o_done[j & 1]));
                 CITRUS_TR(30 + j);
             }
-            if (j + 2 < nt) ok = qk(j + 2);
+            if (j + 2 < nt) { qk(j + 2); if (WITH_PV) CITRUS_TR(10 + j + 2); }
         }
         // all tensor-core work retired before tensor memory is released
         if (elect_one()) mma_commit(smem_u32(&bars->drain));
         __syncwarp();
         mbar_wait_warp(smem_u32(&bars->drain), 0, p.status);
     } else {
-        // ---------------------------------------------------------------- softmax / epilogue (warps 0-3)
-        const int row_in_tile = warp * 32 + lane;
+        // ---------------------------------------------------------------- softmax warpgroups (warps 0-7)
+        const int wg = warp >> 2;                                    // takes key tiles wg, wg+2, ...
+        const int row_in_tile = (warp & 3) * 32 + lane;
         const int r = q_row0 + row_in_tile;                          // row inside the block
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const float scale2 = kLog2e * rsqrtf((float)kD);
         float m_ref = -INFINITY, l_run = 0.f, l_out = 0.f;
         bool ok = true;
-        uint32_t sreg[128];
-        for (int j = 0; j < nt; ++j) {
-            const int b = j & 1;
-            ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (j >> 1) & 1, p.status);
+        int i_last = -1;                                             // local index of this warpgroup's last tile
+        for (int j = wg; j < nt; j += 2) {
+            const int i = j >> 1;
+            i_last = i;
+            ok = mbar_wait_warp(smem_u32(&bars->s_full[wg]), i & 1, p.status);
             if (!ok) break;
-            if (WITH_PV && warp == 0) CITRUS_TR(50 + 2 * j);
+            if (WITH_PV && warp == 0) CITRUS_TR(50 + 5 * i);
             tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tmS(b) + lane_base + c * 32, sreg + c * 32);
-            tmem_wait_ld();
             // number of visible columns of this tile for this row
             int lim = kTile;
             if (j < n_cache_tiles) {
@@ -382,21 +410,26 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                 lim = min(kTile, p.L - u0);
                 if (p.causal) lim = min(lim, p.t0 + r - u0 + 1);
             }
-            if (lim < kTile) {
-#pragma unroll
-                for (int c = 0; c < 128; ++c)
-                    if (c >= lim) sreg[c] = 0xff800000u;             // -inf
-            }
-            // four independent chains keep the single warp of this scheduler from stalling on itself
+            const uint32_t s_addr = tmS(wg) + lane_base;
+            // ---- sweep 1: row maximum over all 128 columns (one round trip to tensor memory)
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            {
+                uint32_t v[128];
 #pragma unroll
-            for (int c = 0; c < 128; c += 4) {
+                for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v + c * 32);
+                tmem_wait_ld();
+                if (lim < kTile) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) mx4[i] = fmaxf(mx4[i], __uint_as_float(sreg[c + i]));
+                    for (int q = 0; q < 128; ++q)
+                        if (q >= lim) v[q] = 0xff800000u;            // -inf
+                }
+#pragma unroll
+                for (int q = 0; q < 128; ++q) mx4[q & 3] = fmaxf(mx4[q & 3], __uint_as_float(v[q]));
             }
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             const float m_new = fmaxf(m_ref, mx * scale2);
-            if (j == 0) {
+            if (WITH_PV && warp == 0) CITRUS_TR(51 + 5 * i);
+            if (i == 0) {
                 m_ref = m_new;
             } else {
                 const bool grow = (m_new - m_ref) > kRescaleTau;
@@ -406,91 +439,138 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                     l_out *= f;
                     m_ref = m_new;
                     if (WITH_PV) {
-                        // O holds tiles 0..j-1 once P.V of tile j-1 has retired
-                        ok = mbar_wait_warp(smem_u32(&bars->o_done), (j - 1) & 1, p.status);
-                        if (!ok) break;
-                        tc_fence_after();
-                        uint32_t oreg[32];
-#pragma unroll
+                        // O[wg] is quiescent here: its last writer, P.V of tile j-2, was issued before Q.K^T of
+                        // tile j, whose completion this warpgroup has just observed through s_full.
+#pragma unroll 1
                         for (int c = 0; c < 4; ++c) {
-                            tmem_ld32(tmO + lane_base + c * 32, oreg);
+                            uint32_t oreg[32];
+                            tmem_ld32(tmO(wg) + lane_base + c * 32, oreg);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * f);
-                            tmem_st32(tmO + lane_base + c * 32, oreg);
+                            for (int q = 0; q < 32; ++q) oreg[q] = __float_as_uint(__uint_as_float(oreg[q]) * f);
+                            tmem_st32(tmO(wg) + lane_base + c * 32, oreg);
                         }
                     }
                 }
             }
-            // rows whose tile is fully masked keep m_ref = -inf only if nothing was visible so far;
-            // the first tile of every row has a visible column, so m_ref is finite here.
-            // l_run sums the fp32 probabilities (it feeds the log-sum-exp that a2-L reuses); l_out sums
-            // the bf16-rounded ones that P.V actually multiplies, so that out = sum(p~ v) / sum(p~) stays a
-            // convex combination of V rows even when one key takes nearly all of the mass.
-            const float neg_m = -m_ref;
+            // ---- sweep 2: probabilities.  l_run sums the fp32 values (it feeds the log-sum-exp that a2-L
+            // reuses); l_out sums the bf16-rounded ones that P.V actually multiplies, so that
+            // out = sum(p~ v) / sum(p~) stays a convex combination of V rows even when one key takes nearly
+            // all of the mass.  P piece c (16 packed columns) lands on S columns that sweep 2 has already read.
+            const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
             float sum4[4] = {0.f, 0.f, 0.f, 0.f}, sumr4[4] = {0.f, 0.f, 0.f, 0.f};
+            // One 32-column piece: exponentials, bf16 packing, P store.  The loop below is ROLLED over pairs of
+            // pieces so the hot code stays small enough for the instruction cache of a scheduler running two
+            // of these warps, and the load of the next piece is in flight while the current one is computed.
+            auto piece = [&](uint32_t (&v)[32], int c) {
+                const int lim_c = lim - c * 32;
+                if (lim_c < 32) {
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
+                    for (int q = 0; q < 32; ++q)
+                        if (q >= lim_c) v[q] = 0xff800000u;
+                }
                 uint32_t packed[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float p0 = ex2(fmaf(__uint_as_float(sreg[c4 * 32 + 2 * i]), scale2, neg_m));
-                    float p1 = ex2(fmaf(__uint_as_float(sreg[c4 * 32 + 2 * i + 1]), scale2, neg_m));
-                    if (NEED_LSE) { sum4[i & 3] += p0; sum4[(i + 2) & 3] += p1; }
-                    packed[i] = pack_bf16(p0, p1);
+                for (int q = 0; q < 16; ++q) {
+                    float p0 = ex2(fmaf(__uint_as_float(v[2 * q]), scale2, neg_m));
+                    float p1 = ex2(fmaf(__uint_as_float(v[2 * q + 1]), scale2, neg_m));
+                    if (NEED_LSE) { sum4[q & 3] += p0; sum4[(q + 2) & 3] += p1; }
+                    packed[q] = pack_bf16(p0, p1);
                     if (WITH_PV) {
-                        sumr4[i & 3] += __uint_as_float(packed[i] << 16);
-                        sumr4[(i + 2) & 3] += __uint_as_float(packed[i] & 0xffff0000u);
+                        sumr4[q & 3] += __uint_as_float(packed[q] << 16);
+                        sumr4[(q + 2) & 3] += __uint_as_float(packed[q] & 0xffff0000u);
                     }
                 }
-                if (WITH_PV) tmem_st16(tmS(b) + lane_base + c4 * 16, packed);
+                if (WITH_PV) tmem_st16(s_addr + c * 16, packed);
+            };
+            {
+                uint32_t va[32], vb[32];
+                tmem_ld32(s_addr, va);
+#pragma unroll 1
+                for (int c = 0; c < 4; c += 2) {
+                    tmem_wait_ld();                                  // piece c has landed in va
+                    tmem_ld32(s_addr + (c + 1) * 32, vb);
+                    piece(va, c);
+                    tmem_wait_ld();                                  // piece c+1 has landed in vb
+                    if (c + 2 < 4) tmem_ld32(s_addr + (c + 2) * 32, va);
+                    piece(vb, c + 1);
+                }
             }
             l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
             l_out += (sumr4[0] + sumr4[1]) + (sumr4[2] + sumr4[3]);
+            if (WITH_PV && warp == 0) CITRUS_TR(52 + 5 * i);
             if (WITH_PV) tmem_wait_st();
+            if (WITH_PV && warp == 0) CITRUS_TR(53 + 5 * i);
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars->p_full[b]));
-            if (WITH_PV && warp == 0) CITRUS_TR(51 + 2 * j);
+            mbar_arrive(smem_u32(&bars->p_full[wg]));
+            if (WITH_PV && warp == 0) CITRUS_TR(54 + 5 * i);
         }
-        if (ok && nt > 0) {
+        // ---- epilogue: merge the two warpgroups' partial results
+        if (ok && WITH_PV && i_last >= 0) {
+            // phases 0..i_last-1 of o_done[wg] are known complete (see the rescale note), so this parity
+            // wait can only mean "P.V of this warpgroup's last tile has retired"
+            ok = mbar_wait_warp(smem_u32(&bars->o_done[wg]), i_last & 1, p.status);
+        }
+        bars->rows[wg][row_in_tile] = RowState{m_ref, l_run, l_out};
+        mbar_arrive(smem_u32(&bars->xch));
+        ok = mbar_wait_warp(smem_u32(&bars->xch), 0, p.status) && ok;
+        if (ok) {
+            tc_fence_after();
+            if (warp == 0) CITRUS_TR(110);
+            const RowState mine = bars->rows[wg][row_in_tile], other = bars->rows[wg ^ 1][row_in_tile];
+            const float M = fmaxf(mine.m, other.m);                  // finite: tile 0 always has a visible column
+            const float w_mine = mine.m == -INFINITY ? 0.f : ex2(mine.m - M);
+            const float w_other = other.m == -INFINITY ? 0.f : ex2(other.m - M);
             if (WITH_PV) {
-                // o_done completes one phase per tile.  Only tiles 0..nt-3 are known to have retired here
-                // (their P.V precedes the last S tile in issue order), so wait for tile nt-2 first: a
-                // parity wait alone cannot tell "tile nt-1 done" from "tile nt-2 still running".
-                if (nt > 1) ok = mbar_wait_warp(smem_u32(&bars->o_done), (nt - 2) & 1, p.status);
-                if (ok) ok = mbar_wait_warp(smem_u32(&bars->o_done), (nt - 1) & 1, p.status);
-                if (ok) {
-                    if (warp == 0) CITRUS_TR(110);
-                    tc_fence_after();
-                    const float inv = 1.f / l_out;
-                    __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + ((size_t)r * p.q_heads + h) * kD;
+                // this thread finishes columns [64 wg, 64 wg + 64) of its row, from both accumulators
+                const float w0 = wg == 0 ? w_mine : w_other, w1 = wg == 0 ? w_other : w_mine;
+                const bool has1 = nt > 1;                            // O[1] was written at all
+                const float inv = 1.f / (mine.lo * w_mine + other.lo * w_other);
+                const float a0 = w0 * inv, a1 = w1 * inv;
+                uint8_t* stage = gQ + wg * kHalfBytes + row_in_tile * 128;   // [128 rows][64 bf16], 128-byte swizzle
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t oreg[32];
-                        tmem_ld32(tmO + lane_base + c * 32, oreg);
-                        tmem_wait_ld();
-                        if (r < p.rows) {
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t o0[32], o1[32];
+                    tmem_ld32(tmO(0) + lane_base + wg * 64 + c * 32, o0);
+                    if (has1) tmem_ld32(tmO(1) + lane_base + wg * 64 + c * 32, o1);
+                    tmem_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                uint4 v;
-                                v.x = pack_bf16(__uint_as_float(oreg[8 * i + 0]) * inv, __uint_as_float(oreg[8 * i + 1]) * inv);
-                                v.y = pack_bf16(__uint_as_float(oreg[8 * i + 2]) * inv, __uint_as_float(oreg[8 * i + 3]) * inv);
-                                v.z = pack_bf16(__uint_as_float(oreg[8 * i + 4]) * inv, __uint_as_float(oreg[8 * i + 5]) * inv);
-                                v.w = pack_bf16(__uint_as_float(oreg[8 * i + 6]) * inv, __uint_as_float(oreg[8 * i + 7]) * inv);
-                                *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = v;
-                            }
+                    for (int q = 0; q < 4; ++q) {
+                        float v[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            v[e] = __uint_as_float(o0[8 * q + e]) * a0;
+                            if (has1) v[e] = fmaf(__uint_as_float(o1[8 * q + e]), a1, v[e]);
                         }
+                        uint4 u;
+                        u.x = pack_bf16(v[0], v[1]); u.y = pack_bf16(v[2], v[3]);
+                        u.z = pack_bf16(v[4], v[5]); u.w = pack_bf16(v[6], v[7]);
+                        const int chunk = c * 4 + q;                 // 16-byte chunk inside the 128-byte row
+                        *reinterpret_cast<uint4*>(stage + ((chunk ^ (row_in_tile & 7)) << 4)) = u;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(smem_u32(&bars->out_ready[wg]));
+                if ((warp & 3) == 0) {
+                    // one warp per warpgroup stores its 128 x 64 half of the output tile
+                    if (mbar_wait_warp(smem_u32(&bars->out_ready[wg]), 0, p.status)) {
+                        if (elect_one()) {
+                            tma_store_3d(&mapO, sQ + wg * kHalfBytes, wg * 64, h, q_row0);
+                            tma_store_wait_read();
+                        }
+                        __syncwarp();
                     }
                 }
             }
-            if (NEED_LSE && ok && r < p.rows && p.lse2 != nullptr) p.lse2[(size_t)h * p.lse_stride + r] = m_ref + log2f(l_run);
+            if (NEED_LSE && wg == 0 && r < p.rows && p.lse2 != nullptr)
+                p.lse2[(size_t)h * p.lse_stride + r] = M + log2f(mine.l * w_mine + other.l * w_other);
         }
     }
     if (WITH_PV && warp == 0) CITRUS_TR(111);
     tc_fence_before();
     __syncthreads();
     if (WITH_PV && warp == 0) CITRUS_TR(112);
-    if (warp == 5) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
+    if (warp == 9) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
 }
 
 // ------------------------------------------------------------------ column sums (a2 pass 2)
@@ -505,7 +585,7 @@ constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 2048;
 
 // grid: (candidate tiles, kv_heads).  Accumulator rows = 128 candidates, columns = scoring rows of one
 // (head, row block); thread i owns candidate i and adds exp2(logit2 - lse2[row]) over its columns.
-__global__ void __launch_bounds__(kAttnThreads, 1)
+__global__ void __launch_bounds__(kColThreads, 1)
 colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
               const __grid_constant__ CUtensorMap mapSK, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -562,7 +642,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         for (int it = 0; it < nb && ok; ++it) {
             const int s = it % kColStages, b = it & 1;
             const int rb = rb0 + it % rb_per_head;
-            const int ncols = min(kTile, ((p.rows - rb * kTile) + 15) & ~15);
+            const int ncols = min(kTile, ((p.rows - rb * kTile) + 31) & ~31);     // whole 32-column pieces
             ok = mbar_wait_warp(smem_u32(&bars->q_full[s]), (it / kColStages) & 1, p.status);
             if (!ok) break;
             ok = mbar_wait_warp(smem_u32(&bars->s_free[b]), ((it >> 1) & 1) ^ 1, p.status);
@@ -588,7 +668,6 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (p.causal && !from_cache) r_first = max(0, key_row0 + key_in_tile - p.t0);
         float acc = 0.f;
         bool ok = true;
-        uint32_t sreg[128];
         for (int it = 0; it < nb; ++it) {
             const int b = it & 1;
             const int h = g * G + it / rb_per_head;
@@ -606,34 +685,36 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             }
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 1) & 1, p.status);
             if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (c * 32 < ncols) tmem_ld32(tmS(b) + lane_base + c * 32, sreg + c * 32);
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(smem_u32(&bars->s_free[b]));
             if (warp == 0) CITRUS_TR(160 + 3 * (it & 7));
             ok = mbar_wait_warp(smem_u32(&bars->lse_full[lb]), (it >> 2) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(161 + 3 * (it & 7));
+            tc_fence_after();
             const float4* lse4 = reinterpret_cast<const float4*>(bars->lse[lb]);
-            const int c_lo = max(0, r_first - r0);
+            const int c_lo = max(0, r_first - r0);                 // first column (scoring row) this candidate is visible to
+            const int n_pieces = (ncols + 31) >> 5;                // the MMA wrote round_up(ncols, 32) columns
             float part[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+            for (int c = 0; c < n_pieces; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tmS(b) + lane_base + c * 32, v);
+                tmem_wait_ld();
+                const int lo = c_lo - c * 32;                      // columns below lo do not see this candidate
 #pragma unroll
-            for (int c = 0; c < 128; c += 4) {
-                if (c < ncols) {                               // rows past the block end carry lse = +inf -> exp2 = 0
-                    const float4 l = lse4[c >> 2];
-                    float e0 = ex2(fmaf(__uint_as_float(sreg[c + 0]), scale2, -l.x));
-                    float e1 = ex2(fmaf(__uint_as_float(sreg[c + 1]), scale2, -l.y));
-                    float e2 = ex2(fmaf(__uint_as_float(sreg[c + 2]), scale2, -l.z));
-                    float e3 = ex2(fmaf(__uint_as_float(sreg[c + 3]), scale2, -l.w));
-                    part[0] += c + 0 >= c_lo ? e0 : 0.f;
-                    part[1] += c + 1 >= c_lo ? e1 : 0.f;
-                    part[2] += c + 2 >= c_lo ? e2 : 0.f;
-                    part[3] += c + 3 >= c_lo ? e3 : 0.f;
+                for (int q = 0; q < 32; q += 4) {
+                    const float4 l = lse4[c * 8 + (q >> 2)];        // rows past the block end carry +inf -> exp2 = 0
+                    float e0 = ex2(fmaf(__uint_as_float(v[q + 0]), scale2, -l.x));
+                    float e1 = ex2(fmaf(__uint_as_float(v[q + 1]), scale2, -l.y));
+                    float e2 = ex2(fmaf(__uint_as_float(v[q + 2]), scale2, -l.z));
+                    float e3 = ex2(fmaf(__uint_as_float(v[q + 3]), scale2, -l.w));
+                    part[0] += q + 0 >= lo ? e0 : 0.f;
+                    part[1] += q + 1 >= lo ? e1 : 0.f;
+                    part[2] += q + 2 >= lo ? e2 : 0.f;
+                    part[3] += q + 3 >= lo ? e3 : 0.f;
                 }
             }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->s_free[b]));
             acc += (part[0] + part[1]) + (part[2] + part[3]);
             if (warp == 0) CITRUS_TR(162 + 3 * (it & 7));
         }
@@ -672,7 +753,7 @@ bool map_cache(CUtensorMap* map, const void* ptr, int cap, int heads) {
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct Maps { CUtensorMap Q, CK, CV, SK, SV; };
+struct Maps { CUtensorMap Q, CK, CV, SK, SV, O; };
 
 // The tensor map's row extent is the number of valid rows, so rows past it read as zero.
 bool build_maps(Maps* mp, const void* Qbase, int q_rows_total, const QueryRows& q, const Candidates& c, bool with_v) {
@@ -718,11 +799,12 @@ cudaError_t tc_attention(const QueryRows& q, const Candidates& c, void* out, flo
                          int* status, cudaStream_t s) {
     Maps mp;
     if (!build_maps(&mp, q.Q, q.rows, q, c, true)) return cudaErrorInvalidValue;
+    if (!map_token_major(&mp.O, out, q.rows, q.q_heads)) return cudaErrorInvalidValue;
     TcParams p = base_params(q, c, status);
     p.out = out; p.lse2 = lse2; p.lse_stride = lse_stride;
     dim3 grid((q.rows + kTile - 1) / kTile, q.q_heads);
-    if (lse2 != nullptr) attn_kernel<true, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
-    else attn_kernel<true, false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
+    if (lse2 != nullptr) attn_kernel<true, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, mp.O, p);
+    else attn_kernel<true, false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, mp.O, p);
     return cudaGetLastError();
 }
 
@@ -730,10 +812,11 @@ cudaError_t tc_score_lse(const QueryRows& q, const Candidates& c, float* lse2, i
                          int* status, cudaStream_t s) {
     Maps mp;
     if (!build_maps(&mp, q.Q, q.rows, q, c, false)) return cudaErrorInvalidValue;
+    mp.O = mp.Q;                                     // unused by the log-sum-exp pass
     TcParams p = base_params(q, c, status);
     p.out = nullptr; p.lse2 = lse2; p.lse_stride = lse_stride;
     dim3 grid((q.rows + kTile - 1) / kTile, q.q_heads);
-    attn_kernel<false, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, p);
+    attn_kernel<false, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, mp.O, p);
     return cudaGetLastError();
 }
 
@@ -745,7 +828,7 @@ cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse2
     p.lse_in = lse2; p.lse_stride = lse_stride; p.scores = scores; p.score_stride = score_stride;
     const int n_tiles = (c.m + kTile - 1) / kTile + (c.L + kTile - 1) / kTile;
     dim3 grid(n_tiles, c.kv_heads);
-    colsum_kernel<<<grid, kAttnThreads, kColSmemBytes, s>>>(mp.Q, mp.CK, mp.SK, p);
+    colsum_kernel<<<grid, kColThreads, kColSmemBytes, s>>>(mp.Q, mp.CK, mp.SK, p);
     return cudaGetLastError();
 }
 
