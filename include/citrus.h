@@ -155,11 +155,11 @@ int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
  * the number of launches per kernel id since the last read into ms[CITRUS_N_KERNELS]
  * and launches[CITRUS_N_KERNELS] (host arrays), and clears the record.
  */
-#define CITRUS_KERNEL_ATTENTION 0   /* a1 */
-#define CITRUS_KERNEL_SCORE_LSE 1   /* a2, log-sum-exp pass of the instruction queries */
+#define CITRUS_KERNEL_ATTENTION 0   /* a1 (bf16 path: one launch with the log-sum-exp pass of a2) */
+#define CITRUS_KERNEL_SCORE_LSE 1   /* a2, log-sum-exp pass of the instruction queries (fp32 path only) */
 #define CITRUS_KERNEL_COLSUM    2   /* a2, column sums (instruction and LM) */
-#define CITRUS_KERNEL_SELECT    3   /* a3 */
-#define CITRUS_KERNEL_COMPACT   4   /* a4 */
+#define CITRUS_KERNEL_SELECT    3   /* a3 (separate launch only with CITRUS_MODE_LAYERWISE) */
+#define CITRUS_KERNEL_COMPACT   4   /* a4 (per-head granularity: one launch with a3) */
 #define CITRUS_N_KERNELS        5
 int citrus_profile(citrus_handle h, int enable);
 int citrus_profile_read(citrus_handle h, double* ms, long long* launches);

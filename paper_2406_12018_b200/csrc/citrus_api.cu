@@ -27,6 +27,7 @@ struct Unit {                       // one (layer, sequence slot)
     int* idx = nullptr;             // [n_caches, kv_heads, budget_k]
     float* lse_chunk = nullptr;     // [q_heads, chunk_s]
     float* lse_instr = nullptr;     // [q_heads, CITRUS_MAX_INSTR]
+    float* part = nullptr;          // key-split (max, sum) pairs of a2 pass 1 [splits, q_heads, CITRUS_MAX_INSTR] (tensor-core path)
     int m = 0;                      // rows retained in every cache
     long long tokens_seen = 0;
     int last_n = 0, last_kept = 0, last_m = 0;
@@ -106,6 +107,7 @@ int alloc_units(citrus_ctx* c) {
         if ((rc = dev_alloc(c, (void**)&u.idx, (size_t)c->n_caches * c->Hkv * c->k * sizeof(int), true))) return rc;
         if ((rc = dev_alloc(c, (void**)&u.lse_chunk, (size_t)c->Hq * c->ls * sizeof(float), true))) return rc;
         if ((rc = dev_alloc(c, (void**)&u.lse_instr, (size_t)c->Hq * CITRUS_MAX_INSTR * sizeof(float), true))) return rc;
+        if (c->use_tc && (rc = dev_alloc(c, (void**)&u.part, (size_t)kTcMaxLseSplits * c->Hq * CITRUS_MAX_INSTR * 2 * sizeof(float), true))) return rc;
     }
     return CITRUS_OK;
 }
@@ -162,12 +164,23 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     const int ic = c->individual ? 1 : 0;     // the cache scored by the instruction text
 
     cudaError_t e;
-    // a1: attention of the chunk over [cache 0 ; chunk], row log-sum-exp kept for a2-L
-    {
+    float* lse_chunk = c->individual ? u.lse_chunk : nullptr;     // only a2-L reads a1's row log-sum-exp
+    int splits = 1;
+    if (c->use_tc) {
+        // a1 and pass 1 of a2-I (row log-sum-exp of the instruction queries, possibly split over key ranges): one launch
+        splits = tc_lse_splits(nI, c->Hq, m, L, ((L + 127) / 128) * c->Hq);
         LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
-        float* lse_chunk = c->individual ? u.lse_chunk : nullptr;     // only a2-L reads it
-        if (c->use_tc) e = tc_attention(q_chunk, cand[0], out, lse_chunk, c->ls, c->status, st);
-        else e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, lse_chunk, c->ls, st);
+        e = tc_attention_lse(q_chunk, cand[0], out, lse_chunk, c->ls, q_instr, cand[ic], u.lse_instr, u.part,
+                             CITRUS_MAX_INSTR, splits, c->status, st);
+    } else {
+        {
+            LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
+            e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, lse_chunk, c->ls, st);
+        }
+        if (e == cudaSuccess) {
+            LaunchTimer t(c, CITRUS_KERNEL_SCORE_LSE, st);
+            e = simt_attention(c->fp32, c->D, q_instr, cand[ic], nullptr, u.lse_instr, CITRUS_MAX_INSTR, st);
+        }
     }
     if (e != cudaSuccess) return cuda_rc(e);
 
@@ -177,25 +190,20 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         const char* q0 = reinterpret_cast<const char*>(Qc) + (size_t)(L - w) * c->Hq * c->D * c->elt;
         QueryRows q_lm{q0, w, c->Hq, 1, L - w};
         LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
-        if (c->use_tc) e = tc_colsum(q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, c->status, st);
+        if (c->use_tc) e = tc_colsum(q_lm, cand[0], u.lse_chunk + (L - w), c->ls, 1, scores[0], c->score_stride, c->status, st);
         else e = simt_colsum(c->fp32, c->D, q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, st);
         if (e != cudaSuccess) return cuda_rc(e);
     }
-    // a2-I: Eq. 1 with the instruction queries over the instruction-side cache's candidates
-    {
-        LaunchTimer t(c, CITRUS_KERNEL_SCORE_LSE, st);
-        if (c->use_tc) e = tc_score_lse(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, c->status, st);
-        else e = simt_attention(c->fp32, c->D, q_instr, cand[ic], nullptr, u.lse_instr, CITRUS_MAX_INSTR, st);
-    }
-    if (e != cudaSuccess) return cuda_rc(e);
+    // a2-I pass 2: Eq. 1 column sums of the instruction queries over the instruction-side cache's candidates
     {
         LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
-        if (c->use_tc) e = tc_colsum(q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, c->status, st);
+        if (c->use_tc) e = tc_colsum(q_instr, cand[ic], splits > 1 ? u.part : u.lse_instr, CITRUS_MAX_INSTR, splits,
+                                     scores[ic], c->score_stride, c->status, st);
         else e = simt_colsum(c->fp32, c->D, q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, st);
     }
     if (e != cudaSuccess) return cuda_rc(e);
 
-    // a3 + a4 for every cache in one launch each
+    // a3 + a4 for every cache
     SelectJob sj[2];
     CompactJob cj[2];
     for (int ci = 0; ci < c->n_caches; ++ci) {
@@ -205,16 +213,23 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
                             cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, m};
     }
-    {
-        LaunchTimer t(c, CITRUS_KERNEL_SELECT, st);
-        e = select_topk(sj, c->n_caches, c->Hkv, n, c->k, c->layerwise ? 1 : 0, st);
-    }
-    if (e != cudaSuccess) return cuda_rc(e);
-    {
+    if (!c->layerwise) {
+        // one cluster launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-        e = compact_kv(cj, c->n_caches, Kc, Vc, c->Hkv, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
+        e = select_compact(sj, cj, c->n_caches, Kc, Vc, c->Hkv, n, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
+        if (e != cudaSuccess) return cuda_rc(e);
+    } else {
+        {
+            LaunchTimer t(c, CITRUS_KERNEL_SELECT, st);
+            e = select_topk(sj, c->n_caches, c->Hkv, n, c->k, 1, st);
+        }
+        if (e != cudaSuccess) return cuda_rc(e);
+        {
+            LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
+            e = compact_kv(cj, c->n_caches, Kc, Vc, c->Hkv, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
+        }
+        if (e != cudaSuccess) return cuda_rc(e);
     }
-    if (e != cudaSuccess) return cuda_rc(e);
 
     for (int ci = 0; ci < c->n_caches; ++ci) u.cache[ci].cur ^= 1;
     u.last_n = n; u.last_kept = kept; u.last_m = m; u.has_step = true;

@@ -40,11 +40,17 @@ cudaError_t simt_colsum(bool is_fp32, int D, const QueryRows& q, const Candidate
 
 // ---- tensor-core (tcgen05 / TMEM / TMA) path: bf16, D = 128 ----------------
 cudaError_t tc_init();   // resolves the driver entry point for tensor-map encoding
-cudaError_t tc_attention(const QueryRows& q, const Candidates& c, void* out, float* lse2, int lse_stride,
-                         int* status, cudaStream_t s);
-cudaError_t tc_score_lse(const QueryRows& q, const Candidates& c, float* lse2, int lse_stride,
-                         int* status, cudaStream_t s);
-cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse2, int lse_stride,
+// Number of key splits for pass 1 of a2-I (1 = the pass writes final log-sum-exp values).
+int tc_lse_splits(int n_rows, int q_heads, int m, int L, int n_attn_items);
+constexpr int kTcMaxLseSplits = 8;
+// One launch: a1 (qa over ca -> out, optional row log-sum-exp) and pass 1 of a2-I (qi over ci).  Either part
+// may be empty (rows == 0).  With splits > 1 the pass writes (max, sum) pairs to `part`
+// [splits, q_heads, lse_instr_stride] (float2), otherwise log-sum-exp values to lse_instr.
+cudaError_t tc_attention_lse(const QueryRows& qa, const Candidates& ca, void* out, float* lse_chunk, int lse_chunk_stride,
+                             const QueryRows& qi, const Candidates& ci, float* lse_instr, float* part, int lse_instr_stride,
+                             int splits, int* status, cudaStream_t s);
+// Pass 2: column sums; lse_or_part is the matching output of pass 1 (or a1's row log-sum-exp with splits = 1).
+cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse_or_part, int lse_stride, int splits,
                       float* scores, int score_stride, int* status, cudaStream_t s);
 
 // ---- select (a3) and compaction (a4) ---------------------------------------
@@ -64,4 +70,7 @@ struct CompactJob {
 };
 cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
                        int kv_heads, int cap, int row_bytes, int kept, int chunk_pos0, cudaStream_t s);
+// a3 + a4 in one launch (per-head granularity): clusters of CTAs per (cache, KV head).
+cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
+                           int kv_heads, int n, int k, int row_bytes, int kept, int chunk_pos0, cudaStream_t s);
 }  // namespace citrus

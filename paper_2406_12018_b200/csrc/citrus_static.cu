@@ -75,8 +75,9 @@ extern "C" int citrus_importance_static(const void* Q_s, int n_s, const void* K,
         e = simt_attention(true, head_dim, q, cand, nullptr, lse, lse_stride, st);
         if (e == cudaSuccess) e = simt_colsum(true, head_dim, q, cand, lse, lse_stride, scores, score_stride, st);
     } else {
-        e = tc_score_lse(q, cand, lse, lse_stride, status, st);
-        if (e == cudaSuccess) e = tc_colsum(q, cand, lse, lse_stride, scores, score_stride, status, st);
+        const QueryRows none{nullptr, 0, q_heads, 0, 0};
+        e = tc_attention_lse(none, cand, nullptr, nullptr, 0, q, cand, lse, nullptr, lse_stride, 1, status, st);
+        if (e == cudaSuccess) e = tc_colsum(q, cand, lse, lse_stride, 1, scores, score_stride, status, st);
     }
     if (e != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
     return CITRUS_OK;

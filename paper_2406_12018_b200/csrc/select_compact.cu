@@ -22,15 +22,12 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 // select finds the k-th largest key T and how many candidates equal to T are kept;
 // a flagged block scan in index order then emits kept indices ascending, taking the
 // lowest-index candidates among those equal to T.
-__global__ void __launch_bounds__(kSelThreads)
-select_topk_kernel(SelectArgs args, int kv_heads, int n, int k, int layerwise) {
-    extern __shared__ uint32_t keys[];            // [n]
+__device__ __forceinline__ void select_body(const SelectJob& job, const int g, int kv_heads, int n, int k, int layerwise,
+                                            uint32_t* keys /* shared, [n] */) {
     __shared__ uint32_t hist[256];
     __shared__ uint32_t s_prefix, s_remaining;
     __shared__ uint32_t warp_gt[32], warp_eq[32];
 
-    const SelectJob job = args.job[blockIdx.y];
-    const int g = blockIdx.x;
     const int tid = threadIdx.x;
     const int heads_out = layerwise ? kv_heads : 1;
     int* idx0 = job.idx + (size_t)g * k;
@@ -132,27 +129,24 @@ select_topk_kernel(SelectArgs args, int kv_heads, int n, int k, int layerwise) {
     }
 }
 
-// Rows are copied with 128-bit accesses, row_bytes/16 lanes per row.
-// grid: (row tiles, KV heads, caches)
-constexpr int kCompactThreads = 256;
-constexpr int kCompactRowsPerCta = 64;
+__global__ void __launch_bounds__(kSelThreads)
+select_topk_kernel(SelectArgs args, int kv_heads, int n, int k, int layerwise) {
+    extern __shared__ uint32_t keys[];            // [n]
+    select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, n, k, layerwise, keys);
+}
 
-__global__ void __launch_bounds__(kCompactThreads)
-compact_kv_kernel(CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
-                  int kv_heads, int cap, int row_vecs, int kept, int chunk_pos0) {
-    const CompactJob job = args.job[blockIdx.z];
-    const int g = blockIdx.y;
-    const int r_base = blockIdx.x * kCompactRowsPerCta;
-    const int rows_per_pass = kCompactThreads / row_vecs;
+// Rows [r_begin, r_end) of one (cache, head) are copied with 128-bit accesses, row_bytes/16 lanes per row.
+__device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4* __restrict__ chunkK,
+                                             const uint4* __restrict__ chunkV, const int g, int kv_heads, int cap,
+                                             int row_vecs, int r_begin, int r_end, int chunk_pos0) {
+    const int rows_per_pass = blockDim.x / row_vecs;
     const int sub = threadIdx.x / row_vecs, v = threadIdx.x % row_vecs;
     const int* idx = job.idx + (size_t)g * cap;
     const uint4* srcK = reinterpret_cast<const uint4*>(job.srcK);
     const uint4* srcV = reinterpret_cast<const uint4*>(job.srcV);
     uint4* dstK = reinterpret_cast<uint4*>(job.dstK);
     uint4* dstV = reinterpret_cast<uint4*>(job.dstV);
-    for (int rr = sub; rr < kCompactRowsPerCta; rr += rows_per_pass) {
-        const int r = r_base + rr;
-        if (r >= kept) break;
+    for (int r = r_begin + sub; r < r_end; r += rows_per_pass) {
         const int j = idx[r];
         const uint4 *pk, *pv;
         if (j < job.m) {
@@ -168,6 +162,37 @@ compact_kv_kernel(CompactArgs args, const uint4* __restrict__ chunkK, const uint
         dstV[doff] = b;
         if (v == 0) job.dstPos[(size_t)g * cap + r] = j < job.m ? job.srcPos[(size_t)g * cap + j] : chunk_pos0 + (j - job.m);
     }
+}
+
+// grid: (row tiles, KV heads, caches)
+constexpr int kCompactThreads = 256;
+constexpr int kCompactRowsPerCta = 64;
+
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kv_kernel(CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
+                  int kv_heads, int cap, int row_vecs, int kept, int chunk_pos0) {
+    const int r0 = blockIdx.x * kCompactRowsPerCta;
+    compact_rows(args.job[blockIdx.z], chunkK, chunkV, blockIdx.y, kv_heads, cap, row_vecs,
+                 r0, min(kept, r0 + kCompactRowsPerCta), chunk_pos0);
+}
+
+// a3 + a4 in one launch: a cluster of kFusedCluster CTAs per (cache, KV head).  The first CTA of the cluster
+// selects, the cluster barrier publishes the index list, then every CTA gathers its share of the kept rows.
+// grid: (kFusedCluster, KV heads, caches), cluster (kFusedCluster, 1, 1)
+constexpr int kFusedCluster = 8;
+
+__global__ void __launch_bounds__(kSelThreads)
+select_compact_kernel(SelectArgs sel, CompactArgs cmp, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
+                      int kv_heads, int n, int k, int row_vecs, int kept, int chunk_pos0) {
+    extern __shared__ uint32_t keys[];            // [n], used by the selecting CTA only
+    const int g = blockIdx.y;
+    if (blockIdx.x == 0) select_body(sel.job[blockIdx.z], g, kv_heads, n, k, 0, keys);
+    // hardware cluster barrier with release/acquire semantics: the index list written above is visible to all
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    const int per = (kept + kFusedCluster - 1) / kFusedCluster;
+    const int r0 = blockIdx.x * per;
+    compact_rows(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, k, row_vecs, r0, min(kept, r0 + per), chunk_pos0);
 }
 
 }  // namespace
@@ -186,6 +211,30 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, 
     dim3 grid(layerwise ? 1 : kv_heads, n_jobs);
     select_topk_kernel<<<grid, kSelThreads, smem, s>>>(a, kv_heads, n, k, layerwise);
     return cudaGetLastError();
+}
+
+cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
+                           int kv_heads, int n, int k, int row_bytes, int kept, int chunk_pos0, cudaStream_t s) {
+    if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
+    SelectArgs sa; CompactArgs ca;
+    for (int i = 0; i < n_jobs; ++i) { sa.job[i] = sjobs[i]; ca.job[i] = cjobs[i]; }
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kFusedCluster, kv_heads, n_jobs);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = (size_t)n * sizeof(uint32_t);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kFusedCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, select_compact_kernel, sa, ca, reinterpret_cast<const uint4*>(chunkK),
+                              reinterpret_cast<const uint4*>(chunkV), kv_heads, n, k, row_bytes / 16, kept, chunk_pos0);
 }
 
 cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,

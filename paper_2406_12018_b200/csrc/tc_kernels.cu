@@ -3,8 +3,9 @@
 // tcgen05.mma accumulates in tensor memory, and the softmax / column-sum warps read
 // the accumulators back with tcgen05.ld.  Three kernels share the machinery:
 //
-//   attn_kernel<true,*> a1: causal attention of the chunk over [cache ; chunk] (+ row LSE)
-//   attn_kernel<false,*> a2 pass 1: row log-sum-exp of the scoring queries over all candidates
+//   attn_lse_kernel     one launch of attn_body items:
+//     attn_body<true,*>   a1: causal attention of the chunk over [cache ; chunk] (+ row LSE)
+//     attn_body<false,*>  a2 pass 1: row log-sum-exp of the scoring queries over (a split of) the candidates
 //   colsum_kernel       a2 pass 2: S^T = K Q^T with the candidates on the accumulator's rows,
 //                       so the column sum of Eq. 1 over scoring rows is a per-thread sum
 //
@@ -17,7 +18,7 @@
 // Optional cycle stamps of one CTA's roles (build with -DCITRUS_TRACE; compiled out otherwise).
 #ifdef CITRUS_TRACE
 __device__ unsigned long long g_citrus_trace[256];
-#define CITRUS_TR(i) do { if (blockIdx.x == gridDim.x - 1 && blockIdx.y == 0 && (threadIdx.x & 31) == 0) \
+#define CITRUS_TR(i) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0) \
                               g_citrus_trace[(i)] = clock64(); } while (0)
 extern "C" int citrus_trace_read(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_citrus_trace, sizeof(g_citrus_trace)); }
 extern "C" int citrus_trace_clear() { static unsigned long long z[256]; return (int)cudaMemcpyToSymbol(g_citrus_trace, z, sizeof(z)); }
@@ -193,6 +194,8 @@ struct TcParams {
     void* out;       // [rows, q_heads, 128] bf16 or null
     float* lse2;     // [q_heads, lse_stride]
     int lse_stride;
+    float2* part;    // a2 pass 1 with key splits: (max, sum) of every (split, head, row), [splits, q_heads, lse_stride]
+    int splits;      // number of key splits (1: lse2 / lse_in hold final log-sum-exp values)
     const float* lse_in;   // colsum: log-sum-exp of the scoring rows
     float* scores;   // colsum: [kv_heads, score_stride]
     int score_stride;
@@ -247,6 +250,7 @@ constexpr int kStagesV = 2;             // V ring
 constexpr int kAttnThreads = 352;       // 2 softmax warpgroups (8 warps), K-TMA warp, MMA warp, V-TMA warp
 constexpr int kColThreads = 192;        // 4 column-sum warps, 1 TMA warp, 1 MMA warp
 constexpr int kTmemCols = 512;
+constexpr int kMaxLseSplits = 8;
 constexpr float kRescaleTau = 8.f;      // rescale O only when the row max grows by more than 2^8
 
 // Bulk tensor store shared -> global (rows past the tensor map's extent are clipped).
@@ -275,11 +279,10 @@ constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + kStagesK
 // anything inside the loop and each scheduler always has a second warp to run.  The two partial results
 // are merged once, in the epilogue:  out = (w0 O[0] + w1 O[1]) / (w0 l0 + w1 l1),  w_b = 2^(m_b - max m).
 template <bool WITH_PV, bool NEED_LSE>
-__global__ void __launch_bounds__(kAttnThreads, 1)
-attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
-            const __grid_constant__ CUtensorMap mapCV, const __grid_constant__ CUtensorMap mapSK,
-            const __grid_constant__ CUtensorMap mapSV, const __grid_constant__ CUtensorMap mapO, const TcParams p) {
-    extern __shared__ uint8_t smem_raw[];
+__device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtensorMap& mapCK, const CUtensorMap& mapCV,
+                                          const CUtensorMap& mapSK, const CUtensorMap& mapSV, const CUtensorMap& mapO,
+                                          const TcParams& p, const int qt, const int h, const int tile_begin, int tile_end,
+                                          const int split, uint8_t* smem_raw) {
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = base;
     const uint32_t sK = sQ + kTileBytes;
@@ -288,7 +291,6 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
     AttnSmem* bars = reinterpret_cast<AttnSmem*>(smem_raw + (sV + kStagesV * kTileBytes - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int qt = blockIdx.x, h = blockIdx.y;
     const int g = h / (p.q_heads / p.kv_heads);
     if (WITH_PV && warp == 0) CITRUS_TR(0);
     const int q_row0 = qt * kTile;                                  // first row of this tile inside the block
@@ -299,7 +301,9 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
         int last_t = p.t0 + min(q_row0 + kTile, p.rows) - 1;         // highest chunk index among the rows
         n_chunk_tiles = min(n_chunk_tiles, last_t / kTile + 1);
     }
-    const int nt = n_cache_tiles + n_chunk_tiles;
+    // this CTA sweeps key tiles [tile_begin, tile_end) of the candidate list; j below is local to that range
+    tile_end = min(tile_end, n_cache_tiles + n_chunk_tiles);
+    const int nt = max(0, tile_end - tile_begin);
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars->q_full), 1);
@@ -327,9 +331,9 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
         // ---------------------------------------------------------------- K (and Q) TMA producer (converged warp)
         load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
         for (int j = 0; j < nt; ++j) {
-            const int s = j % kStagesK;
-            const bool from_cache = j < n_cache_tiles;
-            const int row = from_cache ? j * kTile : (j - n_cache_tiles) * kTile;
+            const int s = j % kStagesK, jg = tile_begin + j;
+            const bool from_cache = jg < n_cache_tiles;
+            const int row = from_cache ? jg * kTile : (jg - n_cache_tiles) * kTile;
             if (!mbar_wait_warp(smem_u32(&bars->k_empty[s]), ((j / kStagesK) & 1) ^ 1, p.status)) break;
             load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, g, !from_cache);
         }
@@ -337,9 +341,9 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
         // ---------------------------------------------------------------- V TMA producer (converged warp)
         if (WITH_PV) {
             for (int j = 0; j < nt; ++j) {
-                const int s = j % kStagesV;
-                const bool from_cache = j < n_cache_tiles;
-                const int row = from_cache ? j * kTile : (j - n_cache_tiles) * kTile;
+                const int s = j % kStagesV, jg = tile_begin + j;
+                const bool from_cache = jg < n_cache_tiles;
+                const int row = from_cache ? jg * kTile : (jg - n_cache_tiles) * kTile;
                 if (!mbar_wait_warp(smem_u32(&bars->v_empty[s]), ((j / kStagesV) & 1) ^ 1, p.status)) break;
                 load_tile(sV + s * kTileBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
             }
@@ -403,10 +407,11 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
             tc_fence_after();
             // number of visible columns of this tile for this row
             int lim = kTile;
-            if (j < n_cache_tiles) {
-                lim = min(kTile, p.m - j * kTile);
+            const int jg = tile_begin + j;
+            if (jg < n_cache_tiles) {
+                lim = min(kTile, p.m - jg * kTile);
             } else {
-                const int u0 = (j - n_cache_tiles) * kTile;
+                const int u0 = (jg - n_cache_tiles) * kTile;
                 lim = min(kTile, p.L - u0);
                 if (p.causal) lim = min(lim, p.t0 + r - u0 + 1);
             }
@@ -562,8 +567,11 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
                     }
                 }
             }
-            if (NEED_LSE && wg == 0 && r < p.rows && p.lse2 != nullptr)
-                p.lse2[(size_t)h * p.lse_stride + r] = M + log2f(mine.l * w_mine + other.l * w_other);
+            if (NEED_LSE && wg == 0 && r < p.rows) {
+                const float l = mine.l * w_mine + other.l * w_other;
+                if (p.splits > 1) p.part[((size_t)split * p.q_heads + h) * p.lse_stride + r] = make_float2(M, l);
+                else if (p.lse2 != nullptr) p.lse2[(size_t)h * p.lse_stride + r] = M + log2f(l);
+            }
         }
     }
     if (WITH_PV && warp == 0) CITRUS_TR(111);
@@ -571,6 +579,34 @@ attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CU
     __syncthreads();
     if (WITH_PV && warp == 0) CITRUS_TR(112);
     if (warp == 9) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
+}
+
+// One launch for a1 and for pass 1 of a2-I.  Blocks [0, n_attn) are attention items (query tile, head),
+// longest first; the rest are log-sum-exp items (instruction row tile, head, key split), which fill the SMs
+// that a partial wave of attention items leaves idle.
+//   pa / maps Q, CK, CV, SK, SV, O : attention of the chunk over [cache 0 ; chunk]
+//   pl / maps QI, CKI, SK          : instruction queries over [instruction-side cache ; chunk]
+template <bool NEED_LSE>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
+                const __grid_constant__ CUtensorMap mapCV, const __grid_constant__ CUtensorMap mapSK,
+                const __grid_constant__ CUtensorMap mapSV, const __grid_constant__ CUtensorMap mapO,
+                const __grid_constant__ CUtensorMap mapQI, const __grid_constant__ CUtensorMap mapCKI,
+                const TcParams pa, const TcParams pl, const int n_attn) {
+    extern __shared__ uint8_t smem_raw[];
+    const int id = blockIdx.x;
+    if (id < n_attn) {
+        const int n_qt = (pa.rows + kTile - 1) / kTile;
+        const int qt = n_qt - 1 - id / pa.q_heads, h = id % pa.q_heads;      // later query tiles see more keys
+        attn_body<true, NEED_LSE>(mapQ, mapCK, mapCV, mapSK, mapSV, mapO, pa, qt, h, 0, 1 << 30, 0, smem_raw);
+    } else {
+        const int item = id - n_attn;
+        const int split = item % pl.splits, rest = item / pl.splits;
+        const int h = rest % pl.q_heads, rt = rest / pl.q_heads;
+        const int tiles = (pl.m + kTile - 1) / kTile + (pl.L + kTile - 1) / kTile;
+        const int t0 = (int)((long long)split * tiles / pl.splits), t1 = (int)((long long)(split + 1) * tiles / pl.splits);
+        attn_body<false, true>(mapQI, mapCKI, mapCKI, mapSK, mapSK, mapQI, pl, rt, h, t0, t1, split, smem_raw);
+    }
 }
 
 // ------------------------------------------------------------------ column sums (a2 pass 2)
@@ -680,7 +716,22 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             const int lb = it & 3;
             {
                 const int rr = r0 + key_in_tile;
-                bars->lse[lb][key_in_tile] = rr < p.rows ? __ldg(p.lse_in + (size_t)h * p.lse_stride + rr) : INFINITY;
+                float lse = INFINITY;
+                if (rr < p.rows) {
+                    if (p.splits > 1) {                              // merge the key splits of pass 1
+                        float M = -INFINITY, l = 0.f;
+                        for (int sp = 0; sp < p.splits; ++sp)
+                            M = fmaxf(M, __ldg(&p.part[((size_t)sp * p.q_heads + h) * p.lse_stride + rr]).x);
+                        for (int sp = 0; sp < p.splits; ++sp) {
+                            const float2 ml = __ldg(&p.part[((size_t)sp * p.q_heads + h) * p.lse_stride + rr]);
+                            l += ml.y * ex2(ml.x - M);
+                        }
+                        lse = M + log2f(l);
+                    } else {
+                        lse = __ldg(p.lse_in + (size_t)h * p.lse_stride + rr);
+                    }
+                }
+                bars->lse[lb][key_in_tile] = lse;
                 mbar_arrive(smem_u32(&bars->lse_full[lb]));
             }
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 1) & 1, p.status);
@@ -785,47 +836,70 @@ cudaError_t tc_init() {
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
     if (e != cudaSuccess) return e;
     if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+    e = cudaFuncSetAttribute(attn_lse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_lse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kColSmemBytes);
+    if (e != cudaSuccess) return e;
     g_encode = reinterpret_cast<EncodeFn>(fn);
-    e = cudaFuncSetAttribute(attn_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kColSmemBytes);
+    return cudaSuccess;
 }
 
-cudaError_t tc_attention(const QueryRows& q, const Candidates& c, void* out, float* lse2, int lse_stride,
-                         int* status, cudaStream_t s) {
-    Maps mp;
-    if (!build_maps(&mp, q.Q, q.rows, q, c, true)) return cudaErrorInvalidValue;
-    if (!map_token_major(&mp.O, out, q.rows, q.q_heads)) return cudaErrorInvalidValue;
-    TcParams p = base_params(q, c, status);
-    p.out = out; p.lse2 = lse2; p.lse_stride = lse_stride;
-    dim3 grid((q.rows + kTile - 1) / kTile, q.q_heads);
-    if (lse2 != nullptr) attn_kernel<true, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, mp.O, p);
-    else attn_kernel<true, false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, mp.O, p);
+int tc_lse_splits(int n_rows, int q_heads, int m, int L, int n_attn_items) {
+    // The log-sum-exp items share a launch with the attention items.  When those leave SMs idle (fewer items than
+    // SMs), split the key range so that there is about one short item per idle SM; otherwise keep whole sweeps,
+    // because every extra item pays a CTA prologue.
+    const int kSMs = 148;
+    const int tiles = (m + kTile - 1) / kTile + (L + kTile - 1) / kTile;
+    const int base_items = ((n_rows + kTile - 1) / kTile) * q_heads;
+    const int idle = n_attn_items < kSMs ? kSMs - n_attn_items : 0;
+    int s = idle / base_items;
+    if (s > tiles) s = tiles;
+    if (s > kMaxLseSplits) s = kMaxLseSplits;
+    return s < 1 ? 1 : s;
+}
+
+cudaError_t tc_attention_lse(const QueryRows& qa, const Candidates& ca, void* out, float* lse_chunk, int lse_chunk_stride,
+                             const QueryRows& qi, const Candidates& ci, float* lse_instr, float* part, int lse_instr_stride,
+                             int splits, int* status, cudaStream_t s) {
+    const bool has_attn = qa.rows > 0, has_lse = qi.rows > 0;
+    if (!has_attn && !has_lse) return cudaSuccess;
+    Maps ma{}, mi{};
+    CUtensorMap mapO{};
+    if (has_attn) {
+        if (!build_maps(&ma, qa.Q, qa.rows, qa, ca, true)) return cudaErrorInvalidValue;
+        if (!map_token_major(&mapO, out, qa.rows, qa.q_heads)) return cudaErrorInvalidValue;
+    }
+    if (has_lse) {
+        if (!build_maps(&mi, qi.Q, qi.rows, qi, ci, false)) return cudaErrorInvalidValue;
+    }
+    if (!has_attn) { ma = mi; mapO = mi.Q; }
+    if (!has_lse) mi = ma;
+    TcParams pa = base_params(has_attn ? qa : qi, has_attn ? ca : ci, status);
+    pa.out = out; pa.lse2 = lse_chunk; pa.lse_stride = lse_chunk_stride; pa.splits = 1;
+    TcParams pl = base_params(has_lse ? qi : qa, has_lse ? ci : ca, status);
+    pl.lse2 = lse_instr; pl.part = reinterpret_cast<float2*>(part); pl.lse_stride = lse_instr_stride; pl.splits = splits;
+    const int n_attn = has_attn ? ((qa.rows + kTile - 1) / kTile) * qa.q_heads : 0;
+    const int n_lse = has_lse ? ((qi.rows + kTile - 1) / kTile) * qi.q_heads * splits : 0;
+    dim3 grid(n_attn + n_lse);
+    // both parts read the chunk's K through the same caller tensor, so one chunk-K map serves them
+    if (lse_chunk != nullptr)
+        attn_lse_kernel<true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(ma.Q, ma.CK, ma.CV, ma.SK, ma.SV, mapO,
+                                                                        mi.Q, mi.CK, pa, pl, n_attn);
+    else
+        attn_lse_kernel<false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(ma.Q, ma.CK, ma.CV, ma.SK, ma.SV, mapO,
+                                                                         mi.Q, mi.CK, pa, pl, n_attn);
     return cudaGetLastError();
 }
 
-cudaError_t tc_score_lse(const QueryRows& q, const Candidates& c, float* lse2, int lse_stride,
-                         int* status, cudaStream_t s) {
-    Maps mp;
-    if (!build_maps(&mp, q.Q, q.rows, q, c, false)) return cudaErrorInvalidValue;
-    mp.O = mp.Q;                                     // unused by the log-sum-exp pass
-    TcParams p = base_params(q, c, status);
-    p.out = nullptr; p.lse2 = lse2; p.lse_stride = lse_stride;
-    dim3 grid((q.rows + kTile - 1) / kTile, q.q_heads);
-    attn_kernel<false, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mp.Q, mp.CK, mp.CV, mp.SK, mp.SV, mp.O, p);
-    return cudaGetLastError();
-}
-
-cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse2, int lse_stride,
+cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse_or_part, int lse_stride, int splits,
                       float* scores, int score_stride, int* status, cudaStream_t s) {
     Maps mp;
     if (!build_maps(&mp, q.Q, q.rows, q, c, false)) return cudaErrorInvalidValue;
     TcParams p = base_params(q, c, status);
-    p.lse_in = lse2; p.lse_stride = lse_stride; p.scores = scores; p.score_stride = score_stride;
+    p.lse_in = lse_or_part; p.part = reinterpret_cast<float2*>(const_cast<float*>(lse_or_part));
+    p.lse_stride = lse_stride; p.splits = splits; p.scores = scores; p.score_stride = score_stride;
     const int n_tiles = (c.m + kTile - 1) / kTile + (c.L + kTile - 1) / kTile;
     dim3 grid(n_tiles, c.kv_heads);
     colsum_kernel<<<grid, kColThreads, kColSmemBytes, s>>>(mp.Q, mp.CK, mp.SK, p);
