@@ -168,7 +168,7 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     int splits = 1;
     if (c->use_tc) {
         // a1 and pass 1 of a2-I (row log-sum-exp of the instruction queries, possibly split over key ranges): one launch
-        splits = tc_lse_splits(nI, c->Hq, m, L, ((L + 127) / 128) * c->Hq);
+        splits = tc_lse_splits(nI, c->Hq, c->Hkv, m, L, ((L + 127) / 128) * c->Hq);
         LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
         e = tc_attention_lse(q_chunk, cand[0], out, lse_chunk, c->ls, q_instr, cand[ic], u.lse_instr, u.part,
                              CITRUS_MAX_INSTR, splits, c->status, st);

@@ -41,7 +41,7 @@ cudaError_t simt_colsum(bool is_fp32, int D, const QueryRows& q, const Candidate
 // ---- tensor-core (tcgen05 / TMEM / TMA) path: bf16, D = 128 ----------------
 cudaError_t tc_init();   // resolves the driver entry point for tensor-map encoding
 // Number of key splits for pass 1 of a2-I (1 = the pass writes final log-sum-exp values).
-int tc_lse_splits(int n_rows, int q_heads, int m, int L, int n_attn_items);
+int tc_lse_splits(int n_rows, int q_heads, int kv_heads, int m, int L, int n_attn_items);
 constexpr int kTcMaxLseSplits = 8;
 // One launch: a1 (qa over ca -> out, optional row log-sum-exp) and pass 1 of a2-I (qi over ci).  Either part
 // may be empty (rows == 0).  With splits > 1 the pass writes (max, sum) pairs to `part`

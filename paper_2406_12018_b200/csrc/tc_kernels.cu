@@ -196,6 +196,8 @@ struct TcParams {
     int lse_stride;
     float2* part;    // a2 pass 1 with key splits: (max, sum) of every (split, head, row), [splits, q_heads, lse_stride]
     int splits;      // number of key splits (1: lse2 / lse_in hold final log-sum-exp values)
+    int pack;        // a2 pass 1: heads of one KV group sharing a 128-row tile (short instruction texts), 1 = none
+    int pack_rows;   // rows per head in a packed tile (= rows)
     const float* lse_in;   // colsum: log-sum-exp of the scoring rows
     float* scores;   // colsum: [kv_heads, score_stride]
     int score_stride;
@@ -329,7 +331,20 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
 
     if (warp == 8) {
         // ---------------------------------------------------------------- K (and Q) TMA producer (converged warp)
-        load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
+        if (!WITH_PV && p.pack > 1) {
+            // several heads' scoring rows side by side in one tile (mapQ's box is pack_rows rows high)
+            if (elect_one()) {
+                const uint32_t bar = smem_u32(&bars->q_full);
+                mbar_expect_tx(bar, (uint32_t)(p.pack * p.pack_rows * 256));
+                for (int hh = 0; hh < p.pack; ++hh) {
+                    tma_load_3d(sQ + hh * p.pack_rows * 128, &mapQ, bar, 0, h + hh, 0);
+                    tma_load_3d(sQ + kHalfBytes + hh * p.pack_rows * 128, &mapQ, bar, 64, h + hh, 0);
+                }
+            }
+            __syncwarp();
+        } else {
+            load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
+        }
         for (int j = 0; j < nt; ++j) {
             const int s = j % kStagesK, jg = tile_begin + j;
             const bool from_cache = jg < n_cache_tiles;
@@ -567,10 +582,18 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                     }
                 }
             }
-            if (NEED_LSE && wg == 0 && r < p.rows) {
+            // which (head, row) this thread's tile row stands for
+            int oh = h, orow = r;
+            bool row_ok = r < p.rows;
+            if (!WITH_PV && p.pack > 1) {
+                oh = h + row_in_tile / p.pack_rows;
+                orow = row_in_tile % p.pack_rows;
+                row_ok = row_in_tile < p.pack * p.pack_rows;
+            }
+            if (NEED_LSE && wg == 0 && row_ok) {
                 const float l = mine.l * w_mine + other.l * w_other;
-                if (p.splits > 1) p.part[((size_t)split * p.q_heads + h) * p.lse_stride + r] = make_float2(M, l);
-                else if (p.lse2 != nullptr) p.lse2[(size_t)h * p.lse_stride + r] = M + log2f(l);
+                if (p.splits > 1) p.part[((size_t)split * p.q_heads + oh) * p.lse_stride + orow] = make_float2(M, l);
+                else if (p.lse2 != nullptr) p.lse2[(size_t)oh * p.lse_stride + orow] = M + log2f(l);
             }
         }
     }
@@ -602,7 +625,8 @@ attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     } else {
         const int item = id - n_attn;
         const int split = item % pl.splits, rest = item / pl.splits;
-        const int h = rest % pl.q_heads, rt = rest / pl.q_heads;
+        const int head_slots = pl.q_heads / pl.pack;
+        const int h = (rest % head_slots) * pl.pack, rt = rest / head_slots;
         const int tiles = (pl.m + kTile - 1) / kTile + (pl.L + kTile - 1) / kTile;
         const int t0 = (int)((long long)split * tiles / pl.splits), t1 = (int)((long long)(split + 1) * tiles / pl.splits);
         attn_body<false, true>(mapQI, mapCKI, mapCKI, mapSK, mapSK, mapQI, pl, rt, h, t0, t1, split, smem_raw);
@@ -784,10 +808,10 @@ typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void
 EncodeFn g_encode = nullptr;
 
 // Token-major tensor [rows, heads, 128] bf16: coordinates (d, head, row), box 64 x 1 x 128.
-bool map_token_major(CUtensorMap* map, const void* ptr, int rows, int heads) {
+bool map_token_major(CUtensorMap* map, const void* ptr, int rows, int heads, int box_rows = kTile) {
     cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)heads, (cuuint64_t)rows};
     cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)heads * kD * 2};
-    cuuint32_t box[3] = {64, 1, (cuuint32_t)kTile};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
     cuuint32_t es[3] = {1, 1, 1};
     return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -846,13 +870,22 @@ cudaError_t tc_init() {
     return cudaSuccess;
 }
 
-int tc_lse_splits(int n_rows, int q_heads, int m, int L, int n_attn_items) {
+// Heads of one KV group whose scoring rows share a 128-row tile in pass 1 of a2-I (1 = one head per tile).
+static int lse_pack(int n_rows, int q_heads, int kv_heads) {
+    const int G = q_heads / kv_heads;
+    if (n_rows > 64 || n_rows % 8 != 0 || kTile % n_rows != 0) return 1;
+    int pack = kTile / n_rows;
+    while (pack > 1 && (pack > G || G % pack != 0)) pack >>= 1;
+    return pack < 1 ? 1 : pack;
+}
+
+int tc_lse_splits(int n_rows, int q_heads, int kv_heads, int m, int L, int n_attn_items) {
     // The log-sum-exp items share a launch with the attention items.  When those leave SMs idle (fewer items than
     // SMs), split the key range so that there is about one short item per idle SM; otherwise keep whole sweeps,
     // because every extra item pays a CTA prologue.
     const int kSMs = 148;
     const int tiles = (m + kTile - 1) / kTile + (L + kTile - 1) / kTile;
-    const int base_items = ((n_rows + kTile - 1) / kTile) * q_heads;
+    const int base_items = ((n_rows + kTile - 1) / kTile) * q_heads / lse_pack(n_rows, q_heads, kv_heads);
     const int idle = n_attn_items < kSMs ? kSMs - n_attn_items : 0;
     int s = idle / base_items;
     if (s > tiles) s = tiles;
@@ -871,8 +904,10 @@ cudaError_t tc_attention_lse(const QueryRows& qa, const Candidates& ca, void* ou
         if (!build_maps(&ma, qa.Q, qa.rows, qa, ca, true)) return cudaErrorInvalidValue;
         if (!map_token_major(&mapO, out, qa.rows, qa.q_heads)) return cudaErrorInvalidValue;
     }
+    const int pack = has_lse ? lse_pack(qi.rows, qi.q_heads, ci.kv_heads) : 1;
     if (has_lse) {
         if (!build_maps(&mi, qi.Q, qi.rows, qi, ci, false)) return cudaErrorInvalidValue;
+        if (pack > 1 && !map_token_major(&mi.Q, qi.Q, qi.rows, qi.q_heads, qi.rows)) return cudaErrorInvalidValue;
     }
     if (!has_attn) { ma = mi; mapO = mi.Q; }
     if (!has_lse) mi = ma;
@@ -880,8 +915,10 @@ cudaError_t tc_attention_lse(const QueryRows& qa, const Candidates& ca, void* ou
     pa.out = out; pa.lse2 = lse_chunk; pa.lse_stride = lse_chunk_stride; pa.splits = 1;
     TcParams pl = base_params(has_lse ? qi : qa, has_lse ? ci : ca, status);
     pl.lse2 = lse_instr; pl.part = reinterpret_cast<float2*>(part); pl.lse_stride = lse_instr_stride; pl.splits = splits;
+    pl.pack = pack; pl.pack_rows = qi.rows;
+    pa.pack = 1; pa.pack_rows = 0;
     const int n_attn = has_attn ? ((qa.rows + kTile - 1) / kTile) * qa.q_heads : 0;
-    const int n_lse = has_lse ? ((qi.rows + kTile - 1) / kTile) * qi.q_heads * splits : 0;
+    const int n_lse = has_lse ? ((qi.rows + kTile - 1) / kTile) * (qi.q_heads / pack) * splits : 0;
     dim3 grid(n_attn + n_lse);
     // both parts read the chunk's K through the same caller tensor, so one chunk-K map serves them
     if (lse_chunk != nullptr)
