@@ -55,9 +55,14 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         if (tid < 256) hist[tid] = 0u;
         __syncthreads();
         const uint32_t prefix = s_prefix;
-        for (int j = tid; j < n; j += kSelThreads) {
-            uint32_t key = keys[j];
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        for (int j0 = 0; j0 < n; j0 += kSelThreads) {            // warp-uniform trip count
+            const int j = j0 + tid;
+            const uint32_t key = j < n ? keys[j] : 0u;
+            const bool act = j < n && (key & mask) == prefix;
+            const uint32_t bin = (key >> shift) & 255u;
+            // scores of one head crowd into a few exponent bins: one shared-memory atomic per (warp, bin)
+            const uint32_t peers = __match_any_sync(0xffffffffu, act ? bin : 256u);
+            if (act && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
         }
         __syncthreads();
         if (tid < 32) {
@@ -186,6 +191,9 @@ select_compact_kernel(SelectArgs sel, CompactArgs cmp, const uint4* __restrict__
                       int kv_heads, int n, int k, int row_vecs, int kept, int chunk_pos0) {
     extern __shared__ uint32_t keys[];            // [n], used by the selecting CTA only
     const int g = blockIdx.y;
+    // programmatic dependent launch: let the next kernel start its prologue, then wait for the scores
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (blockIdx.x == 0) select_body(sel.job[blockIdx.z], g, kv_heads, n, k, 0, keys);
     // hardware cluster barrier with release/acquire semantics: the index list written above is visible to all
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -229,10 +237,12 @@ cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int 
     cfg.blockDim = dim3(kSelThreads);
     cfg.dynamicSmemBytes = (size_t)n * sizeof(uint32_t);
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = kFusedCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, select_compact_kernel, sa, ca, reinterpret_cast<const uint4*>(chunkK),
                               reinterpret_cast<const uint4*>(chunkV), kv_heads, n, k, row_bytes / 16, kept, chunk_pos0);
 }

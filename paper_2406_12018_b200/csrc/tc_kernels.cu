@@ -15,6 +15,8 @@
 
 #include <cuda.h>
 
+#include <utility>
+
 // Optional cycle stamps of one CTA's roles (build with -DCITRUS_TRACE; compiled out otherwise).
 #ifdef CITRUS_TRACE
 __device__ unsigned long long g_citrus_trace[256];
@@ -324,6 +326,9 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // programmatic dependent launch: everything above overlapped the previous kernel's tail; its results
+    // (the compacted cache) are only touched after this wait
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
     auto tmO = [tmem](int b) { return tmem + 256u + (uint32_t)b * 128u; };
@@ -617,6 +622,7 @@ attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 const __grid_constant__ CUtensorMap mapQI, const __grid_constant__ CUtensorMap mapCKI,
                 const TcParams pa, const TcParams pl, const int n_attn) {
     extern __shared__ uint8_t smem_raw[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int id = blockIdx.x;
     if (id < n_attn) {
         const int n_qt = (pa.rows + kTile - 1) / kTile;
@@ -649,6 +655,7 @@ __global__ void __launch_bounds__(kColThreads, 1)
 colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
               const __grid_constant__ CUtensorMap mapSK, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sK = base;
     const uint32_t sQ = sK + kTileBytes;
@@ -683,6 +690,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // pass 1's log-sum-exp values are final after this
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
 
@@ -844,6 +852,19 @@ bool build_maps(Maps* mp, const void* Qbase, int q_rows_total, const QueryRows& 
     return true;
 }
 
+// Launch with programmatic stream serialisation: the kernel may begin (prologue only) before its predecessor
+// in the stream has finished; it reads the predecessor's results after griddepcontrol.wait.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 TcParams base_params(const QueryRows& q, const Candidates& c, int* status) {
     TcParams p{};
     p.rows = q.rows; p.row0 = 0; p.q_heads = q.q_heads; p.kv_heads = c.kv_heads;
@@ -922,12 +943,10 @@ cudaError_t tc_attention_lse(const QueryRows& qa, const Candidates& ca, void* ou
     dim3 grid(n_attn + n_lse);
     // both parts read the chunk's K through the same caller tensor, so one chunk-K map serves them
     if (lse_chunk != nullptr)
-        attn_lse_kernel<true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(ma.Q, ma.CK, ma.CV, ma.SK, ma.SV, mapO,
-                                                                        mi.Q, mi.CK, pa, pl, n_attn);
-    else
-        attn_lse_kernel<false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(ma.Q, ma.CK, ma.CV, ma.SK, ma.SV, mapO,
-                                                                         mi.Q, mi.CK, pa, pl, n_attn);
-    return cudaGetLastError();
+        return launch_pdl(attn_lse_kernel<true>, grid, kAttnThreads, kAttnSmemBytes, s, ma.Q, ma.CK, ma.CV, ma.SK, ma.SV, mapO,
+                          mi.Q, mi.CK, pa, pl, n_attn);
+    return launch_pdl(attn_lse_kernel<false>, grid, kAttnThreads, kAttnSmemBytes, s, ma.Q, ma.CK, ma.CV, ma.SK, ma.SV, mapO,
+                      mi.Q, mi.CK, pa, pl, n_attn);
 }
 
 cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse_or_part, int lse_stride, int splits,
@@ -939,8 +958,7 @@ cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse_
     p.lse_stride = lse_stride; p.splits = splits; p.scores = scores; p.score_stride = score_stride;
     const int n_tiles = (c.m + kTile - 1) / kTile + (c.L + kTile - 1) / kTile;
     dim3 grid(n_tiles, c.kv_heads);
-    colsum_kernel<<<grid, kColThreads, kColSmemBytes, s>>>(mp.Q, mp.CK, mp.SK, p);
-    return cudaGetLastError();
+    return launch_pdl(colsum_kernel, grid, kColThreads, kColSmemBytes, s, mp.Q, mp.CK, mp.SK, p);
 }
 
 }  // namespace citrus
