@@ -4,6 +4,20 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+// Optional cycle stamps of one CTA's roles (build with -DCITRUS_TRACE; compiled out otherwise).
+// Every translation unit that stamps keeps its own buffer and exports its own reader.
+#ifdef CITRUS_TRACE
+static __device__ unsigned long long g_citrus_trace[256];
+#define CITRUS_TR(i) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 31) == 0) \
+                              g_citrus_trace[(i)] = clock64(); } while (0)
+#define CITRUS_TRACE_EXPORT(suffix) \
+    extern "C" int citrus_trace_read##suffix(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_citrus_trace, sizeof(g_citrus_trace)); } \
+    extern "C" int citrus_trace_clear##suffix() { static unsigned long long z[256]; return (int)cudaMemcpyToSymbol(g_citrus_trace, z, sizeof(z)); }
+#else
+#define CITRUS_TR(i) do { } while (0)
+#define CITRUS_TRACE_EXPORT(suffix)
+#endif
+
 namespace citrus {
 
 // Where the n = m + L candidate states of one call live.  Candidate j < m is row

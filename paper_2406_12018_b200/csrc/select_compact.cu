@@ -135,7 +135,7 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
 }
 
 __global__ void __launch_bounds__(kSelThreads)
-select_topk_kernel(SelectArgs args, int kv_heads, int n, int k, int layerwise) {
+select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int n, int k, int layerwise) {
     extern __shared__ uint32_t keys[];            // [n]
     select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, n, k, layerwise, keys);
 }
@@ -151,21 +151,38 @@ __device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4*
     const uint4* srcV = reinterpret_cast<const uint4*>(job.srcV);
     uint4* dstK = reinterpret_cast<uint4*>(job.dstK);
     uint4* dstV = reinterpret_cast<uint4*>(job.dstV);
-    for (int r = r_begin + sub; r < r_end; r += rows_per_pass) {
-        const int j = idx[r];
-        const uint4 *pk, *pv;
-        if (j < job.m) {
-            size_t off = ((size_t)g * cap + j) * row_vecs + v;
-            pk = srcK + off; pv = srcV + off;
-        } else {
-            size_t off = ((size_t)(j - job.m) * kv_heads + g) * row_vecs + v;
-            pk = chunkK + off; pv = chunkV + off;
+    // four rows per thread in flight: first every index, then every load, then the stores
+    constexpr int kInFlight = 4;
+    for (int rb = r_begin + sub; rb < r_end; rb += kInFlight * rows_per_pass) {
+        int j[kInFlight];
+        uint4 a[kInFlight], b[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const int r = rb + u * rows_per_pass;
+            j[u] = r < r_end ? idx[r] : -1;
         }
-        uint4 a = __ldg(pk), b = __ldg(pv);
-        size_t doff = ((size_t)g * cap + r) * row_vecs + v;
-        dstK[doff] = a;
-        dstV[doff] = b;
-        if (v == 0) job.dstPos[(size_t)g * cap + r] = j < job.m ? job.srcPos[(size_t)g * cap + j] : chunk_pos0 + (j - job.m);
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            if (j[u] < 0) continue;
+            const uint4 *pk, *pv;
+            if (j[u] < job.m) {
+                size_t off = ((size_t)g * cap + j[u]) * row_vecs + v;
+                pk = srcK + off; pv = srcV + off;
+            } else {
+                size_t off = ((size_t)(j[u] - job.m) * kv_heads + g) * row_vecs + v;
+                pk = chunkK + off; pv = chunkV + off;
+            }
+            a[u] = __ldg(pk); b[u] = __ldg(pv);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            if (j[u] < 0) continue;
+            const int r = rb + u * rows_per_pass;
+            size_t doff = ((size_t)g * cap + r) * row_vecs + v;
+            dstK[doff] = a[u];
+            dstV[doff] = b[u];
+            if (v == 0) job.dstPos[(size_t)g * cap + r] = j[u] < job.m ? job.srcPos[(size_t)g * cap + j[u]] : chunk_pos0 + (j[u] - job.m);
+        }
     }
 }
 
@@ -174,7 +191,7 @@ constexpr int kCompactThreads = 256;
 constexpr int kCompactRowsPerCta = 64;
 
 __global__ void __launch_bounds__(kCompactThreads)
-compact_kv_kernel(CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
+compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
                   int kv_heads, int cap, int row_vecs, int kept, int chunk_pos0) {
     const int r0 = blockIdx.x * kCompactRowsPerCta;
     compact_rows(args.job[blockIdx.z], chunkK, chunkV, blockIdx.y, kv_heads, cap, row_vecs,
@@ -187,7 +204,7 @@ compact_kv_kernel(CompactArgs args, const uint4* __restrict__ chunkK, const uint
 constexpr int kFusedCluster = 8;
 
 __global__ void __launch_bounds__(kSelThreads)
-select_compact_kernel(SelectArgs sel, CompactArgs cmp, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
+select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_constant__ CompactArgs cmp, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
                       int kv_heads, int n, int k, int row_vecs, int kept, int chunk_pos0) {
     extern __shared__ uint32_t keys[];            // [n], used by the selecting CTA only
     const int g = blockIdx.y;

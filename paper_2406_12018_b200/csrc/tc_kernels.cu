@@ -17,16 +17,7 @@
 
 #include <utility>
 
-// Optional cycle stamps of one CTA's roles (build with -DCITRUS_TRACE; compiled out otherwise).
-#ifdef CITRUS_TRACE
-__device__ unsigned long long g_citrus_trace[256];
-#define CITRUS_TR(i) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0) \
-                              g_citrus_trace[(i)] = clock64(); } while (0)
-extern "C" int citrus_trace_read(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_citrus_trace, sizeof(g_citrus_trace)); }
-extern "C" int citrus_trace_clear() { static unsigned long long z[256]; return (int)cudaMemcpyToSymbol(g_citrus_trace, z, sizeof(z)); }
-#else
-#define CITRUS_TR(i) do { } while (0)
-#endif
+CITRUS_TRACE_EXPORT()
 
 namespace citrus {
 namespace {
