@@ -32,6 +32,9 @@ sys.path.insert(0, ROOT)
 from paper_2406_12018_b200 import workloads as wl  # noqa: E402
 
 WORKLOAD = "mistral7b_layer"
+# dram__bytes_read.sum + dram__bytes_write.sum of one steady-state attn_lse_kernel launch, from
+# profiles/attn_lse_kernel_mistral7b_layer.md; set to None whenever that kernel changes after the capture.
+ATTN_DRAM_TRAFFIC_BYTES = 10.07e6
 METRIC = "document tokens/s through chunked eviction per layer"
 UNIT = "tokens/s"
 
@@ -339,7 +342,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch every chunk from the host instead of a CUDA graph")
     ap.add_argument("--skip-cpu", action="store_true", help="do not time the oracle (profiling runs)")
-    ap.add_argument("--traffic", type=float, default=None,
+    ap.add_argument("--traffic", type=float, default=ATTN_DRAM_TRAFFIC_BYTES,
                     help="DRAM bytes per attention launch from the committed ncu summary (null if stale)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
