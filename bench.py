@@ -190,7 +190,9 @@ def run_ours(args, rank, world, local_rank):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    w = wl.CONFIGS[WORKLOAD]
+    w = wl.CONFIGS[args.workload]
+    if args.doc_tokens:
+        w = wl.scaled(w, doc_tokens=args.doc_tokens, n_seqs=1, min_tokens=0)
     doc = rank_document(w, rank)
     N = doc.Q.shape[0]
     n_chunks = -(-N // w.chunk_s)
@@ -262,6 +264,8 @@ def run_ours(args, rank, world, local_rank):
     peaks = measured_peaks()
     achieved = total_flops * prof_steps / (attn_ms / 1e3) / 1e12
     kern_total = sum(v[0] for v in prof.values())
+    launches_per_step = sum(v[1] for v in prof.values()) // prof_steps
+    n_caches = 2 if w.mode == "individual" else 1
     elt = 2
     sel_bytes = sum(4.0 * (min(w.budget_k, s) + min(w.chunk_s, N - s)) * w.kv_heads + 4.0 * min(w.budget_k, s + w.chunk_s) * w.kv_heads
                     for s in range(0, N, w.chunk_s))
@@ -275,13 +279,20 @@ def run_ours(args, rank, world, local_rank):
     kernels["attention"]["note"] = "one launch: a1 plus the log-sum-exp pass of a2-I"
     # a3 + a4 run as one cluster launch (recorded under "compact"): algorithmic bytes of both steps
     kernels["compact"]["note"] = "one launch: a3 select + a4 compaction"
-    kernels["compact"]["gbs"] = (sel_bytes + cmp_bytes) * prof_steps / (prof["compact"][0] / 1e3) / 1e9
-    kernels["compact"]["mb_per_launch"] = (sel_bytes + cmp_bytes) / n_chunks / 1e6
+    if "select" in kernels:       # large steps: a3 and a4 are separate launches
+        kernels["compact"]["note"] = "a4 compaction"
+        kernels["select"]["gbs"] = n_caches * sel_bytes * prof_steps / (prof["select"][0] / 1e3) / 1e9
+        kernels["compact"]["gbs"] = n_caches * cmp_bytes * prof_steps / (prof["compact"][0] / 1e3) / 1e9
+        kernels["compact"]["mb_per_launch"] = n_caches * cmp_bytes / n_chunks / 1e6
+    else:
+        kernels["compact"]["gbs"] = n_caches * (sel_bytes + cmp_bytes) * prof_steps / (prof["compact"][0] / 1e3) / 1e9
+        kernels["compact"]["mb_per_launch"] = n_caches * (sel_bytes + cmp_bytes) / n_chunks / 1e6
+    kernels["compact"]["frac_of_hbm_peak"] = kernels["compact"]["gbs"] / peaks["hbm_gbs"]
     roofline = {"bound": "tensor", "kernel": "attn_lse_kernel (a1 flops only; the launch also runs pass 1 of a2-I)", "achieved": achieved,
                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                 "peak_source": f"{peaks['source']} burst bf16 (kernel launches are short and separated)",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
-                "traffic": args.traffic, "timing": f"{prof_steps} of the same steps repeated with per-launch CUDA events on the launch stream",
+                "traffic": args.traffic if (args.workload == WORKLOAD and not args.doc_tokens) else None, "timing": f"{prof_steps} of the same steps repeated with per-launch CUDA events on the launch stream",
                 "hbm_peak_gbs": peaks["hbm_gbs"], "kernels": kernels}
 
     # ---- end to end through the host-buffer ABI call (pinned host memory, copies inside)
@@ -321,12 +332,12 @@ def run_ours(args, rank, world, local_rank):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "q_heads": w.q_heads, "kv_heads": w.kv_heads, "head_dim": w.head_dim,
-                           "budget_k": w.budget_k, "chunk_s": w.chunk_s, "doc_tokens": N, "n_instr": w.n_instr,
+                "config": {"workload": args.workload, "q_heads": w.q_heads, "kv_heads": w.kv_heads, "head_dim": w.head_dim,
+                           "budget_k": w.budget_k, "chunk_s": w.chunk_s, "doc_tokens": N, "lm_window": w.lm_window, "n_instr": w.n_instr,
                            "mode": w.mode, "parallelism": f"{world} independent documents" if world > 1 else "1 GPU",
                            "launch": "cuda_graph" if graph is not None else "stream",
                            "l2": f"inputs larger than L2: {in_bytes / 1e6:.0f} MB of Q/K/V/out per step"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * n_chunks * args.steps,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
                 "roofline": roofline, "cpu_baseline": cpu}
         print(json.dumps(line), flush=True)
     ctx.close()
@@ -340,6 +351,9 @@ def main():
     ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD, choices=[k for k, v in wl.CONFIGS.items() if v.dtype == "bf16"],
+                    help="another named workload (layer 0, one sequence) instead of the headline one")
+    ap.add_argument("--doc-tokens", type=int, default=0, help="truncate / set the document length")
     ap.add_argument("--no-graph", action="store_true", help="launch every chunk from the host instead of a CUDA graph")
     ap.add_argument("--skip-cpu", action="store_true", help="do not time the oracle (profiling runs)")
     ap.add_argument("--traffic", type=float, default=ATTN_DRAM_TRAFFIC_BYTES,

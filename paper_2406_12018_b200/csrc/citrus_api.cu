@@ -213,7 +213,10 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
                             cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, m};
     }
-    if (!c->layerwise) {
+    // Small steps (a few MB to move) are latency-bound: one cluster launch does a3 and a4.  Large steps want every
+    // SM streaming rows, which the clusters (idle while their first CTA selects) cannot give: two launches.
+    const size_t gather_bytes = (size_t)c->n_caches * c->Hkv * kept * c->D * c->elt * 2;
+    if (!c->layerwise && gather_bytes <= ((size_t)8 << 20)) {
         // one cluster launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
         e = select_compact(sj, cj, c->n_caches, Kc, Vc, c->Hkv, n, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
@@ -221,7 +224,7 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     } else {
         {
             LaunchTimer t(c, CITRUS_KERNEL_SELECT, st);
-            e = select_topk(sj, c->n_caches, c->Hkv, n, c->k, 1, st);
+            e = select_topk(sj, c->n_caches, c->Hkv, n, c->k, c->layerwise ? 1 : 0, st);
         }
         if (e != cudaSuccess) return cuda_rc(e);
         {

@@ -137,6 +137,8 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
 __global__ void __launch_bounds__(kSelThreads)
 select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int n, int k, int layerwise) {
     extern __shared__ uint32_t keys[];            // [n]
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the scores are final after this
     select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, n, k, layerwise, keys);
 }
 
@@ -193,6 +195,8 @@ constexpr int kCompactRowsPerCta = 64;
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
                   int kv_heads, int cap, int row_vecs, int kept, int chunk_pos0) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the index lists are final after this
     const int r0 = blockIdx.x * kCompactRowsPerCta;
     compact_rows(args.job[blockIdx.z], chunkK, chunkV, blockIdx.y, kv_heads, cap, row_vecs,
                  r0, min(kept, r0 + kCompactRowsPerCta), chunk_pos0);
@@ -233,9 +237,16 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    dim3 grid(layerwise ? 1 : kv_heads, n_jobs);
-    select_topk_kernel<<<grid, kSelThreads, smem, s>>>(a, kv_heads, n, k, layerwise);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(layerwise ? 1 : kv_heads, n_jobs);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, select_topk_kernel, a, kv_heads, n, k, layerwise);
 }
 
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
@@ -270,11 +281,16 @@ cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, c
     CompactArgs a;
     for (int i = 0; i < n_jobs; ++i) a.job[i] = jobs[i];
     int row_vecs = row_bytes / 16;
-    dim3 grid((kept + kCompactRowsPerCta - 1) / kCompactRowsPerCta, kv_heads, n_jobs);
-    compact_kv_kernel<<<grid, kCompactThreads, 0, s>>>(a, reinterpret_cast<const uint4*>(chunkK),
-                                                       reinterpret_cast<const uint4*>(chunkV),
-                                                       kv_heads, cap, row_vecs, kept, chunk_pos0);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((kept + kCompactRowsPerCta - 1) / kCompactRowsPerCta, kv_heads, n_jobs);
+    cfg.blockDim = dim3(kCompactThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, compact_kv_kernel, a, reinterpret_cast<const uint4*>(chunkK),
+                              reinterpret_cast<const uint4*>(chunkV), kv_heads, cap, row_vecs, kept, chunk_pos0);
 }
 
 }  // namespace citrus
