@@ -114,6 +114,20 @@ int citrus_process_chunk_slot(citrus_handle h, int layer, int seq_slot,
                               const void* Q_instr, int n_instr, void* out, citrus_stream_t stream);
 
 /*
+ * Ragged batch (serving mix): one chunk for each of n_active sequences, packed token-major.  Sequence i uses slot
+ * seq_slot[i]; its chunk rows are [tok_offset[i], tok_offset[i+1]) of Q / K / V / out and its instruction rows are
+ * [instr_offset[i], instr_offset[i+1]) of Q_instr.  seq_slot, tok_offset and instr_offset are HOST arrays
+ * (n_active, n_active + 1 and n_active + 1 ints); the tensors are device pointers as in citrus_process_chunk.
+ * Every sequence's chunk obeys the single-call rules (1..chunk_s tokens, 1..CITRUS_MAX_INSTR instruction rows,
+ * distinct slots).  All arguments are validated before anything is enqueued; sequences are independent (no state
+ * is shared between slots), and their steps are enqueued one after the other on `stream`.
+ * Errors: as citrus_process_chunk; INVALID_ARG for duplicate slots or non-increasing offsets.
+ */
+int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const int* seq_slot, const int* tok_offset,
+                               const void* Q, const void* K, const void* V, const int* instr_offset,
+                               const void* Q_instr, void* out, citrus_stream_t stream);
+
+/*
  * End-to-end variant with HOST buffers (pinned memory recommended): copies the
  * four inputs to device staging owned by the context, runs a1-a4, copies `out`
  * back and waits for that copy.  Same argument rules otherwise.

@@ -26,7 +26,7 @@ KERNEL_NAMES = ["attention", "score_lse", "colsum", "select", "compact"]
 
 EXPORTS = [
     "citrus_create", "citrus_set_batch", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
-    "citrus_process_chunk_host", "citrus_cache_view", "citrus_step_view", "citrus_profile",
+    "citrus_process_chunk_host", "citrus_process_chunk_batch", "citrus_cache_view", "citrus_step_view", "citrus_profile",
     "citrus_profile_read", "citrus_importance_static", "citrus_poll_status",
     "citrus_destroy", "citrus_strerror",
 ]
@@ -55,6 +55,7 @@ def load() -> C.CDLL:
     lib.citrus_reset.argtypes = [vp]
     lib.citrus_process_chunk.argtypes = [vp, i, vp, vp, vp, i, vp, i, vp, vp]
     lib.citrus_process_chunk_slot.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, vp]
+    lib.citrus_process_chunk_batch.argtypes = [vp, i, i, C.POINTER(i), C.POINTER(i), vp, vp, vp, C.POINTER(i), vp, vp, vp]
     lib.citrus_process_chunk_host.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, vp]
     lib.citrus_cache_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(i)]
     lib.citrus_step_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(i), C.POINTER(vp),
@@ -148,6 +149,21 @@ class Citrus:
                                               _stream_ptr(stream))
         if rc != 0:
             raise CitrusError(rc, "citrus_process_chunk")
+        return out
+
+    def process_chunk_batch(self, layer, slots, tok_offset, Q, K, V, instr_offset, Qi, out=None, stream=None):
+        """One chunk for each active sequence, packed token-major (offsets are host lists of len(slots) + 1)."""
+        for t in (Q, K, V, Qi):
+            self._check(t, True)
+        if out is None:
+            out = torch.empty_like(Q)
+        n = len(slots)
+        arr = lambda xs: (C.c_int * len(xs))(*[int(x) for x in xs])
+        rc = load().citrus_process_chunk_batch(self._h, layer, n, arr(slots), arr(tok_offset), Q.data_ptr(), K.data_ptr(),
+                                               V.data_ptr(), arr(instr_offset), Qi.data_ptr(), out.data_ptr(),
+                                               _stream_ptr(stream))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_process_chunk_batch")
         return out
 
     def process_chunk_host(self, layer, Qc, Kc, Vc, Qi, out, slot=0, stream=None):

@@ -331,6 +331,36 @@ int citrus_process_chunk(citrus_handle h, int layer,
     return citrus_process_chunk_slot(h, layer, 0, Q_chunk, K_chunk, V_chunk, n_tokens, Q_instr, n_instr, out, stream);
 }
 
+int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const int* seq_slot, const int* tok_offset,
+                               const void* Q, const void* K, const void* V, const int* instr_offset,
+                               const void* Q_instr, void* out, citrus_stream_t stream) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    if (n_active < 1 || !seq_slot || !tok_offset || !instr_offset || !Q || !K || !V || !Q_instr || !out) return CITRUS_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= h->layers) return CITRUS_ERR_LAYER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(Q_instr) || !aligned16(out)) return CITRUS_ERR_ALIGN;
+    std::set<int> seen;
+    for (int i = 0; i < n_active; ++i) {
+        const int L = tok_offset[i + 1] - tok_offset[i], nI = instr_offset[i + 1] - instr_offset[i];
+        if (seq_slot[i] < 0 || seq_slot[i] >= h->n_slots || !seen.insert(seq_slot[i]).second) return CITRUS_ERR_INVALID_ARG;
+        if (tok_offset[i] < 0 || instr_offset[i] < 0) return CITRUS_ERR_INVALID_ARG;
+        if (L < 1 || L > h->ls || nI < 1 || nI > CITRUS_MAX_INSTR) return CITRUS_ERR_SHAPE;
+        const Unit& u = h->units[(size_t)layer * h->n_slots + seq_slot[i]];
+        if (u.tokens_seen + L > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
+    }
+    const size_t qrow = (size_t)h->Hq * h->D * h->elt, krow = (size_t)h->Hkv * h->D * h->elt;   // multiples of 16 bytes
+    for (int i = 0; i < n_active; ++i) {
+        const char* q = reinterpret_cast<const char*>(Q) + qrow * tok_offset[i];
+        const char* k = reinterpret_cast<const char*>(K) + krow * tok_offset[i];
+        const char* v = reinterpret_cast<const char*>(V) + krow * tok_offset[i];
+        const char* qi = reinterpret_cast<const char*>(Q_instr) + qrow * instr_offset[i];
+        char* o = reinterpret_cast<char*>(out) + qrow * tok_offset[i];
+        int rc = run_step(h, layer, seq_slot[i], q, k, v, tok_offset[i + 1] - tok_offset[i], qi,
+                          instr_offset[i + 1] - instr_offset[i], o, reinterpret_cast<cudaStream_t>(stream));
+        if (rc != CITRUS_OK) return rc;     // only a launch failure can get here; earlier sequences have advanced
+    }
+    return CITRUS_OK;
+}
+
 int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,
                               const void* Qh, const void* Kh, const void* Vh, int n_tokens,
                               const void* Qih, int n_instr, void* out_h, citrus_stream_t stream) {

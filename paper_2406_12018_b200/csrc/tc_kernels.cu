@@ -899,7 +899,9 @@ int tc_lse_splits(int n_rows, int q_heads, int kv_heads, int m, int L, int n_att
     const int tiles = (m + kTile - 1) / kTile + (L + kTile - 1) / kTile;
     const int base_items = ((n_rows + kTile - 1) / kTile) * q_heads / lse_pack(n_rows, q_heads, kv_heads);
     const int idle = n_attn_items < kSMs ? kSMs - n_attn_items : 0;
-    int s = idle / base_items;
+    // several waves of attention items: short log-sum-exp items (about four key tiles each) at the end of the
+    // grid fill the ragged tail of the last wave instead of extending it
+    int s = n_attn_items < kSMs ? idle / base_items : (tiles + 3) / 4;
     if (s > tiles) s = tiles;
     if (s > kMaxLseSplits) s = kMaxLseSplits;
     return s < 1 ? 1 : s;

@@ -129,6 +129,44 @@ def test_config5_long_document_sampled():
     ctx.close()
 
 
+def test_ragged_batch_call_matches_per_sequence_calls_and_rejects_bad_batches():
+    # three sequences of the serving mix advance in lock step through the packed call; finished ones drop out
+    w = wl.scaled(C["serving_mix"], n_seqs=3, budget_k=256, chunk_s=256, n_instr=24, doc_tokens=1024, min_tokens=300)
+    lens = [700, 300, 1024]
+    docs = [wl.make_document(w, seq=s, n_tokens=n) for s, n in enumerate(lens)]
+    a, b = pu.make_pair(w), pu.make_pair(w)
+    step = 0
+    while True:
+        active = [s for s in range(3) if step * w.chunk_s < lens[s]]
+        if not active:
+            break
+        sl = {s: slice(step * w.chunk_s, min(lens[s], (step + 1) * w.chunk_s)) for s in active}
+        Q = torch.cat([docs[s].Q[sl[s]] for s in active]).cuda()
+        K = torch.cat([docs[s].K[sl[s]] for s in active]).cuda()
+        V = torch.cat([docs[s].V[sl[s]] for s in active]).cuda()
+        Qi = torch.cat([docs[s].Q_instr for s in active]).cuda()
+        tok = [0]
+        for s in active:
+            tok.append(tok[-1] + (sl[s].stop - sl[s].start))
+        ins = [w.n_instr * i for i in range(len(active) + 1)]
+        out = a.process_chunk_batch(0, active, tok, Q, K, V, ins, Qi)
+        for i, s in enumerate(active):
+            ref = b.process_chunk(0, docs[s].Q[sl[s]].cuda(), docs[s].K[sl[s]].cuda(), docs[s].V[sl[s]].cuda(),
+                                  docs[s].Q_instr.cuda(), slot=s)
+            torch.cuda.synchronize()
+            assert torch.equal(out[tok[i]:tok[i + 1]], ref)
+            assert torch.equal(a.cache_view(0, 0, s)[2], b.cache_view(0, 0, s)[2])
+            assert torch.equal(a.step_view(0, 0, s)[0], b.step_view(0, 0, s)[0])
+        step += 1
+    with pytest.raises(CitrusError) as e:
+        a.process_chunk_batch(0, [0, 0], [0, 8, 16], Q, K, V, [0, 24, 48], Qi)          # duplicate slot
+    assert e.value.code == -1
+    with pytest.raises(CitrusError) as e:
+        a.process_chunk_batch(0, [0, 1], [0, 300, 310], Q, K, V, [0, 24, 48], Qi)       # chunk longer than chunk_s
+    assert e.value.code == -2
+    a.close(); b.close()
+
+
 def test_host_buffer_variant_matches_device_variant():
     w = wl.scaled(C["mistral7b_layer"], doc_tokens=2048)
     doc = wl.make_document(w)
