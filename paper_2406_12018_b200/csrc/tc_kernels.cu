@@ -317,9 +317,15 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    // programmatic dependent launch: everything above overlapped the previous kernel's tail; its results
-    // (the compacted cache) are only touched after this wait
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Programmatic dependent launch: this kernel may run while its predecessor (the previous chunk's compaction)
+    // still does.  The chunk's own tiles come first in the sweep and need nothing from it, so only two things
+    // wait for the predecessor (griddepcontrol.wait): the first load of a retained-cache tile, and the
+    // log-sum-exp writes of the epilogue (the previous chunk's column-sum kernel may still be reading them).
+    // Sweep order: tile index jg(j) = chunk tiles first, then cache tiles.
+    auto sweep_tile = [&](int j) {
+        const int t = tile_begin + j;
+        return t < n_chunk_tiles ? n_cache_tiles + t : t - n_chunk_tiles;
+    };
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
     auto tmO = [tmem](int b) { return tmem + 256u + (uint32_t)b * 128u; };
@@ -341,20 +347,24 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
         } else {
             load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
         }
+        bool dep_waited = false;
         for (int j = 0; j < nt; ++j) {
-            const int s = j % kStagesK, jg = tile_begin + j;
+            const int s = j % kStagesK, jg = sweep_tile(j);
             const bool from_cache = jg < n_cache_tiles;
             const int row = from_cache ? jg * kTile : (jg - n_cache_tiles) * kTile;
+            if (from_cache && !dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
             if (!mbar_wait_warp(smem_u32(&bars->k_empty[s]), ((j / kStagesK) & 1) ^ 1, p.status)) break;
             load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, g, !from_cache);
         }
     } else if (warp == 10) {
         // ---------------------------------------------------------------- V TMA producer (converged warp)
         if (WITH_PV) {
+            bool dep_waited = false;
             for (int j = 0; j < nt; ++j) {
-                const int s = j % kStagesV, jg = tile_begin + j;
+                const int s = j % kStagesV, jg = sweep_tile(j);
                 const bool from_cache = jg < n_cache_tiles;
                 const int row = from_cache ? jg * kTile : (jg - n_cache_tiles) * kTile;
+                if (from_cache && !dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
                 if (!mbar_wait_warp(smem_u32(&bars->v_empty[s]), ((j / kStagesV) & 1) ^ 1, p.status)) break;
                 load_tile(sV + s * kTileBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
             }
@@ -418,7 +428,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             tc_fence_after();
             // number of visible columns of this tile for this row
             int lim = kTile;
-            const int jg = tile_begin + j;
+            const int jg = sweep_tile(j);
             if (jg < n_cache_tiles) {
                 lim = min(kTile, p.m - jg * kTile);
             } else {
@@ -586,6 +596,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 orow = row_in_tile % p.pack_rows;
                 row_ok = row_in_tile < p.pack * p.pack_rows;
             }
+            if (NEED_LSE && wg == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // see the note on the sweep order
             if (NEED_LSE && wg == 0 && row_ok) {
                 const float l = mine.l * w_mine + other.l * w_other;
                 if (p.splits > 1) p.part[((size_t)split * p.q_heads + oh) * p.lse_stride + orow] = make_float2(M, l);
