@@ -53,6 +53,9 @@ typedef struct CUstream_st* citrus_stream_t;
 #define CITRUS_MODE_INDIVIDUAL  1u        /* LM cache C + instruction cache C^I       (Section 4.2, Eq. 4-5)        */
 #define CITRUS_MODE_FP32        2u        /* tensors are fp32 (default bf16)                                         */
 #define CITRUS_MODE_LAYERWISE   4u        /* one index set per layer from head-summed scores (Section 4.1, last par.) */
+#define CITRUS_MODE_STANDARD    8u        /* standard chunked eviction: one cache scored by the chunk itself (Section 4.1); a call
+                                             that does pass instruction queries is scored by them instead (the final eviction
+                                             "with the instruction text as a new chunk") */
 #define CITRUS_MODE_LM_WINDOW(w) (((unsigned)(w) & 0xFFFFu) << 8)   /* w scoring queries for C; 0 = whole chunk */
 
 #define CITRUS_OK                 0
@@ -96,7 +99,8 @@ int citrus_reset(citrus_handle h);
  *   Q_chunk [n_tokens, q_heads, D], K_chunk / V_chunk [n_tokens, kv_heads, D],
  *   Q_instr [n_instr, q_heads, D] (queries of the instruction text I for this
  *   layer), out [n_tokens, q_heads, D] receives the attention output of a1 in the
- *   element type.  1 <= n_tokens <= chunk_s (a shorter chunk is allowed anywhere,
+ *   element type.  With CITRUS_MODE_STANDARD, n_instr == 0 (Q_instr may then be NULL) selects scoring by the chunk.
+ *   1 <= n_tokens <= chunk_s (a shorter chunk is allowed anywhere,
  *   cf. "except for the final chunk", Section 4.1); 1 <= n_instr <= CITRUS_MAX_INSTR.
  * Chunks of one (layer, slot) must be submitted in document order on one stream.
  * The caller's K_chunk / V_chunk must stay valid until the stream work is done

@@ -32,6 +32,7 @@ import numpy as np
 
 SHARED = "shared"
 INDIVIDUAL = "individual"
+STANDARD = "standard"     # standard chunked eviction (Section 4.1): one cache, scored by the chunk itself
 
 
 # --------------------------------------------------------------------------
@@ -198,14 +199,19 @@ class CitrusOracle:
         Qc = np.asarray(Qc, dtype=np.float64)
         Kc = np.asarray(Kc, dtype=np.float64)
         Vc = np.asarray(Vc, dtype=np.float64)
-        Qi = np.asarray(Qi, dtype=np.float64)
+        Qi = None if Qi is None else np.asarray(Qi, dtype=np.float64)
         L = Qc.shape[0]
         c0 = self.caches[0]
         m = c0.K.shape[1]
         chunk_pos = self.tokens_seen + np.arange(L, dtype=np.int64)
 
         scores: Dict[int, np.ndarray] = {}
-        if self.mode == SHARED:
+        if self.mode == STANDARD and Qi is None:
+            # Eq. 1 with s = the chunk: its last w queries vote on [cache ; chunk]
+            w = L if self.lm_window is None else min(self.lm_window, L)
+            out, s_lm = chunk_attention(Qc, c0.K, c0.V, Kc, Vc, lm_window=w)
+            scores[0] = s_lm
+        elif self.mode in (SHARED, STANDARD):
             out, _ = chunk_attention(Qc, c0.K, c0.V, Kc, Vc, lm_window=0)
             scores[0] = importance_sum(Qi, c0.K, Kc)
         else:

@@ -19,6 +19,7 @@ MODE_SHARED = 0
 MODE_INDIVIDUAL = 1
 MODE_FP32 = 2
 MODE_LAYERWISE = 4
+MODE_STANDARD = 8
 MAX_INSTR = 4096
 MAX_CANDIDATES = 49152
 
@@ -116,7 +117,7 @@ class Citrus:
     def __init__(self, layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, mode="shared", dtype="bf16",
                  lm_window=0, layerwise=False, n_seqs=1):
         lib = load()
-        bits = (MODE_INDIVIDUAL if mode == "individual" else MODE_SHARED)
+        bits = {"individual": MODE_INDIVIDUAL, "standard": MODE_STANDARD}.get(mode, MODE_SHARED)
         bits |= MODE_FP32 if dtype == "fp32" else 0
         bits |= MODE_LAYERWISE if layerwise else 0
         bits |= (int(lm_window) & 0xFFFF) << 8
@@ -140,13 +141,14 @@ class Citrus:
         assert t.dtype == self.torch_dtype and t.is_contiguous() and t.is_cuda == cuda
 
     def process_chunk(self, layer, Qc, Kc, Vc, Qi, out: Optional[torch.Tensor] = None, slot=0, stream=None):
-        for t in (Qc, Kc, Vc, Qi):
+        """Qi = None is only valid in standard mode (the chunk scores its own eviction)."""
+        for t in (Qc, Kc, Vc) + (() if Qi is None else (Qi,)):
             self._check(t, True)
         if out is None:
             out = torch.empty_like(Qc)
         rc = load().citrus_process_chunk_slot(self._h, layer, slot, Qc.data_ptr(), Kc.data_ptr(), Vc.data_ptr(),
-                                              Qc.shape[0], Qi.data_ptr(), Qi.shape[0], out.data_ptr(),
-                                              _stream_ptr(stream))
+                                              Qc.shape[0], None if Qi is None else Qi.data_ptr(),
+                                              0 if Qi is None else Qi.shape[0], out.data_ptr(), _stream_ptr(stream))
         if rc != 0:
             raise CitrusError(rc, "citrus_process_chunk")
         return out

@@ -39,7 +39,7 @@ struct Unit {                       // one (layer, sequence slot)
 struct citrus_ctx {
     int device = 0;
     int layers = 0, Hq = 0, Hkv = 0, D = 0, k = 0, ls = 0;
-    bool individual = false, fp32 = false, layerwise = false, use_tc = false;
+    bool individual = false, standard = false, fp32 = false, layerwise = false, use_tc = false;
     int lm_window = 0;
     int elt = 2;
     int n_caches = 1;
@@ -123,10 +123,12 @@ int cuda_rc(cudaError_t e) {
 int check_process_args(citrus_ctx* h, int layer, int slot, const void* Q, const void* K, const void* V, int L,
                        const void* Qi, int nI, const void* out) {
     if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
-    if (!Q || !K || !V || !Qi || !out) return CITRUS_ERR_INVALID_ARG;
+    // standard chunked eviction: a call without instruction queries (n_instr == 0) is scored by the chunk itself
+    const bool no_instr = h->standard && nI == 0;
+    if (!Q || !K || !V || (!Qi && !no_instr) || !out) return CITRUS_ERR_INVALID_ARG;
     if (layer < 0 || layer >= h->layers) return CITRUS_ERR_LAYER;
     if (slot < 0 || slot >= h->n_slots) return CITRUS_ERR_INVALID_ARG;
-    if (L < 1 || L > h->ls || nI < 1 || nI > CITRUS_MAX_INSTR) return CITRUS_ERR_SHAPE;
+    if (L < 1 || L > h->ls || (nI < 1 && !no_instr) || nI > CITRUS_MAX_INSTR) return CITRUS_ERR_SHAPE;
     return CITRUS_OK;
 }
 
@@ -162,13 +164,16 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     QueryRows q_instr{Qi, nI, c->Hq, 0, 0};
     float* scores[2] = {u.scores, u.scores + (size_t)c->Hkv * c->score_stride};
     const int ic = c->individual ? 1 : 0;     // the cache scored by the instruction text
+    const bool lm_scoring = c->individual || (c->standard && nI == 0);   // cache 0 is scored by the chunk's own queries
+    const bool instr_scoring = nI > 0;
+    if (!instr_scoring) q_instr.rows = 0;
 
     cudaError_t e;
-    float* lse_chunk = c->individual ? u.lse_chunk : nullptr;     // only a2-L reads a1's row log-sum-exp
+    float* lse_chunk = lm_scoring ? u.lse_chunk : nullptr;        // only a2-L reads a1's row log-sum-exp
     int splits = 1;
     if (c->use_tc) {
         // a1 and pass 1 of a2-I (row log-sum-exp of the instruction queries, possibly split over key ranges): one launch
-        splits = tc_lse_splits(nI, c->Hq, c->Hkv, m, L, ((L + 127) / 128) * c->Hq);
+        if (instr_scoring) splits = tc_lse_splits(nI, c->Hq, c->Hkv, m, L, ((L + 127) / 128) * c->Hq);
         LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
         e = tc_attention_lse(q_chunk, cand[0], out, lse_chunk, c->ls, q_instr, cand[ic], u.lse_instr, u.part,
                              CITRUS_MAX_INSTR, splits, c->status, st);
@@ -177,15 +182,15 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
             LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
             e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, lse_chunk, c->ls, st);
         }
-        if (e == cudaSuccess) {
+        if (e == cudaSuccess && instr_scoring) {
             LaunchTimer t(c, CITRUS_KERNEL_SCORE_LSE, st);
             e = simt_attention(c->fp32, c->D, q_instr, cand[ic], nullptr, u.lse_instr, CITRUS_MAX_INSTR, st);
         }
     }
     if (e != cudaSuccess) return cuda_rc(e);
 
-    // a2-L (individual design): votes of the chunk's last w queries on cache 0's candidates
-    if (c->individual) {
+    // a2-L (individual design, standard chunked eviction): votes of the chunk's last w queries on cache 0's candidates
+    if (lm_scoring) {
         int w = c->lm_window > 0 && c->lm_window < L ? c->lm_window : L;
         const char* q0 = reinterpret_cast<const char*>(Qc) + (size_t)(L - w) * c->Hq * c->D * c->elt;
         QueryRows q_lm{q0, w, c->Hq, 1, L - w};
@@ -195,7 +200,7 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         if (e != cudaSuccess) return cuda_rc(e);
     }
     // a2-I pass 2: Eq. 1 column sums of the instruction queries over the instruction-side cache's candidates
-    {
+    if (instr_scoring) {
         LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
         if (c->use_tc) e = tc_colsum(q_instr, cand[ic], splits > 1 ? u.part : u.lse_instr, CITRUS_MAX_INSTR, splits,
                                      scores[ic], c->score_stride, c->status, st);
@@ -250,7 +255,8 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     if (out == nullptr) return CITRUS_ERR_INVALID_ARG;
     *out = nullptr;
     if (layers < 1 || q_heads < 1 || kv_heads < 1 || budget_k < 1 || chunk_s < 1) return CITRUS_ERR_INVALID_ARG;
-    if (mode & ~(0x7u | 0xFFFF00u)) return CITRUS_ERR_INVALID_ARG;
+    if (mode & ~(0xFu | 0xFFFF00u)) return CITRUS_ERR_INVALID_ARG;
+    if ((mode & CITRUS_MODE_STANDARD) && (mode & CITRUS_MODE_INDIVIDUAL)) return CITRUS_ERR_INVALID_ARG;
     if (q_heads % kv_heads != 0) return CITRUS_ERR_SHAPE;
     if (head_dim != 64 && head_dim != 128) return CITRUS_ERR_UNSUPPORTED;
     const bool fp32 = (mode & CITRUS_MODE_FP32) != 0;
@@ -262,6 +268,7 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     if (cudaGetDevice(&c->device) != cudaSuccess) { cudaGetLastError(); delete c; return CITRUS_ERR_CUDA; }
     c->layers = layers; c->Hq = q_heads; c->Hkv = kv_heads; c->D = head_dim; c->k = budget_k; c->ls = chunk_s;
     c->individual = (mode & CITRUS_MODE_INDIVIDUAL) != 0;
+    c->standard = (mode & CITRUS_MODE_STANDARD) != 0;
     c->fp32 = fp32;
     c->layerwise = (mode & CITRUS_MODE_LAYERWISE) != 0;
     c->lm_window = (int)((mode >> 8) & 0xFFFFu);
@@ -379,7 +386,7 @@ int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,
     if ((e = cudaMemcpyAsync(h->stQ, Qh, qrow * n_tokens, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
     if ((e = cudaMemcpyAsync(h->stK, Kh, krow * n_tokens, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
     if ((e = cudaMemcpyAsync(h->stV, Vh, krow * n_tokens, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
-    if ((e = cudaMemcpyAsync(h->stQi, Qih, qrow * n_instr, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
+    if (n_instr > 0 && (e = cudaMemcpyAsync(h->stQi, Qih, qrow * n_instr, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
     rc = run_step(h, layer, seq_slot, h->stQ, h->stK, h->stV, n_tokens, h->stQi, n_instr, h->stOut, st);
     if (rc) return rc;
     if ((e = cudaMemcpyAsync(out_h, h->stOut, qrow * n_tokens, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_rc(e);

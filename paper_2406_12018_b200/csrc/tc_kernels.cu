@@ -738,39 +738,42 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (p.causal && !from_cache) r_first = max(0, key_row0 + key_in_tile - p.t0);
         float acc = 0.f;
         bool ok = true;
+        // Stage the log-sum-exp values of iteration `it2` (thread i brings row r0 + i) into buffer it2 & 3.  It is
+        // called one iteration ahead, so the global load hides behind the current iteration's exponentials.  A
+        // thread that is in iteration `it` has seen the MMA of `it`, which needed everybody's s_free of it-2,
+        // i.e. everybody has finished reading buffer (it+1) & 3 = (it-3) & 3.
+        auto stage_lse = [&](int it2) {
+            const int h2 = g * G + it2 / rb_per_head;
+            const int rr = (rb0 + it2 % rb_per_head) * kTile + key_in_tile;
+            float lse = INFINITY;
+            if (rr < p.rows) {
+                if (p.splits > 1) {                              // merge the key splits of pass 1
+                    float M = -INFINITY, l = 0.f;
+                    for (int sp = 0; sp < p.splits; ++sp)
+                        M = fmaxf(M, __ldg(&p.part[((size_t)sp * p.q_heads + h2) * p.lse_stride + rr]).x);
+                    for (int sp = 0; sp < p.splits; ++sp) {
+                        const float2 ml = __ldg(&p.part[((size_t)sp * p.q_heads + h2) * p.lse_stride + rr]);
+                        l += ml.y * ex2(ml.x - M);
+                    }
+                    lse = M + log2f(l);
+                } else {
+                    lse = __ldg(p.lse_in + (size_t)h2 * p.lse_stride + rr);
+                }
+            }
+            bars->lse[it2 & 3][key_in_tile] = lse;
+            mbar_arrive(smem_u32(&bars->lse_full[it2 & 3]));
+        };
+        if (nb > 0) stage_lse(0);
         for (int it = 0; it < nb; ++it) {
             const int b = it & 1;
-            const int h = g * G + it / rb_per_head;
             const int rb = rb0 + it % rb_per_head;
             const int r0 = rb * kTile;
             const int ncols = min(kTile, p.rows - r0);
-            // stage this block's log-sum-exp values (thread i brings row r0 + i).  A thread can run at most
-            // three iterations ahead of the slowest one (the MMA of it-1 needs everybody's s_free of it-3),
-            // so with four buffers nobody is still reading the one written here.
             const int lb = it & 3;
-            {
-                const int rr = r0 + key_in_tile;
-                float lse = INFINITY;
-                if (rr < p.rows) {
-                    if (p.splits > 1) {                              // merge the key splits of pass 1
-                        float M = -INFINITY, l = 0.f;
-                        for (int sp = 0; sp < p.splits; ++sp)
-                            M = fmaxf(M, __ldg(&p.part[((size_t)sp * p.q_heads + h) * p.lse_stride + rr]).x);
-                        for (int sp = 0; sp < p.splits; ++sp) {
-                            const float2 ml = __ldg(&p.part[((size_t)sp * p.q_heads + h) * p.lse_stride + rr]);
-                            l += ml.y * ex2(ml.x - M);
-                        }
-                        lse = M + log2f(l);
-                    } else {
-                        lse = __ldg(p.lse_in + (size_t)h * p.lse_stride + rr);
-                    }
-                }
-                bars->lse[lb][key_in_tile] = lse;
-                mbar_arrive(smem_u32(&bars->lse_full[lb]));
-            }
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 1) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(160 + 3 * (it & 7));
+            if (it + 1 < nb) stage_lse(it + 1);
             ok = mbar_wait_warp(smem_u32(&bars->lse_full[lb]), (it >> 2) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(161 + 3 * (it & 7));

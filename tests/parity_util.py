@@ -113,14 +113,18 @@ def run_document(w: wl.Workload, ctx: Citrus, layer=0, slot=0, seq=0, n_tokens=N
         if use_oracle and not oracle_synced:
             load_oracle_from_library(orc, ctx, layer, slot, tokens_seen)
             oracle_synced = True
-        out = ctx.process_chunk(layer, Qd[a:b], Kd[a:b], Vd[a:b], Qid, slot=slot)
+        # standard chunked eviction: chunks score their own eviction; the last call passes the instruction
+        # queries (the paper's final eviction with the instruction text)
+        with_instr = w.mode != "standard" or ci == len(bounds) - 1
+        out = ctx.process_chunk(layer, Qd[a:b], Kd[a:b], Vd[a:b], Qid if with_instr else None, slot=slot)
         torch.cuda.synchronize()
         tokens_seen += L
         n_caches = 2 if ctx.individual else 1
         views = [ctx.step_view(layer, cid, slot) for cid in range(n_caches)]
         if use_oracle:
             forced = {cid: views[cid][1].cpu().numpy().astype(np.int64) for cid in range(n_caches)}
-            res = orc.process_chunk(wl.to_f64(doc.Q[a:b]), wl.to_f64(doc.K[a:b]), wl.to_f64(doc.V[a:b]), Qi64, forced)
+            res = orc.process_chunk(wl.to_f64(doc.Q[a:b]), wl.to_f64(doc.K[a:b]), wl.to_f64(doc.V[a:b]),
+                                    Qi64 if with_instr else None, forced)
             n = res.m_before + L
             err = float(np.abs(out.to(torch.float64).cpu().numpy() - res.out).max())
             st["max_out_err"] = max(st["max_out_err"], err)
@@ -129,7 +133,7 @@ def run_document(w: wl.Workload, ctx: Citrus, layer=0, slot=0, seq=0, n_tokens=N
                 S_gpu = views[cid][0].to(torch.float64).cpu().numpy()
                 assert views[cid][2] == res.m_before
                 S_or = res.scores[cid]
-                if ctx.individual and cid == 0:
+                if (ctx.individual and cid == 0) or not with_instr:
                     wrows = L if not w.lm_window else min(w.lm_window, L)
                 else:
                     wrows = w.n_instr

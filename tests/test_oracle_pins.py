@@ -310,6 +310,41 @@ def test_selection_invariant_to_positive_rescaling_and_layerwise():
     assert res.idx[0][0].tolist() == ref and res.idx[0][1].tolist() == ref
 
 
+def test_standard_mode_scores_by_the_chunk_and_by_the_instruction_when_given():
+    rng = np.random.default_rng(17)
+    Hq, Hkv, D, k, ls, w = 4, 2, 4, 6, 5, 3
+    G = Hq // Hkv
+    orc = CitrusOracle(Hq, Hkv, D, k, oracle.STANDARD, lm_window=w)
+    chunks = [(rand(rng, ls, Hq, D), rand(rng, ls, Hkv, D), rand(rng, ls, Hkv, D)) for _ in range(3)]
+    Qi = rand(rng, 2, Hq, D)
+    for c, (Q, K, V) in enumerate(chunks):
+        cache = orc.caches[0]
+        m = cache.K.shape[1]
+        last = c == len(chunks) - 1
+        res = orc.process_chunk(Q, K, V, Qi if last else None)
+        # brute force: votes of the scoring rows on every candidate
+        ref = [[0.0] * (m + ls) for _ in range(Hkv)]
+        for h in range(Hq):
+            g = h // G
+            keys = [list(cache.K[g, j]) for j in range(m)] + [list(K[u, g]) for u in range(ls)]
+            rows = range(Qi.shape[0]) if last else range(ls - w, ls)
+            for t in rows:
+                q = list(Qi[t, h]) if last else list(Q[t, h])
+                visible = [True] * (m + ls) if last else [True] * m + [u <= t for u in range(ls)]
+                p, _ = brute_attention_row(q, keys, keys, visible)
+                for j in range(m + ls):
+                    ref[g][j] += p[j]
+        assert np.allclose(res.scores[0], np.array(ref), rtol=0, atol=1e-12)
+        for g in range(Hkv):
+            want = sorted(sorted(range(m + ls), key=lambda j: (-ref[g][j], j))[:k])
+            got = res.idx[0][g].tolist()
+            # brute-force and numpy sums may differ in the last bit: only compare when the cut is clear
+            srt = sorted(ref[g], reverse=True)
+            if m + ls <= k or srt[k - 1] - srt[k] > 1e-9:
+                assert got == want
+    assert len(orc.caches) == 1 and orc.caches[0].K.shape[1] == k
+
+
 def test_forced_selection_is_adopted():
     rng = np.random.default_rng(16)
     N, Hq, Hkv, D, k = 10, 2, 1, 4, 3

@@ -53,6 +53,31 @@ def test_budget_not_reached_and_window_whole_chunk(dtype):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_standard_chunked_eviction_mode(dtype):
+    # one cache scored by the chunk's own last w queries; the last call is scored by the instruction instead
+    w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=2, head_dim=128, budget_k=200, chunk_s=256, doc_tokens=1100,
+                  n_instr=20, dtype=dtype, mode="standard", lm_window=48, n_planted=4, n_sinks=1)
+    ctx = pu.make_pair(w)
+    doc, st = pu.run_document(w, ctx)
+    _report(f"standard {dtype}", st)
+    # the same document through the individual design: its LM cache sees identical steps until the last call
+    wi = wl.scaled(w, mode="individual")
+    a, b = pu.make_pair(w), pu.make_pair(wi)
+    for s in range(0, 768, 256):
+        sl = slice(s, s + 256)
+        args = (doc.Q[sl].cuda(), doc.K[sl].cuda(), doc.V[sl].cuda())
+        o1 = a.process_chunk(0, *args, None)
+        o2 = b.process_chunk(0, *args, doc.Q_instr.cuda())
+        torch.cuda.synchronize()
+        assert torch.equal(o1, o2)
+        assert torch.equal(a.cache_view(0, 0)[2], b.cache_view(0, 0)[2])
+        assert torch.equal(a.step_view(0, 0)[0], b.step_view(0, 0)[0])
+    with pytest.raises(CitrusError):
+        b.process_chunk(0, *args, None)                      # only the standard mode may omit the instruction
+    ctx.close(); a.close(); b.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_layerwise_granularity(dtype):
     w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=4, head_dim=128, budget_k=96, chunk_s=160, doc_tokens=640,
                   n_instr=12, dtype=dtype, mode="shared", n_planted=4)
