@@ -132,15 +132,18 @@ int check_process_args(citrus_ctx* h, int layer, int slot, const void* Q, const 
     return CITRUS_OK;
 }
 
+thread_local cudaEvent_t t_pending_start = nullptr;      // start event of the launch being prepared, if any
+
 struct LaunchTimer {                 // brackets one kernel launch with events when profiling is on
     citrus_ctx* c; cudaStream_t st; cudaEvent_t a = nullptr, b = nullptr; int id;
     LaunchTimer(citrus_ctx* c_, int id_, cudaStream_t st_) : c(c_), st(st_), id(id_) {
         if (!c->profiling) return;
         if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { a = b = nullptr; cudaGetLastError(); return; }
-        cudaEventRecord(a, st);
+        t_pending_start = a;         // recorded by before_launch(), right in front of the kernel
     }
     ~LaunchTimer() {
         if (a == nullptr) return;
+        if (t_pending_start == a) { cudaEventRecord(a, st); t_pending_start = nullptr; }   // nothing was launched
         cudaEventRecord(b, st);
         c->timed.push_back(citrus_ctx::Timed{id, a, b});
     }
@@ -247,6 +250,13 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
 }
 
 }  // namespace
+
+void citrus::before_launch(cudaStream_t s) {
+    if (t_pending_start != nullptr) {
+        cudaEventRecord(t_pending_start, s);
+        t_pending_start = nullptr;
+    }
+}
 
 extern "C" {
 

@@ -34,6 +34,10 @@ struct Candidates {
     int kv_heads;
 };
 
+// Called by every launcher immediately before its kernel launch: when per-launch timing is on, this is where the
+// start event is recorded, so that host-side preparation (tensor-map encoding) is not counted as kernel time.
+void before_launch(cudaStream_t s);
+
 // A block of scoring / attending query rows, token-major [rows, q_heads, D].
 struct QueryRows {
     const void* Q;

@@ -246,6 +246,7 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
+    before_launch(s);
     return cudaLaunchKernelEx(&cfg, select_topk_kernel, a, kv_heads, n, k, layerwise);
 }
 
@@ -271,6 +272,7 @@ cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int 
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
+    before_launch(s);
     return cudaLaunchKernelEx(&cfg, select_compact_kernel, sa, ca, reinterpret_cast<const uint4*>(chunkK),
                               reinterpret_cast<const uint4*>(chunkV), kv_heads, n, k, row_bytes / 16, kept, chunk_pos0);
 }
@@ -289,6 +291,7 @@ cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, c
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
+    before_launch(s);
     return cudaLaunchKernelEx(&cfg, compact_kv_kernel, a, reinterpret_cast<const uint4*>(chunkK),
                               reinterpret_cast<const uint4*>(chunkV), kv_heads, cap, row_vecs, kept, chunk_pos0);
 }

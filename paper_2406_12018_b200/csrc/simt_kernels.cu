@@ -173,6 +173,7 @@ simt_colsum_kernel(QueryRows q, Candidates c, const float* __restrict__ lse2, in
 template <typename T, int D>
 cudaError_t launch_attention(const QueryRows& q, const Candidates& c, void* out, float* lse2, int lse_stride, cudaStream_t s) {
     dim3 grid((q.rows + kRowsPerCta - 1) / kRowsPerCta, q.q_heads);
+    before_launch(s);
     simt_attention_kernel<T, D><<<grid, kRowsPerCta * 32, 0, s>>>(q, c, reinterpret_cast<T*>(out), lse2, lse_stride);
     return cudaGetLastError();
 }
@@ -181,6 +182,7 @@ cudaError_t launch_colsum(const QueryRows& q, const Candidates& c, const float* 
                           float* scores, int score_stride, cudaStream_t s) {
     int n = c.m + c.L;
     dim3 grid((n + kColsumKeys - 1) / kColsumKeys, c.kv_heads);
+    before_launch(s);
     simt_colsum_kernel<T, D><<<grid, kColsumKeys, 0, s>>>(q, c, lse2, lse_stride, scores, score_stride);
     return cudaGetLastError();
 }

@@ -626,6 +626,10 @@ attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int id = blockIdx.x;
+#ifdef CITRUS_TRACE
+    unsigned long long t_start = 0;
+    if (threadIdx.x == 0) { t_start = global_ns(); atomicMin(&g_citrus_trace[240], t_start); }
+#endif
     if (id < n_attn) {
         const int n_qt = (pa.rows + kTile - 1) / kTile;
         const int qt = n_qt - 1 - id / pa.q_heads, h = id % pa.q_heads;      // later query tiles see more keys
@@ -639,6 +643,13 @@ attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         const int t0 = (int)((long long)split * tiles / pl.splits), t1 = (int)((long long)(split + 1) * tiles / pl.splits);
         attn_body<false, true>(mapQI, mapCKI, mapCKI, mapSK, mapSK, mapQI, pl, rt, h, t0, t1, split, smem_raw);
     }
+#ifdef CITRUS_TRACE
+    if (threadIdx.x == 0) {
+        const unsigned long long t_end = global_ns();
+        atomicMax(&g_citrus_trace[241], t_end);
+        atomicMax(&g_citrus_trace[id < n_attn ? 242 : 243], t_end - t_start);   // longest attention / log-sum-exp item
+    }
+#endif
 }
 
 // ------------------------------------------------------------------ column sums (a2 pass 2)
@@ -867,6 +878,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
+    before_launch(s);
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
