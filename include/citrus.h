@@ -56,6 +56,8 @@ typedef struct CUstream_st* citrus_stream_t;
 #define CITRUS_MODE_STANDARD    8u        /* standard chunked eviction: one cache scored by the chunk itself (Section 4.1); a call
                                              that does pass instruction queries is scored by them instead (the final eviction
                                              "with the instruction text as a new chunk") */
+#define CITRUS_MODE_START_SIZE(n) (((unsigned)(n) & 0xFu) << 24)   /* always keep the first n tokens (appendix on
+                                             initial tokens; the paper's variant uses 4, its main setting 0); n <= budget_k */
 #define CITRUS_MODE_LM_WINDOW(w) (((unsigned)(w) & 0xFFFFu) << 8)   /* w scoring queries for C; 0 = whole chunk */
 
 #define CITRUS_OK                 0

@@ -182,12 +182,13 @@ class CitrusOracle:
     """
 
     def __init__(self, q_heads, kv_heads, head_dim, budget_k, mode=SHARED,
-                 lm_window: Optional[int] = None, layerwise: bool = False):
+                 lm_window: Optional[int] = None, layerwise: bool = False, start_size: int = 0):
         assert q_heads % kv_heads == 0
         self.Hq, self.Hkv, self.D, self.k = q_heads, kv_heads, head_dim, budget_k
         self.mode = mode
         self.lm_window = lm_window          # None -> every chunk query votes (Eq. 1)
         self.layerwise = layerwise
+        self.start_size = start_size        # initial tokens that are always preserved (appendix on initial tokens)
         self.tokens_seen = 0
         n_caches = 2 if mode == INDIVIDUAL else 1
         self.caches = [CacheState(np.zeros((kv_heads, 0, head_dim)),
@@ -226,6 +227,12 @@ class CitrusOracle:
                 # one score vector for the whole layer (paper's stated granularity):
                 # heads are aggregated before the top-k.
                 S = np.broadcast_to(S.sum(axis=0, keepdims=True), S.shape)
+            if self.start_size > 0:
+                # the first start_size tokens of the document are never evicted: give them an unbeatable score
+                S = S.copy()
+                for g in range(self.Hkv):
+                    cand_pos = np.concatenate([self.caches[cid].pos[g], chunk_pos])
+                    S[g][cand_pos < self.start_size] = np.inf
             own = np.stack([select_topk(S[g], self.k) for g in range(self.Hkv)])
             res.idx[cid] = own
             res.gap[cid] = [kth_gap(S[g], self.k) for g in range(self.Hkv)]

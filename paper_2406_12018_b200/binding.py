@@ -115,12 +115,13 @@ class Citrus:
     """One eviction context (all layers and sequence slots of one geometry)."""
 
     def __init__(self, layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, mode="shared", dtype="bf16",
-                 lm_window=0, layerwise=False, n_seqs=1):
+                 lm_window=0, layerwise=False, n_seqs=1, start_size=0):
         lib = load()
         bits = {"individual": MODE_INDIVIDUAL, "standard": MODE_STANDARD}.get(mode, MODE_SHARED)
         bits |= MODE_FP32 if dtype == "fp32" else 0
         bits |= MODE_LAYERWISE if layerwise else 0
         bits |= (int(lm_window) & 0xFFFF) << 8
+        bits |= (int(start_size) & 0xF) << 24
         self._h = C.c_void_p()
         rc = lib.citrus_create(C.byref(self._h), layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, bits)
         if rc != 0:

@@ -41,6 +41,7 @@ struct citrus_ctx {
     int layers = 0, Hq = 0, Hkv = 0, D = 0, k = 0, ls = 0;
     bool individual = false, standard = false, fp32 = false, layerwise = false, use_tc = false;
     int lm_window = 0;
+    int start_size = 0;             // initial tokens that are never evicted
     int elt = 2;
     int n_caches = 1;
     int n_slots = 1;
@@ -217,7 +218,7 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     for (int ci = 0; ci < c->n_caches; ++ci) {
         CacheBufs& cb = u.cache[ci];
         int* idx = u.idx + (size_t)ci * c->Hkv * c->k;
-        sj[ci] = SelectJob{scores[ci], idx, c->score_stride};
+        sj[ci] = SelectJob{scores[ci], idx, c->score_stride, cb.pos[cb.cur], c->k, m, (int)u.tokens_seen, c->start_size};
         cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
                             cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, m};
     }
@@ -265,13 +266,14 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     if (out == nullptr) return CITRUS_ERR_INVALID_ARG;
     *out = nullptr;
     if (layers < 1 || q_heads < 1 || kv_heads < 1 || budget_k < 1 || chunk_s < 1) return CITRUS_ERR_INVALID_ARG;
-    if (mode & ~(0xFu | 0xFFFF00u)) return CITRUS_ERR_INVALID_ARG;
+    if (mode & ~(0xFu | 0xFFFF00u | 0xF000000u)) return CITRUS_ERR_INVALID_ARG;
     if ((mode & CITRUS_MODE_STANDARD) && (mode & CITRUS_MODE_INDIVIDUAL)) return CITRUS_ERR_INVALID_ARG;
     if (q_heads % kv_heads != 0) return CITRUS_ERR_SHAPE;
     if (head_dim != 64 && head_dim != 128) return CITRUS_ERR_UNSUPPORTED;
     const bool fp32 = (mode & CITRUS_MODE_FP32) != 0;
     if (!fp32 && head_dim != 128) return CITRUS_ERR_UNSUPPORTED;
     if ((long long)budget_k + chunk_s > CITRUS_MAX_CANDIDATES) return CITRUS_ERR_UNSUPPORTED;
+    if ((int)((mode >> 24) & 0xFu) > budget_k) return CITRUS_ERR_SHAPE;
 
     citrus_ctx* c = new (std::nothrow) citrus_ctx();
     if (c == nullptr) return CITRUS_ERR_NOMEM;
@@ -282,6 +284,7 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     c->fp32 = fp32;
     c->layerwise = (mode & CITRUS_MODE_LAYERWISE) != 0;
     c->lm_window = (int)((mode >> 8) & 0xFFFFu);
+    c->start_size = (int)((mode >> 24) & 0xFu);
     c->elt = fp32 ? 4 : 2;
     c->n_caches = c->individual ? 2 : 1;
     c->score_stride = (budget_k + chunk_s + 3) & ~3;

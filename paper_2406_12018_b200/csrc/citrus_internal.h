@@ -76,6 +76,9 @@ struct SelectJob {            // one per cache handled by the launch
     const float* scores;      // [kv_heads, score_stride]
     int* idx;                 // [kv_heads, budget_k]
     int score_stride;
+    // forced keeps ("start size"): candidates whose original position is below `start` are always selected
+    const int* pos;           // positions of the old cache rows [kv_heads, pos_stride]
+    int pos_stride, m, chunk_pos0, start;
 };
 // n candidates, keep min(k, n); layerwise: sum scores over heads first and give every head the same set.
 cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, int k, int layerwise, cudaStream_t s);

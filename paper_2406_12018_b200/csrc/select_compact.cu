@@ -45,7 +45,13 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         } else {
             v = job.scores[(size_t)g * job.score_stride + j];
         }
-        keys[j] = order_key(v);
+        uint32_t key = order_key(v);
+        if (job.start > 0) {
+            // original position of candidate j (layer-wise mode: all heads hold the same positions)
+            const int pos = j < job.m ? job.pos[(size_t)(layerwise ? 0 : g) * job.pos_stride + j] : job.chunk_pos0 + (j - job.m);
+            if (pos < job.start) key = 0xffffffffu;           // beats every score; ties among them keep index order
+        }
+        keys[j] = key;
     }
     if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; }
     __syncthreads();

@@ -46,6 +46,7 @@ class Workload:
     heavy_tail: bool = False
     n_seqs: int = 1
     min_tokens: int = 0        # ragged: lengths ~ U{min_tokens..doc_tokens}
+    start_size: int = 0        # initial tokens that are never evicted (paper's appendix variant: 4)
 
     @property
     def torch_dtype(self):

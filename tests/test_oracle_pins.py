@@ -345,6 +345,25 @@ def test_standard_mode_scores_by_the_chunk_and_by_the_instruction_when_given():
     assert len(orc.caches) == 1 and orc.caches[0].K.shape[1] == k
 
 
+def test_start_size_keeps_initial_tokens_and_fills_the_rest_by_score():
+    rng = np.random.default_rng(18)
+    N, Hq, Hkv, D, k, ls, s0 = 60, 2, 1, 4, 10, 20, 4
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, 3, Hq, D)
+    K[:s0] *= 0.01                                        # make the initial tokens unattractive on purpose
+    orc = CitrusOracle(Hq, Hkv, D, k, SHARED, start_size=s0)
+    for c in range(0, N, ls):
+        before = orc.caches[0].pos[0].tolist()
+        res = orc.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        kept = orc.caches[0].pos[0].tolist()
+        assert kept[:s0] == [0, 1, 2, 3]
+        # the other k - s0 places go to the best-scoring remaining candidates (plain definition, pure Python)
+        cand_pos = before + list(range(c, c + ls))
+        sc = res.scores[0][0]
+        rest = [j for j in range(len(cand_pos)) if cand_pos[j] >= s0]
+        best = sorted(sorted(rest, key=lambda j: (-sc[j], j))[:k - s0])
+        assert kept[s0:] == [cand_pos[j] for j in best]
+
+
 def test_forced_selection_is_adopted():
     rng = np.random.default_rng(16)
     N, Hq, Hkv, D, k = 10, 2, 1, 4, 3

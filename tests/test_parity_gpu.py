@@ -77,6 +77,21 @@ def test_standard_chunked_eviction_mode(dtype):
     ctx.close(); a.close(); b.close()
 
 
+@pytest.mark.parametrize("mode,layerwise", [("shared", False), ("individual", False), ("shared", True)])
+def test_start_size_forced_keeps(mode, layerwise):
+    # the first four tokens are never evicted, however little attention they receive
+    w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=2, head_dim=128, budget_k=100, chunk_s=160, doc_tokens=900,
+                  n_instr=12, dtype="bf16", mode=mode, lm_window=16, n_planted=4, start_size=4)
+    ctx = pu.make_pair(w, layerwise=layerwise)
+    _, st = pu.run_document(w, ctx, layerwise=layerwise)
+    for cid in range(2 if mode == "individual" else 1):
+        P = ctx.cache_view(0, cid)[2]
+        assert P[:, :4].cpu().tolist() == [[0, 1, 2, 3]] * w.kv_heads
+    ctx.close()
+    with pytest.raises(CitrusError):
+        Citrus(1, 8, 2, 128, 3, 16, start_size=4)           # more forced keeps than the budget
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_layerwise_granularity(dtype):
     w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=4, head_dim=128, budget_k=96, chunk_s=160, doc_tokens=640,
