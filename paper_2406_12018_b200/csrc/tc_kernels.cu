@@ -149,6 +149,14 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
           "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -156,6 +164,30 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// Two fp32 values in one 64-bit register pair for the packed fp32 instructions.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -240,11 +272,16 @@ __device__ __forceinline__ void issue_pv(uint32_t tmem_o, uint32_t tmem_p, uint3
     __syncwarp();
 }
 
-constexpr int kStagesK = 3;             // K ring
+constexpr int kStagesK = 2;             // K ring
 constexpr int kStagesV = 2;             // V ring
-constexpr int kAttnThreads = 352;       // 2 softmax warpgroups (8 warps), K-TMA warp, MMA warp, V-TMA warp
+constexpr int kVStageBytes = kTileBytes + kHalfBytes;   // a V tile and, right behind it, a [128 keys][64] block of ones
+constexpr int kAttnThreads = 352;       // 8 softmax warps, K-TMA warp, MMA warp, V-TMA warp
 constexpr int kColThreads = 192;        // 4 column-sum warps, 1 TMA warp, 1 MMA warp
 constexpr int kTmemCols = 512;
+constexpr uint32_t kTmemO = 256;        // O accumulator: 128 output columns + 16 columns that all hold the row sum of P
+constexpr uint32_t kTmemL = kTmemO + 128;
+constexpr uint32_t kTmemP = 400;        // P (bf16 pairs), 64 columns
+constexpr int kOCols = 144;
 constexpr int kMaxLseSplits = 8;
 constexpr float kRescaleTau = 8.f;      // rescale O only when the row max grows by more than 2^8
 
@@ -256,23 +293,29 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
 }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
-struct RowState { float m, l, lo; };    // exponent reference, fp32 sum, sum of bf16-rounded probabilities
-
 struct AttnSmem {
     uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
-    uint64_t s_full[2], p_full[2], o_done[2], xch, out_ready[2], drain;
+    uint64_t s_full[2], s_free[2], p_full, o_done[2], xch, out_ready[2], drain;
     uint32_t tmem_base;
-    RowState rows[2][kTile];            // final per-row state of each warpgroup, exchanged once at the end
+    float lsum[2][kTile];               // fp32 row sums of the two column halves, exchanged once at the end
 };
-constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + kStagesK + kStagesV) + 4096;
+constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + kStagesK) + kVStageBytes * kStagesV + 4096;
 
 // grid: (ceil(rows / 128), q_heads).  One CTA = 128 query rows of one head.
 // WITH_PV: accumulate O = P.V and write `out`; NEED_LSE: keep the fp32 row sum and write the row log-sum-exp.
 //
-// Key tiles alternate between two softmax warpgroups: warpgroup b takes tiles b, b+2, ... with its own
-// exponent reference, its own S/P buffer S[b] and its own accumulator O[b], so the two never exchange
-// anything inside the loop and each scheduler always has a second warp to run.  The two partial results
-// are merged once, in the epilogue:  out = (w0 O[0] + w1 O[1]) / (w0 l0 + w1 l1),  w_b = 2^(m_b - max m).
+// Tensor memory: S[0], S[1] (128 fp32 columns each, Q.K^T of alternating key tiles), O (128 + 16 columns),
+// P (64 columns of bf16 pairs).  S is double-buffered and P has a place of its own, so Q.K^T of tile j+2 is issued
+// as soon as the softmax warps have read S of tile j into registers; the tensor pipe never waits for the
+// exponentials of the tile it is about to overwrite, only P.V of tile j waits for P of tile j.
+//
+// Softmax: eight warps; warps w and w+4 share rows 32 (w & 3) .. +31, thread (w, lane) owns columns
+// 64 (w >> 2) .. +63 of its row.  Both threads of a row read all 128 columns once to take the same row maximum
+// (so they agree on the exponent reference and on every rescale without exchanging anything) and keep only their
+// own half for the exponentials.  The row sum of the bf16-rounded probabilities - the normaliser that makes
+// out = sum(p~ v) / sum(p~) a convex combination of V rows - comes from the tensor core itself: the V operand of
+// P.V is 144 columns wide, the last 16 read from a block of ones, so columns 128..143 of O accumulate sum(p~)
+// in the same fp32 arithmetic as the output columns, and are rescaled with them.
 template <bool WITH_PV, bool NEED_LSE>
 __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtensorMap& mapCK, const CUtensorMap& mapCV,
                                           const CUtensorMap& mapSK, const CUtensorMap& mapSV, const CUtensorMap& mapO,
@@ -283,7 +326,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
     const uint32_t sK = sQ + kTileBytes;
     const uint32_t sV = sK + kStagesK * kTileBytes;
     uint8_t* const gQ = smem_raw + (sQ - smem_u32(smem_raw));         // generic pointer to the Q tile / output staging
-    AttnSmem* bars = reinterpret_cast<AttnSmem*>(smem_raw + (sV + kStagesV * kTileBytes - smem_u32(smem_raw)));
+    AttnSmem* bars = reinterpret_cast<AttnSmem*>(smem_raw + (sV + kStagesV * kVStageBytes - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = h / (p.q_heads / p.kv_heads);
@@ -305,14 +348,23 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
         for (int s = 0; s < kStagesK; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
         for (int s = 0; s < kStagesV; ++s) { mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1); }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->p_full[b]), 128);
+            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 256);
             mbar_init(smem_u32(&bars->o_done[b]), 1); mbar_init(smem_u32(&bars->out_ready[b]), 128);
         }
+        mbar_init(smem_u32(&bars->p_full), 256);
         mbar_init(smem_u32(&bars->xch), 256);
         mbar_init(smem_u32(&bars->drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    if (WITH_PV) {
+        // the blocks of ones behind the V stages (bf16 1.0 everywhere, so the swizzle does not matter)
+        constexpr int kVec = kHalfBytes / 16;
+        for (int i = threadIdx.x; i < kStagesV * kVec; i += kAttnThreads) {
+            uint8_t* dst = smem_raw + (sV + (i / kVec) * kVStageBytes + kTileBytes - smem_u32(smem_raw)) + (i % kVec) * 16;
+            *reinterpret_cast<uint4*>(dst) = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     if (warp == 9) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
     tc_fence_before();
     __syncthreads();
@@ -328,7 +380,8 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
     };
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
-    auto tmO = [tmem](int b) { return tmem + 256u + (uint32_t)b * 128u; };
+    // completion of P.V of tile j: phase (j >> 1) of o_done[j & 1]
+    auto pv_done = [&](int j) { return mbar_wait_warp(smem_u32(&bars->o_done[j & 1]), (j >> 1) & 1, p.status); };
     if (WITH_PV && warp == 0) CITRUS_TR(1);
 
     if (warp == 8) {
@@ -366,13 +419,13 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 const int row = from_cache ? jg * kTile : (jg - n_cache_tiles) * kTile;
                 if (from_cache && !dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
                 if (!mbar_wait_warp(smem_u32(&bars->v_empty[s]), ((j / kStagesV) & 1) ^ 1, p.status)) break;
-                load_tile(sV + s * kTileBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
+                load_tile(sV + s * kVStageBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
             }
         }
     } else if (warp == 9) {
         // ---------------------------------------------------------------- MMA issuer (converged warp)
         constexpr uint32_t idesc_qk = make_idesc(128, 0);
-        constexpr uint32_t idesc_pv = make_idesc(128, 1);
+        constexpr uint32_t idesc_pv = make_idesc(kOCols, 1);
         bool ok = mbar_wait_warp(smem_u32(&bars->q_full), 0, p.status);
         if (WITH_PV) CITRUS_TR(2);
         auto k_ready = [&](int j) { return mbar_wait_warp(smem_u32(&bars->k_full[j % kStagesK]), (j / kStagesK) & 1, p.status); };
@@ -385,46 +438,48 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             if (ok) { tc_fence_after(); qk(j); }
         }
         for (int j = 0; j < nt && ok; ++j) {
-            // operands of the next two MMA groups are checked while the softmax of tile j is still running,
-            // so only the p_full wait sits between its arrival and the tensor pipe
-            if (WITH_PV) {
-                ok = mbar_wait_warp(smem_u32(&bars->v_full[j % kStagesV]), (j / kStagesV) & 1, p.status);
+            if (j + 2 < nt) {
+                // S[j & 1] is free as soon as every softmax thread holds tile j in registers
+                ok = k_ready(j + 2) && mbar_wait_warp(smem_u32(&bars->s_free[j & 1]), (j >> 1) & 1, p.status);
                 if (!ok) break;
+                tc_fence_after();
+                qk(j + 2);
+                if (WITH_PV && j + 2 < 12) CITRUS_TR(10 + j + 2);
             }
-            if (j + 2 < nt) { ok = k_ready(j + 2); if (!ok) break; }
-            // warpgroup j&1 has consumed S_j (and, with PV, written P_j over it)
-            ok = mbar_wait_warp(smem_u32(&bars->p_full[j & 1]), (j >> 1) & 1, p.status);
-            if (!ok) break;
-            tc_fence_after();
             if (WITH_PV) {
                 const int s = j % kStagesV;
-                CITRUS_TR(90 + j);
-                issue_pv(tmO(j & 1), tmS(j & 1), sV + s * kTileBytes, idesc_pv, j < 2,
+                ok = mbar_wait_warp(smem_u32(&bars->v_full[s]), (j / kStagesV) & 1, p.status) &&
+                     mbar_wait_warp(smem_u32(&bars->p_full), j & 1, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                if (j < 10) CITRUS_TR(90 + j);
+                issue_pv(tmem + kTmemO, tmem + kTmemP, sV + s * kVStageBytes, idesc_pv, j == 0,
                          smem_u32(&bars->v_empty[s]), smem_u32(&bars->o_done[j & 1]));
-                CITRUS_TR(30 + j);
+                if (j < 10) CITRUS_TR(30 + j);
             }
-            if (j + 2 < nt) { qk(j + 2); if (WITH_PV) CITRUS_TR(10 + j + 2); }
         }
         // all tensor-core work retired before tensor memory is released
         if (elect_one()) mma_commit(smem_u32(&bars->drain));
         __syncwarp();
         mbar_wait_warp(smem_u32(&bars->drain), 0, p.status);
     } else {
-        // ---------------------------------------------------------------- softmax warpgroups (warps 0-7)
-        const int wg = warp >> 2;                                    // takes key tiles wg, wg+2, ...
+        // ---------------------------------------------------------------- softmax warps 0-7
+        const int half = warp >> 2;                                  // which 64 columns of the row this thread keeps
         const int row_in_tile = (warp & 3) * 32 + lane;
         const int r = q_row0 + row_in_tile;                          // row inside the block
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t o_addr = tmem + kTmemO + lane_base;
+        const uint32_t p_addr = tmem + kTmemP + lane_base + (uint32_t)half * 32u;
         const float scale2 = kLog2e * rsqrtf((float)kD);
-        float m_ref = -INFINITY, l_run = 0.f, l_out = 0.f;
+        const uint64_t scale2x2 = pack_f32x2(scale2, scale2);
+        float m_ref = -INFINITY, l_run = 0.f;
         bool ok = true;
-        int i_last = -1;                                             // local index of this warpgroup's last tile
-        for (int j = wg; j < nt; j += 2) {
-            const int i = j >> 1;
-            i_last = i;
-            ok = mbar_wait_warp(smem_u32(&bars->s_full[wg]), i & 1, p.status);
+#pragma unroll 1
+        for (int j = 0; j < nt; ++j) {
+            const int b = j & 1;
+            ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (j >> 1) & 1, p.status);
             if (!ok) break;
-            if (WITH_PV && warp == 0) CITRUS_TR(50 + 5 * i);
+            if (WITH_PV && warp == 0 && j < 10) CITRUS_TR(50 + 4 * j);
             tc_fence_after();
             // number of visible columns of this tile for this row
             int lim = kTile;
@@ -436,138 +491,126 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 lim = min(kTile, p.L - u0);
                 if (p.causal) lim = min(lim, p.t0 + r - u0 + 1);
             }
-            const uint32_t s_addr = tmS(wg) + lane_base;
-            // ---- sweep 1: row maximum over all 128 columns (one round trip to tensor memory)
-            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            {
-                uint32_t v[128];
+            const uint32_t s_addr = tmS(b) + lane_base;
+            uint32_t own[64], oth[64];
+            tmem_ld32(s_addr + (half ^ 1) * 64, oth);
+            tmem_ld32(s_addr + (half ^ 1) * 64 + 32, oth + 32);
+            tmem_ld32(s_addr + half * 64, own);
+            tmem_ld32(s_addr + half * 64 + 32, own + 32);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->s_free[b]));
+            if (lim < kTile) {
+                const int lim_own = lim - half * 64, lim_oth = lim - (half ^ 1) * 64;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v + c * 32);
-                tmem_wait_ld();
-                if (lim < kTile) {
-#pragma unroll
-                    for (int q = 0; q < 128; ++q)
-                        if (q >= lim) v[q] = 0xff800000u;            // -inf
+                for (int q = 0; q < 64; ++q) {
+                    if (q >= lim_own) own[q] = 0xff800000u;          // -inf
+                    if (q >= lim_oth) oth[q] = 0xff800000u;
                 }
+            }
+            // ---- row maximum over all 128 columns
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int q = 0; q < 128; ++q) mx4[q & 3] = fmaxf(mx4[q & 3], __uint_as_float(v[q]));
+            for (int q = 0; q < 64; q += 2) {
+                mx4[(q >> 1) & 1] = max3(mx4[(q >> 1) & 1], __uint_as_float(oth[q]), __uint_as_float(oth[q + 1]));
+                mx4[2 + ((q >> 1) & 1)] = max3(mx4[2 + ((q >> 1) & 1)], __uint_as_float(own[q]), __uint_as_float(own[q + 1]));
             }
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             const float m_new = fmaxf(m_ref, mx * scale2);
-            if (WITH_PV && warp == 0) CITRUS_TR(51 + 5 * i);
-            if (i == 0) {
+            if (WITH_PV && warp == 0 && j < 10) CITRUS_TR(51 + 4 * j);
+            if (j == 0) {
                 m_ref = m_new;
             } else {
+                // both threads of a row see the same values, so they take the same decision
                 const bool grow = (m_new - m_ref) > kRescaleTau;
                 if (__any_sync(0xffffffffu, grow)) {
                     const float f = ex2(m_ref - m_new);
                     l_run *= f;
-                    l_out *= f;
                     m_ref = m_new;
                     if (WITH_PV) {
-                        // O[wg] is quiescent here: its last writer, P.V of tile j-2, was issued before Q.K^T of
-                        // tile j, whose completion this warpgroup has just observed through s_full.
+                        // O must be quiescent: P.V of tile j-1 (and with it every earlier one) has retired
+                        ok = pv_done(j - 1);
+                        if (!ok) break;
+                        tc_fence_after();
 #pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {
+                        for (int c = 0; c < 2; ++c) {
                             uint32_t oreg[32];
-                            tmem_ld32(tmO(wg) + lane_base + c * 32, oreg);
+                            tmem_ld32(o_addr + half * 64 + c * 32, oreg);
                             tmem_wait_ld();
 #pragma unroll
                             for (int q = 0; q < 32; ++q) oreg[q] = __float_as_uint(__uint_as_float(oreg[q]) * f);
-                            tmem_st32(tmO(wg) + lane_base + c * 32, oreg);
+                            tmem_st32(o_addr + half * 64 + c * 32, oreg);
+                        }
+                        if (half == 0) {
+                            uint32_t lreg[16];
+                            tmem_ld16(tmem + kTmemL + lane_base, lreg);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) lreg[q] = __float_as_uint(__uint_as_float(lreg[q]) * f);
+                            tmem_st16(tmem + kTmemL + lane_base, lreg);
                         }
                     }
                 }
             }
-            // ---- sweep 2: probabilities.  l_run sums the fp32 values (it feeds the log-sum-exp that a2-L
-            // reuses); l_out sums the bf16-rounded ones that P.V actually multiplies, so that
-            // out = sum(p~ v) / sum(p~) stays a convex combination of V rows even when one key takes nearly
-            // all of the mass.  P piece c (16 packed columns) lands on S columns that sweep 2 has already read.
+            // ---- probabilities of this thread's 64 columns; with NEED_LSE the fp32 values are summed too (that sum
+            // feeds the log-sum-exp that the LM scoring pass reuses)
             const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f}, sumr4[4] = {0.f, 0.f, 0.f, 0.f};
-            // One 32-column piece: exponentials, bf16 packing, P store.  The loop below is ROLLED over pairs of
-            // pieces so the hot code stays small enough for the instruction cache of a scheduler running two
-            // of these warps, and the load of the next piece is in flight while the current one is computed.
-            auto piece = [&](uint32_t (&v)[32], int c) {
-                const int lim_c = lim - c * 32;
-                if (lim_c < 32) {
+            const uint64_t neg_m2 = pack_f32x2(neg_m, neg_m);
+            uint64_t sum2[2] = {0ull, 0ull};
+            uint32_t packed[32];
 #pragma unroll
-                    for (int q = 0; q < 32; ++q)
-                        if (q >= lim_c) v[q] = 0xff800000u;
-                }
-                uint32_t packed[16];
-#pragma unroll
-                for (int q = 0; q < 16; ++q) {
-                    float p0 = ex2(fmaf(__uint_as_float(v[2 * q]), scale2, neg_m));
-                    float p1 = ex2(fmaf(__uint_as_float(v[2 * q + 1]), scale2, neg_m));
-                    if (NEED_LSE) { sum4[q & 3] += p0; sum4[(q + 2) & 3] += p1; }
-                    packed[q] = pack_bf16(p0, p1);
-                    if (WITH_PV) {
-                        sumr4[q & 3] += __uint_as_float(packed[q] << 16);
-                        sumr4[(q + 2) & 3] += __uint_as_float(packed[q] & 0xffff0000u);
-                    }
-                }
-                if (WITH_PV) tmem_st16(s_addr + c * 16, packed);
-            };
-            {
-                uint32_t va[32], vb[32];
-                tmem_ld32(s_addr, va);
-#pragma unroll 1
-                for (int c = 0; c < 4; c += 2) {
-                    tmem_wait_ld();                                  // piece c has landed in va
-                    tmem_ld32(s_addr + (c + 1) * 32, vb);
-                    piece(va, c);
-                    tmem_wait_ld();                                  // piece c+1 has landed in vb
-                    if (c + 2 < 4) tmem_ld32(s_addr + (c + 2) * 32, va);
-                    piece(vb, c + 1);
-                }
+            for (int q = 0; q < 32; ++q) {
+                float x0, x1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(own[2 * q]), __uint_as_float(own[2 * q + 1])), scale2x2, neg_m2), x0, x1);
+                const float p0 = ex2(x0), p1 = ex2(x1);
+                if (NEED_LSE) sum2[q & 1] = add_f32x2(sum2[q & 1], pack_f32x2(p0, p1));
+                packed[q] = pack_bf16(p0, p1);
             }
-            l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-            l_out += (sumr4[0] + sumr4[1]) + (sumr4[2] + sumr4[3]);
-            if (WITH_PV && warp == 0) CITRUS_TR(52 + 5 * i);
-            if (WITH_PV) tmem_wait_st();
-            if (WITH_PV && warp == 0) CITRUS_TR(53 + 5 * i);
-            tc_fence_before();
-            mbar_arrive(smem_u32(&bars->p_full[wg]));
-            if (WITH_PV && warp == 0) CITRUS_TR(54 + 5 * i);
+            if (NEED_LSE) {
+                float a0, a1, b0, b1;
+                unpack_f32x2(sum2[0], a0, a1); unpack_f32x2(sum2[1], b0, b1);
+                l_run += (a0 + a1) + (b0 + b1);
+            }
+            if (WITH_PV && warp == 0 && j < 10) CITRUS_TR(52 + 4 * j);
+            if (WITH_PV) {
+                // the single P buffer is free once P.V of the previous tile has read it
+                if (j > 0) { ok = pv_done(j - 1); if (!ok) break; }
+                tc_fence_after();
+                tmem_st16(p_addr, packed);
+                tmem_st16(p_addr + 16, packed + 16);
+                tmem_wait_st();                                      // also covers a rescale's stores to O
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars->p_full));
+            }
+            if (WITH_PV && warp == 0 && j < 10) CITRUS_TR(53 + 4 * j);
         }
-        // ---- epilogue: merge the two warpgroups' partial results
-        if (ok && WITH_PV && i_last >= 0) {
-            // phases 0..i_last-1 of o_done[wg] are known complete (see the rescale note), so this parity
-            // wait can only mean "P.V of this warpgroup's last tile has retired"
-            ok = mbar_wait_warp(smem_u32(&bars->o_done[wg]), i_last & 1, p.status);
+        // ---- epilogue
+        if (ok && WITH_PV && nt > 0) ok = pv_done(nt - 1);
+        if (NEED_LSE) {
+            bars->lsum[half][row_in_tile] = l_run;
+            mbar_arrive(smem_u32(&bars->xch));
+            ok = mbar_wait_warp(smem_u32(&bars->xch), 0, p.status) && ok;
         }
-        bars->rows[wg][row_in_tile] = RowState{m_ref, l_run, l_out};
-        mbar_arrive(smem_u32(&bars->xch));
-        ok = mbar_wait_warp(smem_u32(&bars->xch), 0, p.status) && ok;
         if (ok) {
             tc_fence_after();
             if (warp == 0) CITRUS_TR(110);
-            const RowState mine = bars->rows[wg][row_in_tile], other = bars->rows[wg ^ 1][row_in_tile];
-            const float M = fmaxf(mine.m, other.m);                  // finite: tile 0 always has a visible column
-            const float w_mine = mine.m == -INFINITY ? 0.f : ex2(mine.m - M);
-            const float w_other = other.m == -INFINITY ? 0.f : ex2(other.m - M);
-            if (WITH_PV) {
-                // this thread finishes columns [64 wg, 64 wg + 64) of its row, from both accumulators
-                const float w0 = wg == 0 ? w_mine : w_other, w1 = wg == 0 ? w_other : w_mine;
-                const bool has1 = nt > 1;                            // O[1] was written at all
-                const float inv = 1.f / (mine.lo * w_mine + other.lo * w_other);
-                const float a0 = w0 * inv, a1 = w1 * inv;
-                uint8_t* stage = gQ + wg * kHalfBytes + row_in_tile * 128;   // [128 rows][64 bf16], 128-byte swizzle
+            if (WITH_PV && nt > 0) {
+                // this thread finishes columns [64 half, 64 half + 64) of its row
+                uint32_t lreg[16];
+                tmem_ld16(tmem + kTmemL + lane_base, lreg);
+                tmem_wait_ld();
+                const float inv = 1.f / __uint_as_float(lreg[0]);
+                uint8_t* stage = gQ + half * kHalfBytes + row_in_tile * 128;   // [128 rows][64 bf16], 128-byte swizzle
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    uint32_t o0[32], o1[32];
-                    tmem_ld32(tmO(0) + lane_base + wg * 64 + c * 32, o0);
-                    if (has1) tmem_ld32(tmO(1) + lane_base + wg * 64 + c * 32, o1);
+                    uint32_t o0[32];
+                    tmem_ld32(o_addr + half * 64 + c * 32, o0);
                     tmem_wait_ld();
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         float v[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            v[e] = __uint_as_float(o0[8 * q + e]) * a0;
-                            if (has1) v[e] = fmaf(__uint_as_float(o1[8 * q + e]), a1, v[e]);
-                        }
+                        for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(o0[8 * q + e]) * inv;
                         uint4 u;
                         u.x = pack_bf16(v[0], v[1]); u.y = pack_bf16(v[2], v[3]);
                         u.z = pack_bf16(v[4], v[5]); u.w = pack_bf16(v[6], v[7]);
@@ -576,12 +619,12 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                     }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_arrive(smem_u32(&bars->out_ready[wg]));
+                mbar_arrive(smem_u32(&bars->out_ready[half]));
                 if ((warp & 3) == 0) {
-                    // one warp per warpgroup stores its 128 x 64 half of the output tile
-                    if (mbar_wait_warp(smem_u32(&bars->out_ready[wg]), 0, p.status)) {
+                    // one warp per column half stores its 128 x 64 part of the output tile
+                    if (mbar_wait_warp(smem_u32(&bars->out_ready[half]), 0, p.status)) {
                         if (elect_one()) {
-                            tma_store_3d(&mapO, sQ + wg * kHalfBytes, wg * 64, h, q_row0);
+                            tma_store_3d(&mapO, sQ + half * kHalfBytes, half * 64, h, q_row0);
                             tma_store_wait_read();
                         }
                         __syncwarp();
@@ -596,11 +639,11 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 orow = row_in_tile % p.pack_rows;
                 row_ok = row_in_tile < p.pack * p.pack_rows;
             }
-            if (NEED_LSE && wg == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // see the note on the sweep order
-            if (NEED_LSE && wg == 0 && row_ok) {
-                const float l = mine.l * w_mine + other.l * w_other;
-                if (p.splits > 1) p.part[((size_t)split * p.q_heads + oh) * p.lse_stride + orow] = make_float2(M, l);
-                else if (p.lse2 != nullptr) p.lse2[(size_t)oh * p.lse_stride + orow] = M + log2f(l);
+            if (NEED_LSE && half == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // see the note on the sweep order
+            if (NEED_LSE && half == 0 && row_ok) {
+                const float l = bars->lsum[0][row_in_tile] + bars->lsum[1][row_in_tile];
+                if (p.splits > 1) p.part[((size_t)split * p.q_heads + oh) * p.lse_stride + orow] = make_float2(m_ref, l);
+                else if (p.lse2 != nullptr) p.lse2[(size_t)oh * p.lse_stride + orow] = m_ref + log2f(l);
             }
         }
     }
