@@ -2,6 +2,16 @@
 // (ordered gather of K, V and positions into the other ping-pong buffer).
 #include "citrus_internal.h"
 
+CITRUS_TRACE_EXPORT(_sc)
+#ifdef CITRUS_TRACE
+static __device__ __forceinline__ unsigned long long trace_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define CITRUS_SPAN_MIN(i) do { if (threadIdx.x == 0) atomicMax(&g_citrus_trace[(i)], ~trace_ns()); } while (0)
+#define CITRUS_SPAN_MAX(i) do { if (threadIdx.x == 0) atomicMax(&g_citrus_trace[(i)], trace_ns()); } while (0)
+#else
+#define CITRUS_SPAN_MIN(i) do { } while (0)
+#define CITRUS_SPAN_MAX(i) do { } while (0)
+#endif
+
 namespace citrus {
 namespace {
 
@@ -22,10 +32,14 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 // select finds the k-th largest key T and how many candidates equal to T are kept;
 // a flagged block scan in index order then emits kept indices ascending, taking the
 // lowest-index candidates among those equal to T.
+// `also(p, j)` is called for every kept candidate j with its place p in the ascending list (the fused kernel
+// uses it to hand the list to the gathering CTAs through shared memory).
+template <typename Also>
 __device__ __forceinline__ void select_body(const SelectJob& job, const int g, int kv_heads, int n, int k, int layerwise,
-                                            uint32_t* keys /* shared, [n] */) {
+                                            uint32_t* keys /* shared, [n] */, Also also) {
     __shared__ uint32_t hist[256];
-    __shared__ uint32_t s_prefix, s_remaining;
+    __shared__ uint32_t s_prefix, s_remaining, s_bin_count, s_n_short;
+    __shared__ uint32_t s_short[32];
     __shared__ uint32_t warp_gt[32], warp_eq[32];
 
     const int tid = threadIdx.x;
@@ -33,8 +47,10 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
     int* idx0 = job.idx + (size_t)g * k;
 
     if (n <= k) {                                  // nothing to evict: identity
-        for (int j = tid; j < n; j += kSelThreads)
+        for (int j = tid; j < n; j += kSelThreads) {
             for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * k + j] = j;
+            also(j, j);
+        }
         return;
     }
     for (int j = tid; j < n; j += kSelThreads) {
@@ -53,8 +69,9 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         }
         keys[j] = key;
     }
-    if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; }
+    if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; s_bin_count = (uint32_t)n; s_n_short = 0u; }
     __syncthreads();
+    CITRUS_TR(10);
 
     uint32_t mask = 0u;
     for (int shift = 24; shift >= 0; shift -= 8) {
@@ -66,9 +83,15 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
             const uint32_t key = j < n ? keys[j] : 0u;
             const bool act = j < n && (key & mask) == prefix;
             const uint32_t bin = (key >> shift) & 255u;
-            // scores of one head crowd into a few exponent bins: one shared-memory atomic per (warp, bin)
-            const uint32_t peers = __match_any_sync(0xffffffffu, act ? bin : 256u);
-            if (act && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+            // The leading digit (sign and exponent) is the same for nearly every score of a head, later digits are
+            // spread out: one atomic for the warp when all its lanes agree, otherwise one per lane.
+            int all_same;
+            __match_all_sync(0xffffffffu, act ? bin : 256u, &all_same);
+            if (all_same) {
+                if (act && (tid & 31) == 0) atomicAdd(&hist[bin], 32u);
+            } else if (act) {
+                atomicAdd(&hist[bin], 1u);
+            }
         }
         __syncthreads();
         if (tid < 32) {
@@ -93,10 +116,37 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
                 }
                 s_remaining = remaining - cum;                   // still to take inside bin b
                 s_prefix = prefix | ((uint32_t)b << shift);
+                s_bin_count = hist[b];
             }
         }
         mask |= 255u << shift;
         __syncthreads();
+        CITRUS_TR(11 + (24 - shift) / 8);
+        // Short cut: at most 32 candidates still share the prefix.  One warp ranks them directly instead of
+        // walking the remaining digits.
+        if (shift > 0 && s_bin_count <= 32u) {
+            const uint32_t prefix2 = s_prefix;
+            for (int j = tid; j < n; j += kSelThreads) {
+                const uint32_t key = keys[j];
+                if ((key & mask) == prefix2) s_short[atomicAdd(&s_n_short, 1u)] = key;
+            }
+            __syncthreads();
+            if (tid < 32) {
+                const uint32_t c = s_n_short, r = s_remaining;      // r-th largest of the c listed keys (1 <= r <= c)
+                const uint32_t mine = tid < (int)c ? s_short[tid] : 0u;
+                uint32_t n_gt = 0u, n_ge = 0u;
+                for (uint32_t i = 0; i < c; ++i) {
+                    const uint32_t other = __shfl_sync(0xffffffffu, mine, (int)i);
+                    n_gt += other > mine; n_ge += other >= mine;
+                }
+                if (tid < (int)c && n_gt < r && r <= n_ge) {        // every lane holding the r-th largest value writes the same
+                    s_prefix = mine;
+                    s_remaining = r - n_gt;
+                }
+            }
+            __syncthreads();
+            break;
+        }
     }
     const uint32_t T = s_prefix;                   // k-th largest key
     const uint32_t take_eq = s_remaining;          // candidates equal to T that are kept (lowest indices)
@@ -134,10 +184,12 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         if (keep) {
             uint32_t p = gt_before + min(eq_before, take_eq);
             for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * k + p] = j;
+            also((int)p, j);
         }
         gt_before += key > T;
         eq_before += key == T;
     }
+    CITRUS_TR(15);
 }
 
 __global__ void __launch_bounds__(kSelThreads)
@@ -145,16 +197,16 @@ select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int n,
     extern __shared__ uint32_t keys[];            // [n]
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the scores are final after this
-    select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, n, k, layerwise, keys);
+    select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, n, k, layerwise, keys, [](int, int) {});
 }
 
 // Rows [r_begin, r_end) of one (cache, head) are copied with 128-bit accesses, row_bytes/16 lanes per row.
 __device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4* __restrict__ chunkK,
                                              const uint4* __restrict__ chunkV, const int g, int kv_heads, int cap,
-                                             int row_vecs, int r_begin, int r_end, int chunk_pos0) {
+                                             int row_vecs, int r_begin, int r_end, int chunk_pos0, const int* idx) {
+    // idx[r] = candidate kept in row r of this head (global list, or the CTA's slice in shared memory)
     const int rows_per_pass = blockDim.x / row_vecs;
     const int sub = threadIdx.x / row_vecs, v = threadIdx.x % row_vecs;
-    const int* idx = job.idx + (size_t)g * cap;
     const uint4* srcK = reinterpret_cast<const uint4*>(job.srcK);
     const uint4* srcV = reinterpret_cast<const uint4*>(job.srcV);
     uint4* dstK = reinterpret_cast<uint4*>(job.dstK);
@@ -205,29 +257,49 @@ compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restr
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the index lists are final after this
     const int r0 = blockIdx.x * kCompactRowsPerCta;
     compact_rows(args.job[blockIdx.z], chunkK, chunkV, blockIdx.y, kv_heads, cap, row_vecs,
-                 r0, min(kept, r0 + kCompactRowsPerCta), chunk_pos0);
+                 r0, min(kept, r0 + kCompactRowsPerCta), chunk_pos0, args.job[blockIdx.z].idx + (size_t)blockIdx.y * cap);
 }
 
 // a3 + a4 in one launch: a cluster of kFusedCluster CTAs per (cache, KV head).  The first CTA of the cluster
-// selects, the cluster barrier publishes the index list, then every CTA gathers its share of the kept rows.
+// selects and writes each kept index twice: to the global list (part of the result) and into the shared memory
+// of the CTA that will gather that row; the cluster barrier publishes the slices, then every CTA gathers its
+// share of the kept rows without another trip to global memory for the indices.
 // grid: (kFusedCluster, KV heads, caches), cluster (kFusedCluster, 1, 1)
 constexpr int kFusedCluster = 8;
 
 __global__ void __launch_bounds__(kSelThreads)
 select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_constant__ CompactArgs cmp, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
                       int kv_heads, int n, int k, int row_vecs, int kept, int chunk_pos0) {
-    extern __shared__ uint32_t keys[];            // [n], used by the selecting CTA only
+    extern __shared__ uint32_t keys[];            // [n] order keys (selecting CTA only), then this CTA's slice of the list
     const int g = blockIdx.y;
+    const int per = (kept + kFusedCluster - 1) / kFusedCluster;
+    int* s_idx = reinterpret_cast<int*>(keys + n);     // [per]
     // programmatic dependent launch: let the next kernel start its prologue, then wait for the scores
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (blockIdx.x == 0) select_body(sel.job[blockIdx.z], g, kv_heads, n, k, 0, keys);
-    // hardware cluster barrier with release/acquire semantics: the index list written above is visible to all
+    CITRUS_SPAN_MIN(0);
+    // every CTA of the cluster is running (its shared memory may be written) once this first barrier completes
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    const int per = (kept + kFusedCluster - 1) / kFusedCluster;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    CITRUS_SPAN_MIN(1);
+    CITRUS_TR(9);
+    if (blockIdx.x == 0) {
+        const uint32_t slice = (uint32_t)__cvta_generic_to_shared(s_idx);
+        select_body(sel.job[blockIdx.z], g, kv_heads, n, k, 0, keys, [&](int p, int j) {
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(slice + 4u * (uint32_t)(p % per)), "r"(p / per));
+            asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(j) : "memory");
+        });
+    }
+    // hardware cluster barrier with release/acquire semantics: the slices written above are visible to their owners
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    CITRUS_SPAN_MAX(3);
+    CITRUS_TR(16);
     const int r0 = blockIdx.x * per;
-    compact_rows(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, k, row_vecs, r0, min(kept, r0 + per), chunk_pos0);
+    compact_rows(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, k, row_vecs, r0, min(kept, r0 + per), chunk_pos0, s_idx - r0);
+    CITRUS_SPAN_MAX(2);
+    CITRUS_TR(17);
 }
 
 }  // namespace
@@ -270,7 +342,7 @@ cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kFusedCluster, kv_heads, n_jobs);
     cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = (size_t)n * sizeof(uint32_t);
+    cfg.dynamicSmemBytes = ((size_t)n + (size_t)((kept + kFusedCluster - 1) / kFusedCluster)) * sizeof(uint32_t);
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;

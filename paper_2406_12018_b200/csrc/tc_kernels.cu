@@ -41,6 +41,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One arrival for the whole warp: every lane's earlier work (ordered by its own fences) is published by lane 0.
+// 32 per-thread arrivals on one barrier word are 32 serialised shared-memory atomics; this is one.
+__device__ __forceinline__ void mbar_arrive_warp(uint32_t bar) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -296,6 +302,7 @@ __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.b
 struct AttnSmem {
     uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
     uint64_t s_full[2], s_free[2], p_full, o_done[2], xch, out_ready[2], drain;
+    uint64_t turn[4][2];                // exponential-phase hand-over between the two warps of a scheduler
     uint32_t tmem_base;
     float lsum[2][kTile];               // fp32 row sums of the two column halves, exchanged once at the end
 };
@@ -348,11 +355,12 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
         for (int s = 0; s < kStagesK; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
         for (int s = 0; s < kStagesV; ++s) { mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1); }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 256);
-            mbar_init(smem_u32(&bars->o_done[b]), 1); mbar_init(smem_u32(&bars->out_ready[b]), 128);
+            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 8);
+            mbar_init(smem_u32(&bars->o_done[b]), 1); mbar_init(smem_u32(&bars->out_ready[b]), 4);
         }
-        mbar_init(smem_u32(&bars->p_full), 256);
-        mbar_init(smem_u32(&bars->xch), 256);
+        for (int w = 0; w < 4; ++w) { mbar_init(smem_u32(&bars->turn[w][0]), 1); mbar_init(smem_u32(&bars->turn[w][1]), 1); }
+        mbar_init(smem_u32(&bars->p_full), 8);
+        mbar_init(smem_u32(&bars->xch), 8);
         mbar_init(smem_u32(&bars->drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -405,7 +413,13 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             const int s = j % kStagesK, jg = sweep_tile(j);
             const bool from_cache = jg < n_cache_tiles;
             const int row = from_cache ? jg * kTile : (jg - n_cache_tiles) * kTile;
-            if (from_cache && !dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
+            if (from_cache && !dep_waited) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                dep_waited = true;
+#ifdef CITRUS_TRACE
+                if (WITH_PV && lane == 0) atomicMax(&g_citrus_trace[244], ~global_ns());
+#endif
+            }
             if (!mbar_wait_warp(smem_u32(&bars->k_empty[s]), ((j / kStagesK) & 1) ^ 1, p.status)) break;
             load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, g, !from_cache);
         }
@@ -479,7 +493,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             const int b = j & 1;
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (j >> 1) & 1, p.status);
             if (!ok) break;
-            if (WITH_PV && warp == 0 && j < 10) CITRUS_TR(50 + 4 * j);
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 200 : 50) + 5 * j);
             tc_fence_after();
             // number of visible columns of this tile for this row
             int lim = kTile;
@@ -499,7 +513,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             tmem_ld32(s_addr + half * 64 + 32, own + 32);
             tmem_wait_ld();
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars->s_free[b]));
+            mbar_arrive_warp(smem_u32(&bars->s_free[b]));
             if (lim < kTile) {
                 const int lim_own = lim - half * 64, lim_oth = lim - (half ^ 1) * 64;
 #pragma unroll
@@ -517,7 +531,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             }
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             const float m_new = fmaxf(m_ref, mx * scale2);
-            if (WITH_PV && warp == 0 && j < 10) CITRUS_TR(51 + 4 * j);
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 201 : 51) + 5 * j);
             if (j == 0) {
                 m_ref = m_new;
             } else {
@@ -558,6 +572,14 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             const uint64_t neg_m2 = pack_f32x2(neg_m, neg_m);
             uint64_t sum2[2] = {0ull, 0ull};
             uint32_t packed[32];
+            // Warps w and w+4 run on the same scheduler and share its exponential unit.  They take turns in this
+            // phase (w, then w+4, then w again for the next tile), which keeps them half a tile apart: while one
+            // computes exponentials the other waits for tensor memory, takes the row maximum or stores P.
+            if (half == 1 || j > 0) {
+                ok = mbar_wait_warp(smem_u32(&bars->turn[warp & 3][half]), (half == 1 ? j : j - 1) & 1, p.status);
+                if (!ok) break;
+            }
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 202 : 52) + 5 * j);
 #pragma unroll
             for (int q = 0; q < 32; ++q) {
                 float x0, x1;
@@ -566,12 +588,13 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 if (NEED_LSE) sum2[q & 1] = add_f32x2(sum2[q & 1], pack_f32x2(p0, p1));
                 packed[q] = pack_bf16(p0, p1);
             }
+            mbar_arrive_warp(smem_u32(&bars->turn[warp & 3][half ^ 1]));
             if (NEED_LSE) {
                 float a0, a1, b0, b1;
                 unpack_f32x2(sum2[0], a0, a1); unpack_f32x2(sum2[1], b0, b1);
                 l_run += (a0 + a1) + (b0 + b1);
             }
-            if (WITH_PV && warp == 0 && j < 10) CITRUS_TR(52 + 4 * j);
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 203 : 53) + 5 * j);
             if (WITH_PV) {
                 // the single P buffer is free once P.V of the previous tile has read it
                 if (j > 0) { ok = pv_done(j - 1); if (!ok) break; }
@@ -580,15 +603,15 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 tmem_st16(p_addr + 16, packed + 16);
                 tmem_wait_st();                                      // also covers a rescale's stores to O
                 tc_fence_before();
-                mbar_arrive(smem_u32(&bars->p_full));
+                mbar_arrive_warp(smem_u32(&bars->p_full));
             }
-            if (WITH_PV && warp == 0 && j < 10) CITRUS_TR(53 + 4 * j);
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 204 : 54) + 5 * j);
         }
         // ---- epilogue
         if (ok && WITH_PV && nt > 0) ok = pv_done(nt - 1);
         if (NEED_LSE) {
             bars->lsum[half][row_in_tile] = l_run;
-            mbar_arrive(smem_u32(&bars->xch));
+            mbar_arrive_warp(smem_u32(&bars->xch));
             ok = mbar_wait_warp(smem_u32(&bars->xch), 0, p.status) && ok;
         }
         if (ok) {
@@ -619,7 +642,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                     }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_arrive(smem_u32(&bars->out_ready[half]));
+                mbar_arrive_warp(smem_u32(&bars->out_ready[half]));
                 if ((warp & 3) == 0) {
                     // one warp per column half stores its 128 x 64 part of the output tile
                     if (mbar_wait_warp(smem_u32(&bars->out_ready[half]), 0, p.status)) {
@@ -671,7 +694,7 @@ attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     const int id = blockIdx.x;
 #ifdef CITRUS_TRACE
     unsigned long long t_start = 0;
-    if (threadIdx.x == 0) { t_start = global_ns(); atomicMin(&g_citrus_trace[240], t_start); }
+    if (threadIdx.x == 0) { t_start = global_ns(); atomicMax(&g_citrus_trace[240], ~t_start); }   // complemented: max = earliest
 #endif
     if (id < n_attn) {
         const int n_qt = (pa.rows + kTile - 1) / kTile;
@@ -712,6 +735,9 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
               const __grid_constant__ CUtensorMap mapSK, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#ifdef CITRUS_TRACE
+    if (threadIdx.x == 0) atomicMax(&g_citrus_trace[245], ~global_ns());
+#endif
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sK = base;
     const uint32_t sQ = sK + kTileBytes;
@@ -735,9 +761,9 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         mbar_init(smem_u32(&bars->k_full), 1);
         for (int s = 0; s < kColStages; ++s) { mbar_init(smem_u32(&bars->q_full[s]), 1); mbar_init(smem_u32(&bars->q_empty[s]), 1); }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 128);
+            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 4);
         }
-        for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&bars->lse_full[b]), 128);
+        for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&bars->lse_full[b]), 4);
         mbar_init(smem_u32(&bars->drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -747,6 +773,9 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     asm volatile("griddepcontrol.wait;" ::: "memory");      // pass 1's log-sum-exp values are final after this
+#ifdef CITRUS_TRACE
+    if (threadIdx.x == 0) atomicMax(&g_citrus_trace[246], ~global_ns());
+#endif
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
 
@@ -815,7 +844,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 }
             }
             bars->lse[it2 & 3][key_in_tile] = lse;
-            mbar_arrive(smem_u32(&bars->lse_full[it2 & 3]));
+            mbar_arrive_warp(smem_u32(&bars->lse_full[it2 & 3]));
         };
         if (nb > 0) stage_lse(0);
         for (int it = 0; it < nb; ++it) {
@@ -856,7 +885,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 }
             }
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars->s_free[b]));
+            mbar_arrive_warp(smem_u32(&bars->s_free[b]));
             acc += (part[0] + part[1]) + (part[2] + part[3]);
             if (warp == 0) CITRUS_TR(162 + 3 * (it & 7));
         }
@@ -865,6 +894,9 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (warp == 0) CITRUS_TR(190);
+#ifdef CITRUS_TRACE
+    if (threadIdx.x == 0) atomicMax(&g_citrus_trace[247], global_ns());
+#endif
     if (warp == 5) { __syncwarp(); tmem_dealloc(tmem, kColTmemCols); }
 }
 
