@@ -282,7 +282,7 @@ constexpr int kStagesK = 2;             // K ring
 constexpr int kStagesV = 2;             // V ring
 constexpr int kVStageBytes = kTileBytes + kHalfBytes;   // a V tile and, right behind it, a [128 keys][64] block of ones
 constexpr int kAttnThreads = 352;       // 8 softmax warps, K-TMA warp, MMA warp, V-TMA warp
-constexpr int kColThreads = 192;        // 4 column-sum warps, 1 TMA warp, 1 MMA warp
+constexpr int kColThreads = 320;        // 8 column-sum warps (two groups of four), 1 TMA warp, 1 MMA warp
 constexpr int kTmemCols = 512;
 constexpr uint32_t kTmemO = 256;        // O accumulator: 128 output columns + 16 columns that all hold the row sum of P
 constexpr uint32_t kTmemL = kTmemO + 128;
@@ -302,7 +302,6 @@ __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.b
 struct AttnSmem {
     uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
     uint64_t s_full[2], s_free[2], p_full, o_done[2], xch, out_ready[2], drain;
-    uint64_t turn[4][2];                // exponential-phase hand-over between the two warps of a scheduler
     uint32_t tmem_base;
     float lsum[2][kTile];               // fp32 row sums of the two column halves, exchanged once at the end
 };
@@ -358,7 +357,6 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 8);
             mbar_init(smem_u32(&bars->o_done[b]), 1); mbar_init(smem_u32(&bars->out_ready[b]), 4);
         }
-        for (int w = 0; w < 4; ++w) { mbar_init(smem_u32(&bars->turn[w][0]), 1); mbar_init(smem_u32(&bars->turn[w][1]), 1); }
         mbar_init(smem_u32(&bars->p_full), 8);
         mbar_init(smem_u32(&bars->xch), 8);
         mbar_init(smem_u32(&bars->drain), 1);
@@ -572,13 +570,6 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             const uint64_t neg_m2 = pack_f32x2(neg_m, neg_m);
             uint64_t sum2[2] = {0ull, 0ull};
             uint32_t packed[32];
-            // Warps w and w+4 run on the same scheduler and share its exponential unit.  They take turns in this
-            // phase (w, then w+4, then w again for the next tile), which keeps them half a tile apart: while one
-            // computes exponentials the other waits for tensor memory, takes the row maximum or stores P.
-            if (half == 1 || j > 0) {
-                ok = mbar_wait_warp(smem_u32(&bars->turn[warp & 3][half]), (half == 1 ? j : j - 1) & 1, p.status);
-                if (!ok) break;
-            }
             if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 202 : 52) + 5 * j);
 #pragma unroll
             for (int q = 0; q < 32; ++q) {
@@ -588,7 +579,6 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 if (NEED_LSE) sum2[q & 1] = add_f32x2(sum2[q & 1], pack_f32x2(p0, p1));
                 packed[q] = pack_bf16(p0, p1);
             }
-            mbar_arrive_warp(smem_u32(&bars->turn[warp & 3][half ^ 1]));
             if (NEED_LSE) {
                 float a0, a1, b0, b1;
                 unpack_f32x2(sum2[0], a0, a1); unpack_f32x2(sum2[1], b0, b1);
@@ -725,6 +715,7 @@ struct ColSmem {
     uint64_t k_full, q_full[kColStages], q_empty[kColStages], s_full[2], s_free[2], lse_full[4], drain;
     uint32_t tmem_base;
     alignas(16) float lse[4][kTile];          // log-sum-exp of the scoring rows of four consecutive (head, row block)s
+    float acc_other[kTile];                   // partial column sums of the second warp group
 };
 constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 2048;
 
@@ -768,7 +759,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 5) tmem_alloc(smem_u32(&bars->tmem_base), kColTmemCols);
+    if (warp == 9) tmem_alloc(smem_u32(&bars->tmem_base), kColTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -779,7 +770,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
 
-    if (warp == 4) {
+    if (warp == 8) {
         // TMA producer (converged warp)
         load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
         for (int it = 0; it < nb; ++it) {
@@ -789,7 +780,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             if (!mbar_wait_warp(smem_u32(&bars->q_empty[s]), ((it / kColStages) & 1) ^ 1, p.status)) break;
             load_tile(sQ + s * kTileBytes, &mapQ, smem_u32(&bars->q_full[s]), p.row0 + rb * kTile, h, true);
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // MMA issuer (converged warp)
         bool ok = mbar_wait_warp(smem_u32(&bars->k_full), 0, p.status);
         for (int it = 0; it < nb && ok; ++it) {
@@ -810,8 +801,11 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         __syncwarp();
         mbar_wait_warp(smem_u32(&bars->drain), 0, p.status);
     } else {
-        const int key_in_tile = warp * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        // Two groups of four warps: group 0 takes the even (head, row block) iterations and accumulator S[0],
+        // group 1 the odd ones and S[1]; thread i of either group owns candidate i of the tile.
+        const int group = warp >> 2;
+        const int key_in_tile = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const float scale2 = kLog2e * rsqrtf((float)kD);
         const int j = kt < n_cache_tiles ? key_row0 + key_in_tile : p.m + key_row0 + key_in_tile;   // candidate index
         const int n_src = from_cache ? p.m : p.L;
@@ -821,33 +815,41 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (p.causal && !from_cache) r_first = max(0, key_row0 + key_in_tile - p.t0);
         float acc = 0.f;
         bool ok = true;
-        // Stage the log-sum-exp values of iteration `it2` (thread i brings row r0 + i) into buffer it2 & 3.  It is
-        // called one iteration ahead, so the global load hides behind the current iteration's exponentials.  A
-        // thread that is in iteration `it` has seen the MMA of `it`, which needed everybody's s_free of it-2,
-        // i.e. everybody has finished reading buffer (it+1) & 3 = (it-3) & 3.
-        auto stage_lse = [&](int it2) {
+        // The log-sum-exp values of iteration `it2` (thread i brings row r0 + i) go to buffer it2 & 3.  The global
+        // load is issued one iteration before its value is stored to shared memory, so its latency hides behind
+        // the exponentials in between.  A thread that is in iteration `it` has seen the MMA of `it`, which needed
+        // everybody's s_free of it-2, i.e. everybody has finished reading buffer (it+1) & 3 = (it-3) & 3.
+        auto fetch_lse = [&](int it2) -> float {
             const int h2 = g * G + it2 / rb_per_head;
             const int rr = (rb0 + it2 % rb_per_head) * kTile + key_in_tile;
             float lse = INFINITY;
             if (rr < p.rows) {
                 if (p.splits > 1) {                              // merge the key splits of pass 1
+                    float2 ml[kMaxLseSplits];
+#pragma unroll
+                    for (int sp = 0; sp < kMaxLseSplits; ++sp)
+                        ml[sp] = sp < p.splits ? __ldg(&p.part[((size_t)sp * p.q_heads + h2) * p.lse_stride + rr])
+                                               : make_float2(-INFINITY, 0.f);
                     float M = -INFINITY, l = 0.f;
-                    for (int sp = 0; sp < p.splits; ++sp)
-                        M = fmaxf(M, __ldg(&p.part[((size_t)sp * p.q_heads + h2) * p.lse_stride + rr]).x);
-                    for (int sp = 0; sp < p.splits; ++sp) {
-                        const float2 ml = __ldg(&p.part[((size_t)sp * p.q_heads + h2) * p.lse_stride + rr]);
-                        l += ml.y * ex2(ml.x - M);
-                    }
+#pragma unroll
+                    for (int sp = 0; sp < kMaxLseSplits; ++sp) M = fmaxf(M, ml[sp].x);
+#pragma unroll
+                    for (int sp = 0; sp < kMaxLseSplits; ++sp) l += ml[sp].x == -INFINITY ? 0.f : ml[sp].y * ex2(ml[sp].x - M);
                     lse = M + log2f(l);
                 } else {
                     lse = __ldg(p.lse_in + (size_t)h2 * p.lse_stride + rr);
                 }
             }
+            return lse;
+        };
+        auto publish_lse = [&](int it2, float lse) {
             bars->lse[it2 & 3][key_in_tile] = lse;
             mbar_arrive_warp(smem_u32(&bars->lse_full[it2 & 3]));
         };
-        if (nb > 0) stage_lse(0);
-        for (int it = 0; it < nb; ++it) {
+        float lse_next = INFINITY;
+        if (nb > group) publish_lse(group, fetch_lse(group));
+        if (nb > group + 2) lse_next = fetch_lse(group + 2);
+        for (int it = group; it < nb; it += 2) {
             const int b = it & 1;
             const int rb = rb0 + it % rb_per_head;
             const int r0 = rb * kTile;
@@ -856,7 +858,8 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 1) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(160 + 3 * (it & 7));
-            if (it + 1 < nb) stage_lse(it + 1);
+            if (it + 2 < nb) publish_lse(it + 2, lse_next);      // loaded one iteration ago
+            if (it + 4 < nb) lse_next = fetch_lse(it + 4);       // lands during this iteration's exponentials
             ok = mbar_wait_warp(smem_u32(&bars->lse_full[lb]), (it >> 2) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(161 + 3 * (it & 7));
@@ -889,7 +892,10 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             acc += (part[0] + part[1]) + (part[2] + part[3]);
             if (warp == 0) CITRUS_TR(162 + 3 * (it & 7));
         }
-        if (ok && key_ok) p.scores[(size_t)g * p.score_stride + j] = acc;
+        // all eight column-sum warps arrive here, also after a wait that gave up
+        if (group == 1) bars->acc_other[key_in_tile] = acc;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (group == 0 && ok && key_ok) p.scores[(size_t)g * p.score_stride + j] = acc + bars->acc_other[key_in_tile];
     }
     tc_fence_before();
     __syncthreads();
@@ -897,7 +903,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 #ifdef CITRUS_TRACE
     if (threadIdx.x == 0) atomicMax(&g_citrus_trace[247], global_ns());
 #endif
-    if (warp == 5) { __syncwarp(); tmem_dealloc(tmem, kColTmemCols); }
+    if (warp == 9) { __syncwarp(); tmem_dealloc(tmem, kColTmemCols); }
 }
 
 // ------------------------------------------------------------------ host side
