@@ -709,15 +709,15 @@ attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 }
 
 // ------------------------------------------------------------------ column sums (a2 pass 2)
-constexpr int kColStages = 3;
-constexpr int kColTmemCols = 256;
+constexpr int kColStages = 4;
+constexpr int kColTmemCols = 512;         // four S^T accumulators: Q.K^T of four iterations can be in flight
 struct ColSmem {
-    uint64_t k_full, q_full[kColStages], q_empty[kColStages], s_full[2], s_free[2], lse_full[4], drain;
+    uint64_t k_full, q_full[kColStages], q_empty[kColStages], s_full[4], s_free[4], lse_full[8], drain;
     uint32_t tmem_base;
-    alignas(16) float lse[4][kTile];          // log-sum-exp of the scoring rows of four consecutive (head, row block)s
+    alignas(16) float lse[8][kTile];          // log-sum-exp of the scoring rows of eight consecutive (head, row block)s
     float acc_other[kTile];                   // partial column sums of the second warp group
 };
-constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 2048;
+constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 8192;
 
 // grid: (candidate tiles, kv_heads).  Accumulator rows = 128 candidates, columns = scoring rows of one
 // (head, row block); thread i owns candidate i and adds exp2(logit2 - lse2[row]) over its columns.
@@ -751,10 +751,10 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars->k_full), 1);
         for (int s = 0; s < kColStages; ++s) { mbar_init(smem_u32(&bars->q_full[s]), 1); mbar_init(smem_u32(&bars->q_empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < 4; ++b) {
             mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 4);
         }
-        for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&bars->lse_full[b]), 4);
+        for (int b = 0; b < 8; ++b) mbar_init(smem_u32(&bars->lse_full[b]), 4);
         mbar_init(smem_u32(&bars->drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -763,33 +763,39 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // pass 1's log-sum-exp values are final after this
-#ifdef CITRUS_TRACE
-    if (threadIdx.x == 0) atomicMax(&g_citrus_trace[246], ~global_ns());
-#endif
+    // Programmatic dependent launch: the scoring queries and the chunk's keys are the caller's inputs and are loaded
+    // at once; what the preceding kernels produce is touched only after griddepcontrol.wait - a retained-cache
+    // tile (written by the previous chunk's compaction), the log-sum-exp values of pass 1, and the score vector
+    // (still read by the previous chunk's select until that kernel has ended).
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
 
     if (warp == 8) {
         // TMA producer (converged warp)
-        load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
-        for (int it = 0; it < nb; ++it) {
+        auto load_q = [&](int it) {
             const int s = it % kColStages;
             const int h = g * G + it / rb_per_head;
             const int rb = rb0 + it % rb_per_head;
-            if (!mbar_wait_warp(smem_u32(&bars->q_empty[s]), ((it / kColStages) & 1) ^ 1, p.status)) break;
+            if (!mbar_wait_warp(smem_u32(&bars->q_empty[s]), ((it / kColStages) & 1) ^ 1, p.status)) return false;
             load_tile(sQ + s * kTileBytes, &mapQ, smem_u32(&bars->q_full[s]), p.row0 + rb * kTile, h, true);
-        }
+            return true;
+        };
+        bool ok = true;
+        int it = 0;
+        for (; it < nb && it < kColStages && ok; ++it) ok = load_q(it);
+        if (from_cache) asm volatile("griddepcontrol.wait;" ::: "memory");
+        load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
+        for (; it < nb && ok; ++it) ok = load_q(it);
     } else if (warp == 9) {
         // MMA issuer (converged warp)
         bool ok = mbar_wait_warp(smem_u32(&bars->k_full), 0, p.status);
         for (int it = 0; it < nb && ok; ++it) {
-            const int s = it % kColStages, b = it & 1;
+            const int s = it % kColStages, b = it & 3;
             const int rb = rb0 + it % rb_per_head;
             const int ncols = min(kTile, ((p.rows - rb * kTile) + 31) & ~31);     // whole 32-column pieces
             ok = mbar_wait_warp(smem_u32(&bars->q_full[s]), (it / kColStages) & 1, p.status);
             if (!ok) break;
-            ok = mbar_wait_warp(smem_u32(&bars->s_free[b]), ((it >> 1) & 1) ^ 1, p.status);
+            ok = mbar_wait_warp(smem_u32(&bars->s_free[b]), ((it >> 2) & 1) ^ 1, p.status);
             if (!ok) break;
             tc_fence_after();
             CITRUS_TR(140 + 2 * (it & 7));
@@ -801,8 +807,12 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         __syncwarp();
         mbar_wait_warp(smem_u32(&bars->drain), 0, p.status);
     } else {
-        // Two groups of four warps: group 0 takes the even (head, row block) iterations and accumulator S[0],
-        // group 1 the odd ones and S[1]; thread i of either group owns candidate i of the tile.
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef CITRUS_TRACE
+        if (threadIdx.x == 0) atomicMax(&g_citrus_trace[246], ~global_ns());
+#endif
+        // Two groups of four warps: group 0 takes the even (head, row block) iterations (accumulators S[0], S[2]),
+        // group 1 the odd ones (S[1], S[3]); thread i of either group owns candidate i of the tile.
         const int group = warp >> 2;
         const int key_in_tile = (warp & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -815,10 +825,11 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (p.causal && !from_cache) r_first = max(0, key_row0 + key_in_tile - p.t0);
         float acc = 0.f;
         bool ok = true;
-        // The log-sum-exp values of iteration `it2` (thread i brings row r0 + i) go to buffer it2 & 3.  The global
-        // load is issued one iteration before its value is stored to shared memory, so its latency hides behind
-        // the exponentials in between.  A thread that is in iteration `it` has seen the MMA of `it`, which needed
-        // everybody's s_free of it-2, i.e. everybody has finished reading buffer (it+1) & 3 = (it-3) & 3.
+        // The log-sum-exp values of iteration `it2` (thread i brings row r0 + i) go to buffer it2 & 7.  The global
+        // load is issued one iteration of the group before its value is stored to shared memory, so its latency
+        // hides behind the exponentials in between.  A thread in iteration `it` publishes iteration it+2 into the
+        // buffer last read in iteration it-6; it has seen the MMA of `it`, which needed s_free of it-4 from all four
+        // warps of the group, so everybody has finished reading that buffer.
         auto fetch_lse = [&](int it2) -> float {
             const int h2 = g * G + it2 / rb_per_head;
             const int rr = (rb0 + it2 % rb_per_head) * kTile + key_in_tile;
@@ -843,24 +854,24 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             return lse;
         };
         auto publish_lse = [&](int it2, float lse) {
-            bars->lse[it2 & 3][key_in_tile] = lse;
-            mbar_arrive_warp(smem_u32(&bars->lse_full[it2 & 3]));
+            bars->lse[it2 & 7][key_in_tile] = lse;
+            mbar_arrive_warp(smem_u32(&bars->lse_full[it2 & 7]));
         };
         float lse_next = INFINITY;
         if (nb > group) publish_lse(group, fetch_lse(group));
         if (nb > group + 2) lse_next = fetch_lse(group + 2);
         for (int it = group; it < nb; it += 2) {
-            const int b = it & 1;
+            const int b = it & 3;
             const int rb = rb0 + it % rb_per_head;
             const int r0 = rb * kTile;
             const int ncols = min(kTile, p.rows - r0);
-            const int lb = it & 3;
-            ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 1) & 1, p.status);
+            const int lb = it & 7;
+            ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 2) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(160 + 3 * (it & 7));
             if (it + 2 < nb) publish_lse(it + 2, lse_next);      // loaded one iteration ago
             if (it + 4 < nb) lse_next = fetch_lse(it + 4);       // lands during this iteration's exponentials
-            ok = mbar_wait_warp(smem_u32(&bars->lse_full[lb]), (it >> 2) & 1, p.status);
+            ok = mbar_wait_warp(smem_u32(&bars->lse_full[lb]), (it >> 3) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(161 + 3 * (it & 7));
             tc_fence_after();
