@@ -512,15 +512,9 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive_warp(smem_u32(&bars->s_free[b]));
-            if (lim < kTile) {
-                const int lim_own = lim - half * 64, lim_oth = lim - (half ^ 1) * 64;
-#pragma unroll
-                for (int q = 0; q < 64; ++q) {
-                    if (q >= lim_own) own[q] = 0xff800000u;          // -inf
-                    if (q >= lim_oth) oth[q] = 0xff800000u;
-                }
-            }
-            // ---- row maximum over all 128 columns
+            // ---- row maximum over all 128 columns.  Hidden columns (future tokens of the chunk, rows past the end of
+            // the cache or chunk, which TMA zero-fills) take part: the result only serves as the exponent reference,
+            // any finite value near the visible maximum does, and both threads of the row still agree on it.
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int q = 0; q < 64; q += 2) {
@@ -570,6 +564,12 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             const uint64_t neg_m2 = pack_f32x2(neg_m, neg_m);
             uint64_t sum2[2] = {0ull, 0ull};
             uint32_t packed[32];
+            if (lim - half * 64 < 64) {                              // hidden columns get probability zero
+                const int lim_own = lim - half * 64;
+#pragma unroll
+                for (int q = 0; q < 64; ++q)
+                    if (q >= lim_own) own[q] = 0xff800000u;          // -inf
+            }
             if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 202 : 52) + 5 * j);
 #pragma unroll
             for (int q = 0; q < 32; ++q) {
