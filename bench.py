@@ -190,7 +190,7 @@ def run_ours(args, rank, world, local_rank):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    w = wl.CONFIGS[args.workload]
+    w = {**wl.CONFIGS, **wl.PAPER_SHAPES}[args.workload]
     if args.doc_tokens:
         w = wl.scaled(w, doc_tokens=args.doc_tokens, n_seqs=1, min_tokens=0)
     doc = rank_document(w, rank)
@@ -351,7 +351,8 @@ def main():
     ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=WORKLOAD, choices=[k for k, v in wl.CONFIGS.items() if v.dtype == "bf16"],
+    ap.add_argument("--workload", default=WORKLOAD,
+                    choices=[k for k, v in {**wl.CONFIGS, **wl.PAPER_SHAPES}.items() if v.dtype == "bf16"],
                     help="another named workload (layer 0, one sequence) instead of the headline one")
     ap.add_argument("--doc-tokens", type=int, default=0, help="truncate / set the document length")
     ap.add_argument("--no-graph", action="store_true", help="launch every chunk from the host instead of a CUDA graph")

@@ -71,6 +71,18 @@ CONFIGS = {
 }
 
 
+# The paper's own setting (Section "Hyperparameters": k = 768, l_s = 256, cache of 1024 while reading) on the head
+# geometries of its backbone models; one decoder layer each, shared cache.
+PAPER_SHAPES = {
+    "paper_mistral7b": Workload("paper_mistral7b", 11, 1, 32, 8, 128, 768, 256, 16384, 64, "bf16", "shared",
+                                n_planted=32, n_sinks=1),
+    "paper_llama2_13b": Workload("paper_llama2_13b", 12, 1, 40, 40, 128, 768, 256, 16384, 64, "bf16", "shared",
+                                 n_planted=32, n_sinks=1),
+    "paper_llama3_8b": Workload("paper_llama3_8b", 13, 1, 32, 8, 128, 768, 256, 16384, 64, "bf16", "individual",
+                                lm_window=64, n_planted=32, n_sinks=1),
+}
+
+
 def scaled(w: Workload, **kw) -> Workload:
     """A smaller or altered copy of a workload (for tests)."""
     return replace(w, **kw)

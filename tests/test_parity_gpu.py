@@ -133,6 +133,24 @@ def test_config2_mistral_layer_full_document():
     ctx.close()
 
 
+@pytest.mark.parametrize("name", sorted(wl.PAPER_SHAPES))
+def test_paper_setting_k768_ls256_on_backbone_head_geometries(name):
+    # the paper's own (k, l_s) on 32/8, 40/40 and 32/8-individual heads: two query tiles per head, so the grid is
+    # smaller than the machine and the instruction log-sum-exp pass runs split over key ranges
+    w = wl.scaled(wl.PAPER_SHAPES[name], doc_tokens=2560 + 77)
+    ctx = pu.make_pair(w)
+    doc, st = pu.run_document(w, ctx)
+    _report(name, st)
+    for cid in range(2 if w.mode == "individual" else 1):
+        P = ctx.cache_view(0, cid)[2]
+        assert P.shape[1] == w.budget_k
+    P = ctx.cache_view(0, 1 if w.mode == "individual" else 0)[2]
+    for g in range(w.kv_heads):
+        kept = set(P[g].tolist())
+        assert set(doc.planted.tolist()) <= kept and set(doc.sinks.tolist()) <= kept
+    ctx.close()
+
+
 def test_config3_llama_stack_sampled():
     w = C["llama2_7b_stack"]
     layers = [0, 17, 31]
