@@ -220,6 +220,17 @@ int citrus_importance_static(const void* Q_s, int n_s, const void* K, int n_keys
                              float* scores, int score_stride, int* device_status,
                              citrus_stream_t stream);
 
+/*
+ * Intersection ratio of the appendix "Details for the Intersection Probing Experiments":
+ *   ratio[g] = | C(g)  intersect  C^I(g) | / | C^I(g) |
+ * over the states currently retained for KV head g by the language-modelling cache C (selected by the document
+ * context) and by the instruction cache C^I of (layer, seq_slot); states are identified by their original token
+ * position.  Individual mode only (CITRUS_ERR_STATE otherwise, and before the first step).  ratio_dev: device,
+ * [kv_heads] fp32, caller-owned; written by work enqueued on `stream`, which must be ordered after the last
+ * process call of that unit.
+ */
+int citrus_intersection_ratio(citrus_handle h, int layer, int seq_slot, float* ratio_dev, citrus_stream_t stream);
+
 /* Reads the device status word (0, or CITRUS_ERR_TIMEOUT if a bounded wait in a
  * kernel gave up). Synchronises the device. */
 int citrus_poll_status(citrus_handle h);

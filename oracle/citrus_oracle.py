@@ -139,6 +139,19 @@ def kth_gap(score: np.ndarray, k: int):
 
 
 # --------------------------------------------------------------------------
+# Diagnostic of the appendix "Details for the Intersection Probing Experiments":
+# |C_context  intersect  C_instruction| / |C_instruction| for two sets of retained states
+# --------------------------------------------------------------------------
+def intersection_ratio(pos_context: np.ndarray, pos_instruction: np.ndarray) -> np.ndarray:
+    """pos_* [H_kv, rows] original token positions of two caches; ratio per head."""
+    out = np.zeros(pos_instruction.shape[0], dtype=np.float64)
+    for g in range(pos_instruction.shape[0]):
+        a, b = set(pos_context[g].tolist()), set(pos_instruction[g].tolist())
+        out[g] = len(a & b) / len(b)
+    return out
+
+
+# --------------------------------------------------------------------------
 # Step a4 -- the evicted cache C-hat of Eq. 3 with the chunk's states put in
 # --------------------------------------------------------------------------
 def compact(Kcache_g, Vcache_g, pos_g, Kc_g, Vc_g, chunk_pos, idx):

@@ -28,7 +28,7 @@ KERNEL_NAMES = ["attention", "score_lse", "colsum", "select", "compact"]
 EXPORTS = [
     "citrus_create", "citrus_set_batch", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
     "citrus_process_chunk_host", "citrus_process_chunk_batch", "citrus_cache_view", "citrus_step_view", "citrus_profile",
-    "citrus_profile_read", "citrus_importance_static", "citrus_poll_status",
+    "citrus_profile_read", "citrus_importance_static", "citrus_intersection_ratio", "citrus_poll_status",
     "citrus_destroy", "citrus_strerror",
 ]
 
@@ -61,6 +61,7 @@ def load() -> C.CDLL:
     lib.citrus_cache_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(i)]
     lib.citrus_step_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(i), C.POINTER(vp),
                                      C.POINTER(i), C.POINTER(i), C.POINTER(i)]
+    lib.citrus_intersection_ratio.argtypes = [vp, i, i, vp, vp]
     lib.citrus_profile.argtypes = [vp, i]
     lib.citrus_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     lib.citrus_importance_static.argtypes = [vp, i, vp, i, i, i, i, C.c_uint, vp, i, vp, vp]
@@ -192,6 +193,14 @@ class Citrus:
             Kt, Vt = (_view(p.value, (H, k, D), "<i2", 2).view(torch.bfloat16) for p in (K, V))
         Pt = _view(P.value, (H, k), "<i4", 4)
         return Kt[:, :n.value], Vt[:, :n.value], Pt[:, :n.value]
+
+    def intersection_ratio(self, layer, slot=0, stream=None) -> torch.Tensor:
+        """[H_kv] fp32: share of the instruction cache's states that the language-modelling cache also holds."""
+        out = torch.empty(self.kv_heads, dtype=torch.float32, device="cuda")
+        rc = load().citrus_intersection_ratio(self._h, layer, slot, out.data_ptr(), _stream_ptr(stream))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_intersection_ratio")
+        return out
 
     def step_view(self, layer, which=0, slot=0):
         """(scores [H_kv, n] fp32, idx [H_kv, kept] int32, m_before) of the last call."""

@@ -421,6 +421,18 @@ int citrus_cache_view(citrus_handle h, int layer, int which, int seq_slot,
     return CITRUS_OK;
 }
 
+int citrus_intersection_ratio(citrus_handle h, int layer, int seq_slot, float* ratio_dev, citrus_stream_t stream) {
+    if (h == nullptr || !is_live(h) || ratio_dev == nullptr) return CITRUS_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= h->layers) return CITRUS_ERR_LAYER;
+    if (seq_slot < 0 || seq_slot >= h->n_slots) return CITRUS_ERR_INVALID_ARG;
+    if (!h->individual || h->units.empty()) return CITRUS_ERR_STATE;
+    const Unit& u = h->units[(size_t)layer * h->n_slots + seq_slot];
+    if (u.m < 1) return CITRUS_ERR_STATE;
+    const CacheBufs &lm = u.cache[0], &in = u.cache[1];
+    return cuda_rc(intersection_ratio(lm.pos[lm.cur], in.pos[in.cur], h->k, u.m, h->Hkv, ratio_dev,
+                                      reinterpret_cast<cudaStream_t>(stream)));
+}
+
 int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
                      const float** scores, int* score_stride, const int** idx,
                      int* n_candidates, int* n_kept, int* m_before) {

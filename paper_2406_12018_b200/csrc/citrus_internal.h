@@ -94,4 +94,7 @@ cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, c
 // a3 + a4 in one launch (per-head granularity): clusters of CTAs per (cache, KV head).
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
                            int kv_heads, int n, int k, int row_bytes, int kept, int chunk_pos0, cudaStream_t s);
+// ratio[g] = |{positions of a} intersect {positions of b}| / rows over two ascending position lists per head
+cudaError_t intersection_ratio(const int* pos_a, const int* pos_b, int pos_stride, int rows, int kv_heads, float* ratio,
+                               cudaStream_t s);
 }  // namespace citrus

@@ -302,7 +302,39 @@ select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_const
     CITRUS_TR(17);
 }
 
+// One CTA per KV head: thread t looks element t, t + 256, ... of list b up in list a (both strictly ascending) by
+// binary search; the hits are counted with a warp reduction and one shared-memory atomic per warp.
+__global__ void __launch_bounds__(256)
+intersection_kernel(const int* __restrict__ pos_a, const int* __restrict__ pos_b, int pos_stride, int rows, float* __restrict__ ratio) {
+    __shared__ int hits;
+    const int g = blockIdx.x;
+    const int* a = pos_a + (size_t)g * pos_stride;
+    const int* b = pos_b + (size_t)g * pos_stride;
+    if (threadIdx.x == 0) hits = 0;
+    __syncthreads();
+    int mine = 0;
+    for (int i = threadIdx.x; i < rows; i += blockDim.x) {
+        const int x = b[i];
+        int lo = 0, hi = rows;                    // first index with a[idx] >= x
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (a[mid] < x) lo = mid + 1; else hi = mid;
+        }
+        mine += lo < rows && a[lo] == x;
+    }
+    mine = __reduce_add_sync(0xffffffffu, mine);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&hits, mine);
+    __syncthreads();
+    if (threadIdx.x == 0) ratio[g] = (float)hits / (float)rows;
+}
+
 }  // namespace
+
+cudaError_t intersection_ratio(const int* pos_a, const int* pos_b, int pos_stride, int rows, int kv_heads, float* ratio,
+                               cudaStream_t s) {
+    intersection_kernel<<<kv_heads, 256, 0, s>>>(pos_a, pos_b, pos_stride, rows, ratio);
+    return cudaGetLastError();
+}
 
 cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, int k, int layerwise, cudaStream_t s) {
     if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;

@@ -364,6 +364,21 @@ def test_start_size_keeps_initial_tokens_and_fills_the_rest_by_score():
         assert kept[s0:] == [cand_pos[j] for j in best]
 
 
+def test_intersection_ratio_on_a_worked_example_and_its_limits():
+    from oracle import intersection_ratio
+    ctx = np.array([[0, 2, 4, 6, 8, 10], [1, 3, 5, 7, 9, 11]])
+    ins = np.array([[0, 1, 2, 3, 4, 5], [0, 2, 4, 6, 8, 10]])
+    # head 0 shares {0, 2, 4}; head 1 shares nothing
+    assert intersection_ratio(ctx, ins).tolist() == [0.5, 0.0]
+    assert intersection_ratio(ins, ins).tolist() == [1.0, 1.0]
+    rng = np.random.default_rng(3)
+    a = np.sort(rng.choice(1000, size=(3, 200), replace=False) if False else np.stack([rng.choice(1000, 200, replace=False) for _ in range(3)]), axis=1)
+    b = np.stack([np.sort(rng.choice(1000, 200, replace=False)) for _ in range(3)])
+    r = intersection_ratio(a, b)
+    for g in range(3):
+        assert r[g] == sum(int(x in set(a[g].tolist())) for x in b[g].tolist()) / 200   # counted one by one
+
+
 def test_forced_selection_is_adopted():
     rng = np.random.default_rng(16)
     N, Hq, Hkv, D, k = 10, 2, 1, 4, 3

@@ -151,6 +151,27 @@ def test_paper_setting_k768_ls256_on_backbone_head_geometries(name):
     ctx.close()
 
 
+def test_intersection_ratio_of_the_two_caches_matches_the_set_definition():
+    from oracle import intersection_ratio
+    w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=4, head_dim=128, budget_k=300, chunk_s=256, doc_tokens=1500,
+                  n_instr=24, dtype="bf16", mode="individual", lm_window=32, n_planted=6, n_sinks=1)
+    ctx = pu.make_pair(w)
+    with pytest.raises(CitrusError):
+        ctx.intersection_ratio(0)                                     # nothing retained yet
+    pu.run_document(w, ctx)
+    r = ctx.intersection_ratio(0)
+    torch.cuda.synchronize()
+    pos_lm, pos_in = (ctx.cache_view(0, cid)[2].cpu().numpy() for cid in (0, 1))
+    expect = intersection_ratio(pos_lm, pos_in)
+    assert np.array_equal(r.cpu().numpy(), expect.astype(np.float32))   # integer counts over the same denominator
+    assert 0.0 < float(r.min()) and float(r.max()) < 1.0                # the two caches differ, but share states
+    ctx.close()
+    shared = pu.make_pair(wl.scaled(w, mode="shared"))
+    with pytest.raises(CitrusError):
+        shared.intersection_ratio(0)
+    shared.close()
+
+
 def test_config3_llama_stack_sampled():
     w = C["llama2_7b_stack"]
     layers = [0, 17, 31]
