@@ -59,6 +59,11 @@ typedef struct CUstream_st* citrus_stream_t;
 #define CITRUS_MODE_START_SIZE(n) (((unsigned)(n) & 0xFu) << 24)   /* always keep the first n tokens (appendix on
                                              initial tokens; the paper's variant uses 4, its main setting 0); n <= budget_k */
 #define CITRUS_MODE_LM_WINDOW(w) (((unsigned)(w) & 0xFFFFu) << 8)   /* w scoring queries for C; 0 = whole chunk */
+#define CITRUS_MODE_ACCUMULATE  0x20000000u /* accumulative score policy (the "H2O + Shared Cache" variant named in the
+                                             Baselines section): a retained state's importance is the sum of the
+                                             scores it received at every step since it entered the cache; a chunk's
+                                             own states start at this step's score.  citrus_step_view then shows the
+                                             accumulated scores. */
 
 #define CITRUS_OK                 0
 #define CITRUS_ERR_INVALID_ARG   -1

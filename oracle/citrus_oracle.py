@@ -170,6 +170,7 @@ class CacheState:
     K: np.ndarray      # [H_kv, m, D]
     V: np.ndarray      # [H_kv, m, D]
     pos: np.ndarray    # [H_kv, m] original token positions, ascending per head
+    acc: Optional[np.ndarray] = None   # [H_kv, m] importance carried over from earlier steps (accumulate policy)
 
 
 @dataclass
@@ -195,13 +196,17 @@ class CitrusOracle:
     """
 
     def __init__(self, q_heads, kv_heads, head_dim, budget_k, mode=SHARED,
-                 lm_window: Optional[int] = None, layerwise: bool = False, start_size: int = 0):
+                 lm_window: Optional[int] = None, layerwise: bool = False, start_size: int = 0,
+                 accumulate: bool = False):
         assert q_heads % kv_heads == 0
         self.Hq, self.Hkv, self.D, self.k = q_heads, kv_heads, head_dim, budget_k
         self.mode = mode
         self.lm_window = lm_window          # None -> every chunk query votes (Eq. 1)
         self.layerwise = layerwise
         self.start_size = start_size        # initial tokens that are always preserved (appendix on initial tokens)
+        # accumulative score policy (the "H2O + Shared Cache" variant of the Baselines section): a retained state's
+        # importance is the sum of what it received at every eviction step since it entered the cache
+        self.accumulate = accumulate
         self.tokens_seen = 0
         n_caches = 2 if mode == INDIVIDUAL else 1
         self.caches = [CacheState(np.zeros((kv_heads, 0, head_dim)),
@@ -234,8 +239,14 @@ class CitrusOracle:
             scores[0] = s_lm
             scores[1] = importance_sum(Qi, self.caches[1].K, Kc)
 
+        if self.accumulate:
+            for cid in list(scores):
+                prev = self.caches[cid].acc
+                carried = np.zeros((self.Hkv, m)) if prev is None else prev
+                scores[cid] = scores[cid] + np.concatenate([carried, np.zeros((self.Hkv, L))], axis=1)
         res = StepResult(out=out, scores=scores, idx={}, applied={}, m_before=m)
         for cid, S in scores.items():
+            S_total = S
             if self.layerwise:
                 # one score vector for the whole layer (paper's stated granularity):
                 # heads are aggregated before the top-k.
@@ -256,7 +267,8 @@ class CitrusOracle:
             for g in range(self.Hkv):
                 kk, vv, pp = compact(c.K[g], c.V[g], c.pos[g], Kc[:, g, :], Vc[:, g, :], chunk_pos, use[g])
                 newK.append(kk); newV.append(vv); newP.append(pp)
-            self.caches[cid] = CacheState(np.stack(newK), np.stack(newV), np.stack(newP))
+            new_acc = np.stack([S_total[g][use[g]] for g in range(self.Hkv)]) if self.accumulate else None
+            self.caches[cid] = CacheState(np.stack(newK), np.stack(newV), np.stack(newP), new_acc)
         self.tokens_seen += L
         return res
 

@@ -20,6 +20,7 @@ MODE_INDIVIDUAL = 1
 MODE_FP32 = 2
 MODE_LAYERWISE = 4
 MODE_STANDARD = 8
+MODE_ACCUMULATE = 0x20000000
 MAX_INSTR = 4096
 MAX_CANDIDATES = 49152
 
@@ -116,13 +117,14 @@ class Citrus:
     """One eviction context (all layers and sequence slots of one geometry)."""
 
     def __init__(self, layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, mode="shared", dtype="bf16",
-                 lm_window=0, layerwise=False, n_seqs=1, start_size=0):
+                 lm_window=0, layerwise=False, n_seqs=1, start_size=0, accumulate=False):
         lib = load()
         bits = {"individual": MODE_INDIVIDUAL, "standard": MODE_STANDARD}.get(mode, MODE_SHARED)
         bits |= MODE_FP32 if dtype == "fp32" else 0
         bits |= MODE_LAYERWISE if layerwise else 0
         bits |= (int(lm_window) & 0xFFFF) << 8
         bits |= (int(start_size) & 0xF) << 24
+        bits |= MODE_ACCUMULATE if accumulate else 0
         self._h = C.c_void_p()
         rc = lib.citrus_create(C.byref(self._h), layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, bits)
         if rc != 0:

@@ -18,6 +18,7 @@ struct CacheBufs {
     void* K[2] = {nullptr, nullptr};
     void* V[2] = {nullptr, nullptr};
     int* pos[2] = {nullptr, nullptr};
+    float* carried[2] = {nullptr, nullptr};      // accumulative policy: importance carried by the rows
     int cur = 0;
 };
 
@@ -42,6 +43,7 @@ struct citrus_ctx {
     bool individual = false, standard = false, fp32 = false, layerwise = false, use_tc = false;
     int lm_window = 0;
     int start_size = 0;             // initial tokens that are never evicted
+    bool accumulate = false;        // scores carried across steps
     int elt = 2;
     int n_caches = 1;
     int n_slots = 1;
@@ -103,6 +105,8 @@ int alloc_units(citrus_ctx* c) {
                 if ((rc = dev_alloc(c, &u.cache[ci].K[b], kv_bytes, true))) return rc;
                 if ((rc = dev_alloc(c, &u.cache[ci].V[b], kv_bytes, true))) return rc;
                 if ((rc = dev_alloc(c, (void**)&u.cache[ci].pos[b], (size_t)c->Hkv * c->k * sizeof(int), true))) return rc;
+                if (c->accumulate &&
+                    (rc = dev_alloc(c, (void**)&u.cache[ci].carried[b], (size_t)c->Hkv * c->k * sizeof(float), true))) return rc;
             }
         if ((rc = dev_alloc(c, (void**)&u.scores, (size_t)c->n_caches * c->Hkv * c->score_stride * sizeof(float), true))) return rc;
         if ((rc = dev_alloc(c, (void**)&u.idx, (size_t)c->n_caches * c->Hkv * c->k * sizeof(int), true))) return rc;
@@ -218,9 +222,12 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     for (int ci = 0; ci < c->n_caches; ++ci) {
         CacheBufs& cb = u.cache[ci];
         int* idx = u.idx + (size_t)ci * c->Hkv * c->k;
-        sj[ci] = SelectJob{scores[ci], idx, c->score_stride, cb.pos[cb.cur], c->k, m, (int)u.tokens_seen, c->start_size};
+        sj[ci] = SelectJob{scores[ci], idx, c->score_stride, cb.pos[cb.cur], c->k, m, (int)u.tokens_seen, c->start_size,
+                           c->accumulate ? cb.carried[cb.cur] : nullptr};
         cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
-                            cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, m};
+                            cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, m,
+                            c->accumulate ? scores[ci] : nullptr, c->score_stride,
+                            c->accumulate ? cb.carried[cb.cur ^ 1] : nullptr};
     }
     // Small steps (a few MB to move) are latency-bound: one cluster launch does a3 and a4.  Large steps want every
     // SM streaming rows, which the clusters (idle while their first CTA selects) cannot give: two launches.
@@ -266,7 +273,7 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     if (out == nullptr) return CITRUS_ERR_INVALID_ARG;
     *out = nullptr;
     if (layers < 1 || q_heads < 1 || kv_heads < 1 || budget_k < 1 || chunk_s < 1) return CITRUS_ERR_INVALID_ARG;
-    if (mode & ~(0xFu | 0xFFFF00u | 0xF000000u)) return CITRUS_ERR_INVALID_ARG;
+    if (mode & ~(0xFu | 0xFFFF00u | 0xF000000u | CITRUS_MODE_ACCUMULATE)) return CITRUS_ERR_INVALID_ARG;
     if ((mode & CITRUS_MODE_STANDARD) && (mode & CITRUS_MODE_INDIVIDUAL)) return CITRUS_ERR_INVALID_ARG;
     if (q_heads % kv_heads != 0) return CITRUS_ERR_SHAPE;
     if (head_dim != 64 && head_dim != 128) return CITRUS_ERR_UNSUPPORTED;
@@ -285,6 +292,7 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     c->layerwise = (mode & CITRUS_MODE_LAYERWISE) != 0;
     c->lm_window = (int)((mode >> 8) & 0xFFFFu);
     c->start_size = (int)((mode >> 24) & 0xFu);
+    c->accumulate = (mode & CITRUS_MODE_ACCUMULATE) != 0;
     c->elt = fp32 ? 4 : 2;
     c->n_caches = c->individual ? 2 : 1;
     c->score_stride = (budget_k + chunk_s + 3) & ~3;

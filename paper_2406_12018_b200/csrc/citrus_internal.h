@@ -73,12 +73,14 @@ cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse_
 
 // ---- select (a3) and compaction (a4) ---------------------------------------
 struct SelectJob {            // one per cache handled by the launch
-    const float* scores;      // [kv_heads, score_stride]
+    float* scores;            // [kv_heads, score_stride]; with `carried` set, rewritten as score + carried
     int* idx;                 // [kv_heads, budget_k]
     int score_stride;
     // forced keeps ("start size"): candidates whose original position is below `start` are always selected
     const int* pos;           // positions of the old cache rows [kv_heads, pos_stride]
     int pos_stride, m, chunk_pos0, start;
+    // accumulative policy: importance carried by the old cache rows [kv_heads, pos_stride], or null
+    const float* carried;
 };
 // n candidates, keep min(k, n); layerwise: sum scores over heads first and give every head the same set.
 cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, int k, int layerwise, cudaStream_t s);
@@ -88,6 +90,8 @@ struct CompactJob {
     void* dstK; void* dstV; int* dstPos;                      // new cache buffers
     const int* idx;                                           // [kv_heads, budget_k]
     int m;                                                    // rows in the old cache
+    // accumulative policy: the kept candidates' accumulated scores become the new cache's carried importance
+    const float* totals; int score_stride; float* dstCarried;  // null when the policy is off
 };
 cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
                        int kv_heads, int cap, int row_bytes, int kept, int chunk_pos0, cudaStream_t s);

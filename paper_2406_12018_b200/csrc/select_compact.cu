@@ -54,12 +54,23 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         return;
     }
     for (int j = tid; j < n; j += kSelThreads) {
+        // one head's score of candidate j; with the accumulative policy the importance its cache row carries is
+        // added and the sum written back (it is what the compaction hands on, and what the step view shows)
+        auto head_score = [&](int gg) {
+            float* p = job.scores + (size_t)gg * job.score_stride + j;
+            float x = *p;
+            if (job.carried != nullptr) {
+                if (j < job.m) x += job.carried[(size_t)gg * job.pos_stride + j];
+                *p = x;
+            }
+            return x;
+        };
         float v;
         if (layerwise) {
             v = 0.f;
-            for (int gg = 0; gg < kv_heads; ++gg) v += job.scores[(size_t)gg * job.score_stride + j];
+            for (int gg = 0; gg < kv_heads; ++gg) v += head_score(gg);
         } else {
-            v = job.scores[(size_t)g * job.score_stride + j];
+            v = head_score(g);
         }
         uint32_t key = order_key(v);
         if (job.start > 0) {
@@ -241,7 +252,10 @@ __device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4*
             size_t doff = ((size_t)g * cap + r) * row_vecs + v;
             dstK[doff] = a[u];
             dstV[doff] = b[u];
-            if (v == 0) job.dstPos[(size_t)g * cap + r] = j[u] < job.m ? job.srcPos[(size_t)g * cap + j[u]] : chunk_pos0 + (j[u] - job.m);
+            if (v == 0) {
+                job.dstPos[(size_t)g * cap + r] = j[u] < job.m ? job.srcPos[(size_t)g * cap + j[u]] : chunk_pos0 + (j[u] - job.m);
+                if (job.dstCarried != nullptr) job.dstCarried[(size_t)g * cap + r] = job.totals[(size_t)g * job.score_stride + j[u]];
+            }
         }
     }
 }

@@ -47,6 +47,7 @@ class Workload:
     n_seqs: int = 1
     min_tokens: int = 0        # ragged: lengths ~ U{min_tokens..doc_tokens}
     start_size: int = 0        # initial tokens that are never evicted (paper's appendix variant: 4)
+    accumulate: bool = False   # accumulative score policy: importance carried across steps
 
     @property
     def torch_dtype(self):

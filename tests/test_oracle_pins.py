@@ -379,6 +379,48 @@ def test_intersection_ratio_on_a_worked_example_and_its_limits():
         assert r[g] == sum(int(x in set(a[g].tolist())) for x in b[g].tolist()) / 200   # counted one by one
 
 
+def test_accumulated_scores_without_eviction_are_the_sum_of_every_steps_attention():
+    # budget larger than the document: nothing is evicted, so after the last chunk the carried importance of token j
+    # is the attention it received from the instruction at every step it was a candidate, over the prefix seen so far
+    import math
+    rng = np.random.default_rng(21)
+    N, Hq, Hkv, D, ls = 24, 2, 1, 4, 8
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, 3, Hq, D)
+    orc = CitrusOracle(Hq, Hkv, D, 100, SHARED, accumulate=True)
+    for c in range(0, N, ls):
+        orc.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+    expect = [0.0] * N
+    for n_t in range(ls, N + 1, ls):                      # candidates of the step: tokens 0 .. n_t - 1
+        for h in range(Hq):
+            for i in range(Qi.shape[0]):
+                logits = [sum(Qi[i, h, d] * K[j, 0, d] for d in range(D)) / math.sqrt(D) for j in range(n_t)]
+                mx = max(logits)
+                den = sum(math.exp(x - mx) for x in logits)
+                for j in range(n_t):
+                    expect[j] += math.exp(logits[j] - mx) / den
+    assert orc.caches[0].pos[0].tolist() == list(range(N))
+    assert np.allclose(orc.caches[0].acc[0], expect, rtol=1e-12, atol=1e-14)
+
+
+def test_accumulated_scores_change_what_is_kept():
+    # a state that one step rates just below the cut survives when its earlier steps' importance counts
+    rng = np.random.default_rng(22)
+    N, Hq, Hkv, D, k, ls = 96, 2, 1, 8, 12, 16
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, 4, Hq, D)
+    plain, acc = CitrusOracle(Hq, Hkv, D, k, SHARED), CitrusOracle(Hq, Hkv, D, k, SHARED, accumulate=True)
+    differ = False
+    for c in range(0, N, ls):
+        a = plain.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        b = acc.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        # the carried part only ever adds: accumulated scores dominate the step's own
+        m_b = b.m_before
+        assert np.all(b.scores[0][:, m_b:] >= 0) and b.scores[0].shape == (Hkv, m_b + ls)
+        differ |= plain.caches[0].pos[0].tolist() != acc.caches[0].pos[0].tolist()
+        # what is carried forward is exactly the kept candidates' accumulated score
+        assert np.array_equal(acc.caches[0].acc[0], b.scores[0][0][b.applied[0][0]])
+    assert differ
+
+
 def test_forced_selection_is_adopted():
     rng = np.random.default_rng(16)
     N, Hq, Hkv, D, k = 10, 2, 1, 4, 3

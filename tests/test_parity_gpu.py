@@ -92,6 +92,19 @@ def test_start_size_forced_keeps(mode, layerwise):
         Citrus(1, 8, 2, 128, 3, 16, start_size=4)           # more forced keeps than the budget
 
 
+@pytest.mark.parametrize("mode,layerwise,dtype", [("shared", False, "bf16"), ("shared", False, "fp32"),
+                                                   ("individual", False, "bf16"), ("shared", True, "bf16")])
+def test_accumulative_score_policy(mode, layerwise, dtype):
+    # importance carried across steps: scores, kept sets and the carried values follow the oracle chunk after chunk
+    w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=2, head_dim=128, budget_k=200, chunk_s=160, doc_tokens=1300,
+                  n_instr=12, dtype=dtype, mode=mode, lm_window=16, n_planted=4, accumulate=True)
+    ctx = pu.make_pair(w, layerwise=layerwise)
+    _, st = pu.run_document(w, ctx, layerwise=layerwise)
+    _report(f"accumulate {mode} layerwise={layerwise} {dtype}", st)
+    assert st["checked_chunks"] == 9
+    ctx.close()
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_layerwise_granularity(dtype):
     w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=4, head_dim=128, budget_k=96, chunk_s=160, doc_tokens=640,
