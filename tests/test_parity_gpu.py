@@ -221,6 +221,28 @@ def test_config5_long_document_sampled():
     ctx.close()
 
 
+def test_maximum_candidates_and_instruction_rows():
+    # the largest step the library accepts: budget + chunk = 49152 candidates, 4096 instruction queries.  Six full
+    # chunks are property-checked (row counts, ascending positions, rows bit-equal to the document's); the sixth has
+    # the maximal candidate list.  A ragged seventh chunk is compared with the oracle.
+    k, ls = 40960, 8192
+    w = wl.scaled(C["mistral7b_layer"], q_heads=8, kv_heads=2, budget_k=k, chunk_s=ls, doc_tokens=6 * ls + 1000,
+                  n_instr=4096, n_planted=64, n_sinks=2)
+    ctx = pu.make_pair(w)
+    doc, st = pu.run_document(w, ctx, chunk_lengths=[ls] * 6 + [1000], oracle_chunks={6})
+    _report("maximum sizes", st)
+    assert st["checked_chunks"] == 1
+    P = ctx.cache_view(0)[2]
+    assert P.shape[1] == k
+    for g in range(w.kv_heads):
+        kept = set(P[g].tolist())
+        assert set(doc.planted.tolist()) <= kept and set(doc.sinks.tolist()) <= kept
+    assert ctx.poll_status() == 0
+    ctx.close()
+    with pytest.raises(CitrusError):
+        Citrus(1, 8, 2, 128, k, ls + 1)                      # one candidate too many
+
+
 def test_ragged_batch_call_matches_per_sequence_calls_and_rejects_bad_batches():
     # three sequences of the serving mix advance in lock step through the packed call; finished ones drop out
     w = wl.scaled(C["serving_mix"], n_seqs=3, budget_k=256, chunk_s=256, n_instr=24, doc_tokens=1024, min_tokens=300)
