@@ -180,7 +180,8 @@ class StepResult:
     idx: Dict[int, np.ndarray]                        # cache id -> [H_kv, kept] the oracle's own choice
     applied: Dict[int, np.ndarray]                    # cache id -> indices actually applied
     gap: Dict[int, list] = field(default_factory=dict)  # cache id -> per head (kth, k+1th)
-    m_before: int = 0
+    m_before: int = 0                                  # rows of cache 0 before the step
+    m_by_cache: Dict[int, int] = field(default_factory=dict)   # rows of every cache before the step
 
 
 class CitrusOracle:
@@ -197,7 +198,7 @@ class CitrusOracle:
 
     def __init__(self, q_heads, kv_heads, head_dim, budget_k, mode=SHARED,
                  lm_window: Optional[int] = None, layerwise: bool = False, start_size: int = 0,
-                 accumulate: bool = False):
+                 accumulate: bool = False, deferred_lm: bool = False):
         assert q_heads % kv_heads == 0
         self.Hq, self.Hkv, self.D, self.k = q_heads, kv_heads, head_dim, budget_k
         self.mode = mode
@@ -207,6 +208,12 @@ class CitrusOracle:
         # accumulative score policy (the "H2O + Shared Cache" variant of the Baselines section): a retained state's
         # importance is the sum of what it received at every eviction step since it entered the cache
         self.accumulate = accumulate
+        # Standard CSE exactly as Section 4.1 orders it (individual and standard modes): the language-modelling cache
+        # C holds k states plus the previous chunk; the current chunk is encoded against all of them, its attention
+        # evicts C down to k, then ALL of the chunk's states are put in.  Without the flag the chunk's own states
+        # compete for the k places at once.
+        self.deferred_lm = deferred_lm
+        assert not deferred_lm or mode in (INDIVIDUAL, STANDARD)
         self.tokens_seen = 0
         n_caches = 2 if mode == INDIVIDUAL else 1
         self.caches = [CacheState(np.zeros((kv_heads, 0, head_dim)),
@@ -239,14 +246,22 @@ class CitrusOracle:
             scores[0] = s_lm
             scores[1] = importance_sum(Qi, self.caches[1].K, Kc)
 
+        rows = {cid: self.caches[cid].K.shape[1] for cid in scores}
+        lm_scored = self.mode == INDIVIDUAL or (self.mode == STANDARD and Qi is None)   # cache 0 scored by the chunk
         if self.accumulate:
             for cid in list(scores):
                 prev = self.caches[cid].acc
-                carried = np.zeros((self.Hkv, m)) if prev is None else prev
+                carried = np.zeros((self.Hkv, rows[cid])) if prev is None else prev
                 scores[cid] = scores[cid] + np.concatenate([carried, np.zeros((self.Hkv, L))], axis=1)
-        res = StepResult(out=out, scores=scores, idx={}, applied={}, m_before=m)
+        res = StepResult(out=out, scores=scores, idx={}, applied={}, m_before=m, m_by_cache=rows)
         for cid, S in scores.items():
             S_total = S
+            budget = self.k
+            if self.deferred_lm and cid == 0 and lm_scored:
+                # only C's own rows are candidates for eviction; the chunk's states all enter
+                S = S.copy()
+                S[:, m:] = np.inf
+                budget = min(m, self.k) + L
             if self.layerwise:
                 # one score vector for the whole layer (paper's stated granularity):
                 # heads are aggregated before the top-k.
@@ -257,9 +272,9 @@ class CitrusOracle:
                 for g in range(self.Hkv):
                     cand_pos = np.concatenate([self.caches[cid].pos[g], chunk_pos])
                     S[g][cand_pos < self.start_size] = np.inf
-            own = np.stack([select_topk(S[g], self.k) for g in range(self.Hkv)])
+            own = np.stack([select_topk(S[g], budget) for g in range(self.Hkv)])
             res.idx[cid] = own
-            res.gap[cid] = [kth_gap(S[g], self.k) for g in range(self.Hkv)]
+            res.gap[cid] = [kth_gap(S[g], budget) for g in range(self.Hkv)]
             use = own if forced is None or cid not in forced else np.asarray(forced[cid], dtype=np.int64)
             res.applied[cid] = use
             c = self.caches[cid]

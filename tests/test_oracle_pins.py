@@ -10,7 +10,7 @@ import pytest
 import torch
 
 import oracle
-from oracle import CitrusOracle, SHARED, INDIVIDUAL
+from oracle import CitrusOracle, SHARED, INDIVIDUAL, STANDARD
 from paper_2406_12018_b200 import workloads as wl
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -419,6 +419,55 @@ def test_accumulated_scores_change_what_is_kept():
         # what is carried forward is exactly the kept candidates' accumulated score
         assert np.array_equal(acc.caches[0].acc[0], b.scores[0][0][b.applied[0][0]])
     assert differ
+
+
+def test_deferred_lm_eviction_follows_the_three_steps_of_standard_cse():
+    # Section 4.1 in plain Python: C starts as the first chunk; for every later chunk s: encode s against [C ; s],
+    # keep the k states of C that s attends to most (summed over s's queries and the group's heads), put all of s in.
+    import math
+    rng = np.random.default_rng(31)
+    N, Hq, Hkv, D, k, ls = 70, 2, 1, 4, 9, 10
+    Q, K, V = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D)
+    orc = CitrusOracle(Hq, Hkv, D, k, STANDARD, deferred_lm=True)
+    cache = []                                            # original positions held by C
+    for c in range(0, N, ls):
+        orc.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], None)
+        chunk = list(range(c, c + ls))
+        if len(cache) > k:
+            score = {j: 0.0 for j in cache}
+            for t in chunk:                               # every query of the chunk, causal over the chunk itself
+                keys = cache + [u for u in chunk if u <= t]
+                for h in range(Hq):
+                    logits = [sum(Q[t, h, d] * K[j, 0, d] for d in range(D)) / math.sqrt(D) for j in keys]
+                    mx = max(logits)
+                    den = sum(math.exp(x - mx) for x in logits)
+                    for j, x in zip(keys, logits):
+                        if j in score:
+                            score[j] += math.exp(x - mx) / den
+            cache = sorted(sorted(cache, key=lambda j: (-score[j], j))[:k])
+        cache = cache + chunk
+        assert orc.caches[0].pos[0].tolist() == cache
+        assert len(cache) == min(c + ls, k + ls)
+
+
+def test_deferred_lm_eviction_with_unit_chunks_is_tova():
+    # Baselines section: TOVA is standard CSE with l_s = 1 - the newest token's attention over the cache (itself
+    # included) drops the one state it attends to least
+    rng = np.random.default_rng(32)
+    N, Hq, Hkv, D, k = 30, 1, 1, 6, 7
+    Q, K, V = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D)
+    orc = CitrusOracle(Hq, Hkv, D, k, STANDARD, deferred_lm=True)
+    held = []
+    for t in range(N):
+        orc.process_chunk(Q[t:t + 1], K[t:t + 1], V[t:t + 1], None)
+        if len(held) > k:
+            keys = held + [t]
+            logits = np.array([Q[t, 0] @ K[j, 0] for j in keys]) / np.sqrt(D)
+            p = np.exp(logits - logits.max()); p /= p.sum()
+            drop = min(range(len(held)), key=lambda i: (p[i], -held[i]))   # least attended; the later position on a tie
+            held = held[:drop] + held[drop + 1:]
+        held = held + [t]
+        assert orc.caches[0].pos[0].tolist() == held
 
 
 def test_forced_selection_is_adopted():
