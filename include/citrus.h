@@ -65,6 +65,16 @@ typedef struct CUstream_st* citrus_stream_t;
                                              own states start at this step's score.  citrus_step_view then shows the
                                              accumulated scores. */
 
+#define CITRUS_MODE_DEFERRED_LM  0x40000000u /* with INDIVIDUAL or STANDARD: standard chunked eviction in the order of
+                                             Section 4.1 - the language-modelling cache C holds budget_k states plus
+                                             the previous chunk (capacity budget_k + chunk_s rows: K, V, positions and
+                                             index lists of cache 0 are that wide); a chunk is encoded against all of
+                                             them, its attention evicts C's own rows down to budget_k, then all of the
+                                             chunk's states enter.  Without the bit the chunk's own states compete for
+                                             the budget_k places in the same step.  A STANDARD call that passes
+                                             instruction queries (the final eviction) evicts [C ; chunk] to budget_k.
+                                             budget_k + 2 chunk_s <= CITRUS_MAX_CANDIDATES. */
+
 #define CITRUS_OK                 0
 #define CITRUS_ERR_INVALID_ARG   -1
 #define CITRUS_ERR_SHAPE         -2
@@ -151,8 +161,9 @@ int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,
 /*
  * Borrowed device pointers into the current cache of (layer, which, seq_slot);
  * which = 0 the language-modelling / shared cache, 1 the instruction cache C^I
- * (individual mode only).  K, V are [kv_heads, budget_k, D] with rows
- * [0, *n_rows) valid; positions [kv_heads, budget_k] int32 are the original
+ * (individual mode only).  K, V are [kv_heads, cap, D] with rows
+ * [0, *n_rows) valid, cap = budget_k (budget_k + chunk_s for cache 0 of a
+ * CITRUS_MODE_DEFERRED_LM context); positions [kv_heads, cap] int32 are the original
  * token positions, strictly ascending per head (the order a position-shift
  * caller needs).  *n_rows = min(budget_k, tokens seen) is host bookkeeping, so
  * the call does not synchronise; the contents are final once the stream work of

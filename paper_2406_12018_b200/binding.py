@@ -21,6 +21,7 @@ MODE_FP32 = 2
 MODE_LAYERWISE = 4
 MODE_STANDARD = 8
 MODE_ACCUMULATE = 0x20000000
+MODE_DEFERRED_LM = 0x40000000
 MAX_INSTR = 4096
 MAX_CANDIDATES = 49152
 
@@ -117,7 +118,7 @@ class Citrus:
     """One eviction context (all layers and sequence slots of one geometry)."""
 
     def __init__(self, layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, mode="shared", dtype="bf16",
-                 lm_window=0, layerwise=False, n_seqs=1, start_size=0, accumulate=False):
+                 lm_window=0, layerwise=False, n_seqs=1, start_size=0, accumulate=False, deferred_lm=False):
         lib = load()
         bits = {"individual": MODE_INDIVIDUAL, "standard": MODE_STANDARD}.get(mode, MODE_SHARED)
         bits |= MODE_FP32 if dtype == "fp32" else 0
@@ -125,6 +126,7 @@ class Citrus:
         bits |= (int(lm_window) & 0xFFFF) << 8
         bits |= (int(start_size) & 0xF) << 24
         bits |= MODE_ACCUMULATE if accumulate else 0
+        bits |= MODE_DEFERRED_LM if deferred_lm else 0
         self._h = C.c_void_p()
         rc = lib.citrus_create(C.byref(self._h), layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, bits)
         if rc != 0:
@@ -133,6 +135,8 @@ class Citrus:
         self.layers, self.q_heads, self.kv_heads, self.head_dim = layers, q_heads, kv_heads, head_dim
         self.budget_k, self.chunk_s = budget_k, chunk_s
         self.individual = mode == "individual"
+        # row capacity of each cache's buffers: with deferred eviction cache 0 also holds the previous chunk
+        self.cap = (budget_k + (chunk_s if deferred_lm else 0), budget_k)
         self.torch_dtype = torch.float32 if dtype == "fp32" else torch.bfloat16
         if n_seqs != 1:
             rc = lib.citrus_set_batch(self._h, n_seqs)
@@ -188,7 +192,7 @@ class Citrus:
         rc = load().citrus_cache_view(self._h, layer, which, slot, C.byref(K), C.byref(V), C.byref(P), C.byref(n))
         if rc != 0:
             raise CitrusError(rc, "citrus_cache_view")
-        H, k, D = self.kv_heads, self.budget_k, self.head_dim
+        H, k, D = self.kv_heads, self.cap[which], self.head_dim
         if self.torch_dtype == torch.float32:
             Kt, Vt = (_view(p.value, (H, k, D), "<f4", 4) for p in (K, V))
         else:
@@ -213,7 +217,7 @@ class Citrus:
         if rc != 0:
             raise CitrusError(rc, "citrus_step_view")
         St = _view(S.value, (self.kv_heads, stride.value), "<f4", 4)[:, :n.value]
-        It = _view(I.value, (self.kv_heads, self.budget_k), "<i4", 4)[:, :kept.value]
+        It = _view(I.value, (self.kv_heads, self.cap[which]), "<i4", 4)[:, :kept.value]
         return St, It, m.value
 
     def profile(self, enable: bool):

@@ -25,13 +25,13 @@ struct CacheBufs {
 struct Unit {                       // one (layer, sequence slot)
     CacheBufs cache[2];
     float* scores = nullptr;        // [n_caches, kv_heads, score_stride]
-    int* idx = nullptr;             // [n_caches, kv_heads, budget_k]
+    int* idx[2] = {nullptr, nullptr};   // per cache [kv_heads, cap]
     float* lse_chunk = nullptr;     // [q_heads, chunk_s]
     float* lse_instr = nullptr;     // [q_heads, CITRUS_MAX_INSTR]
     float* part = nullptr;          // key-split (max, sum) pairs of a2 pass 1 [splits, q_heads, CITRUS_MAX_INSTR] (tensor-core path)
-    int m = 0;                      // rows retained in every cache
+    int m[2] = {0, 0};              // rows retained in each cache
     long long tokens_seen = 0;
-    int last_n = 0, last_kept = 0, last_m = 0;
+    int last_n[2] = {0, 0}, last_kept[2] = {0, 0}, last_m[2] = {0, 0};
     bool has_step = false;
 };
 
@@ -44,6 +44,8 @@ struct citrus_ctx {
     int lm_window = 0;
     int start_size = 0;             // initial tokens that are never evicted
     bool accumulate = false;        // scores carried across steps
+    bool deferred = false;          // cache 0 holds k states + the previous chunk and is evicted by the next chunk
+    int cap[2] = {0, 0};            // row capacity of each cache's buffers
     int elt = 2;
     int n_caches = 1;
     int n_slots = 1;
@@ -96,20 +98,21 @@ void free_all(citrus_ctx* c) {
 
 int alloc_units(citrus_ctx* c) {
     const size_t row = (size_t)c->D * c->elt;
-    const size_t kv_bytes = (size_t)c->Hkv * c->k * row;
     c->units.assign((size_t)c->layers * c->n_slots, Unit());
     for (Unit& u : c->units) {
         int rc;
-        for (int ci = 0; ci < c->n_caches; ++ci)
+        for (int ci = 0; ci < c->n_caches; ++ci) {
+            const size_t kv_bytes = (size_t)c->Hkv * c->cap[ci] * row;
             for (int b = 0; b < 2; ++b) {
                 if ((rc = dev_alloc(c, &u.cache[ci].K[b], kv_bytes, true))) return rc;
                 if ((rc = dev_alloc(c, &u.cache[ci].V[b], kv_bytes, true))) return rc;
-                if ((rc = dev_alloc(c, (void**)&u.cache[ci].pos[b], (size_t)c->Hkv * c->k * sizeof(int), true))) return rc;
+                if ((rc = dev_alloc(c, (void**)&u.cache[ci].pos[b], (size_t)c->Hkv * c->cap[ci] * sizeof(int), true))) return rc;
                 if (c->accumulate &&
-                    (rc = dev_alloc(c, (void**)&u.cache[ci].carried[b], (size_t)c->Hkv * c->k * sizeof(float), true))) return rc;
+                    (rc = dev_alloc(c, (void**)&u.cache[ci].carried[b], (size_t)c->Hkv * c->cap[ci] * sizeof(float), true))) return rc;
             }
+            if ((rc = dev_alloc(c, (void**)&u.idx[ci], (size_t)c->Hkv * c->cap[ci] * sizeof(int), true))) return rc;
+        }
         if ((rc = dev_alloc(c, (void**)&u.scores, (size_t)c->n_caches * c->Hkv * c->score_stride * sizeof(float), true))) return rc;
-        if ((rc = dev_alloc(c, (void**)&u.idx, (size_t)c->n_caches * c->Hkv * c->k * sizeof(int), true))) return rc;
         if ((rc = dev_alloc(c, (void**)&u.lse_chunk, (size_t)c->Hq * c->ls * sizeof(float), true))) return rc;
         if ((rc = dev_alloc(c, (void**)&u.lse_instr, (size_t)c->Hq * CITRUS_MAX_INSTR * sizeof(float), true))) return rc;
         if (c->use_tc && (rc = dev_alloc(c, (void**)&u.part, (size_t)kTcMaxLseSplits * c->Hq * CITRUS_MAX_INSTR * 2 * sizeof(float), true))) return rc;
@@ -159,21 +162,30 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
              const void* Qi, int nI, void* out, cudaStream_t st) {
     c->used = true;
     Unit& u = c->units[(size_t)layer * c->n_slots + slot];
-    const int m = u.m, n = m + L;
-    const int kept = n < c->k ? n : c->k;
     if (u.tokens_seen + L > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
+    const bool lm_scoring = c->individual || (c->standard && nI == 0);   // cache 0 is scored by the chunk's own queries
+    const bool instr_scoring = nI > 0;
 
+    // sizes of each cache's step.  Deferred eviction (cache 0, when the chunk scores it): only the cache's own rows
+    // compete for the k places, all of the chunk's rows enter.
+    int mc[2], nc[2], kept[2], forced_from[2];
     Candidates cand[2];
     for (int ci = 0; ci < c->n_caches; ++ci) {
         const CacheBufs& cb = u.cache[ci];
-        cand[ci] = Candidates{cb.K[cb.cur], cb.V[cb.cur], Kc, Vc, m, L, c->k, c->Hkv};
+        mc[ci] = u.m[ci]; nc[ci] = mc[ci] + L;
+        forced_from[ci] = nc[ci];
+        kept[ci] = nc[ci] < c->k ? nc[ci] : c->k;
+        if (c->deferred && ci == 0 && lm_scoring) {
+            kept[ci] = (mc[ci] < c->k ? mc[ci] : c->k) + L;
+            forced_from[ci] = mc[ci];
+        }
+        cand[ci] = Candidates{cb.K[cb.cur], cb.V[cb.cur], Kc, Vc, mc[ci], L, c->cap[ci], c->Hkv};
     }
+    const int m = mc[0];
     QueryRows q_chunk{Qc, L, c->Hq, 1, 0};
     QueryRows q_instr{Qi, nI, c->Hq, 0, 0};
     float* scores[2] = {u.scores, u.scores + (size_t)c->Hkv * c->score_stride};
     const int ic = c->individual ? 1 : 0;     // the cache scored by the instruction text
-    const bool lm_scoring = c->individual || (c->standard && nI == 0);   // cache 0 is scored by the chunk's own queries
-    const bool instr_scoring = nI > 0;
     if (!instr_scoring) q_instr.rows = 0;
 
     cudaError_t e;
@@ -181,7 +193,7 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     int splits = 1;
     if (c->use_tc) {
         // a1 and pass 1 of a2-I (row log-sum-exp of the instruction queries, possibly split over key ranges): one launch
-        if (instr_scoring) splits = tc_lse_splits(nI, c->Hq, c->Hkv, m, L, ((L + 127) / 128) * c->Hq);
+        if (instr_scoring) splits = tc_lse_splits(nI, c->Hq, c->Hkv, mc[ic], L, ((L + 127) / 128) * c->Hq);
         LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
         e = tc_attention_lse(q_chunk, cand[0], out, lse_chunk, c->ls, q_instr, cand[ic], u.lse_instr, u.part,
                              CITRUS_MAX_INSTR, splits, c->status, st);
@@ -219,40 +231,45 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     // a3 + a4 for every cache
     SelectJob sj[2];
     CompactJob cj[2];
+    size_t gather_bytes = 0;
     for (int ci = 0; ci < c->n_caches; ++ci) {
         CacheBufs& cb = u.cache[ci];
-        int* idx = u.idx + (size_t)ci * c->Hkv * c->k;
-        sj[ci] = SelectJob{scores[ci], idx, c->score_stride, cb.pos[cb.cur], c->k, m, (int)u.tokens_seen, c->start_size,
-                           c->accumulate ? cb.carried[cb.cur] : nullptr};
+        int* idx = u.idx[ci];
+        sj[ci] = SelectJob{scores[ci], idx, c->score_stride, cb.pos[cb.cur], c->cap[ci], mc[ci], (int)u.tokens_seen,
+                           c->start_size, c->accumulate ? cb.carried[cb.cur] : nullptr,
+                           nc[ci], kept[ci], c->cap[ci], forced_from[ci]};
         cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
-                            cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, m,
+                            cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, mc[ci],
                             c->accumulate ? scores[ci] : nullptr, c->score_stride,
-                            c->accumulate ? cb.carried[cb.cur ^ 1] : nullptr};
+                            c->accumulate ? cb.carried[cb.cur ^ 1] : nullptr, c->cap[ci], kept[ci]};
+        gather_bytes += (size_t)c->Hkv * kept[ci] * c->D * c->elt * 2;
     }
     // Small steps (a few MB to move) are latency-bound: one cluster launch does a3 and a4.  Large steps want every
     // SM streaming rows, which the clusters (idle while their first CTA selects) cannot give: two launches.
-    const size_t gather_bytes = (size_t)c->n_caches * c->Hkv * kept * c->D * c->elt * 2;
     if (!c->layerwise && gather_bytes <= ((size_t)8 << 20)) {
         // one cluster launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-        e = select_compact(sj, cj, c->n_caches, Kc, Vc, c->Hkv, n, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
+        e = select_compact(sj, cj, c->n_caches, Kc, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen, st);
         if (e != cudaSuccess) return cuda_rc(e);
     } else {
         {
             LaunchTimer t(c, CITRUS_KERNEL_SELECT, st);
-            e = select_topk(sj, c->n_caches, c->Hkv, n, c->k, c->layerwise ? 1 : 0, st);
+            e = select_topk(sj, c->n_caches, c->Hkv, c->layerwise ? 1 : 0, st);
         }
         if (e != cudaSuccess) return cuda_rc(e);
         {
             LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-            e = compact_kv(cj, c->n_caches, Kc, Vc, c->Hkv, c->k, c->D * c->elt, kept, (int)u.tokens_seen, st);
+            e = compact_kv(cj, c->n_caches, Kc, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen, st);
         }
         if (e != cudaSuccess) return cuda_rc(e);
     }
 
-    for (int ci = 0; ci < c->n_caches; ++ci) u.cache[ci].cur ^= 1;
-    u.last_n = n; u.last_kept = kept; u.last_m = m; u.has_step = true;
-    u.m = kept;
+    for (int ci = 0; ci < c->n_caches; ++ci) {
+        u.cache[ci].cur ^= 1;
+        u.last_n[ci] = nc[ci]; u.last_kept[ci] = kept[ci]; u.last_m[ci] = mc[ci];
+        u.m[ci] = kept[ci];
+    }
+    u.has_step = true;
     u.tokens_seen += L;
     return CITRUS_OK;
 }
@@ -273,13 +290,14 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     if (out == nullptr) return CITRUS_ERR_INVALID_ARG;
     *out = nullptr;
     if (layers < 1 || q_heads < 1 || kv_heads < 1 || budget_k < 1 || chunk_s < 1) return CITRUS_ERR_INVALID_ARG;
-    if (mode & ~(0xFu | 0xFFFF00u | 0xF000000u | CITRUS_MODE_ACCUMULATE)) return CITRUS_ERR_INVALID_ARG;
+    if (mode & ~(0xFu | 0xFFFF00u | 0xF000000u | CITRUS_MODE_ACCUMULATE | CITRUS_MODE_DEFERRED_LM)) return CITRUS_ERR_INVALID_ARG;
+    if ((mode & CITRUS_MODE_DEFERRED_LM) && !(mode & (CITRUS_MODE_INDIVIDUAL | CITRUS_MODE_STANDARD))) return CITRUS_ERR_INVALID_ARG;
     if ((mode & CITRUS_MODE_STANDARD) && (mode & CITRUS_MODE_INDIVIDUAL)) return CITRUS_ERR_INVALID_ARG;
     if (q_heads % kv_heads != 0) return CITRUS_ERR_SHAPE;
     if (head_dim != 64 && head_dim != 128) return CITRUS_ERR_UNSUPPORTED;
     const bool fp32 = (mode & CITRUS_MODE_FP32) != 0;
     if (!fp32 && head_dim != 128) return CITRUS_ERR_UNSUPPORTED;
-    if ((long long)budget_k + chunk_s > CITRUS_MAX_CANDIDATES) return CITRUS_ERR_UNSUPPORTED;
+    if ((long long)budget_k + chunk_s + ((mode & CITRUS_MODE_DEFERRED_LM) ? chunk_s : 0) > CITRUS_MAX_CANDIDATES) return CITRUS_ERR_UNSUPPORTED;
     if ((int)((mode >> 24) & 0xFu) > budget_k) return CITRUS_ERR_SHAPE;
 
     citrus_ctx* c = new (std::nothrow) citrus_ctx();
@@ -293,9 +311,12 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     c->lm_window = (int)((mode >> 8) & 0xFFFFu);
     c->start_size = (int)((mode >> 24) & 0xFu);
     c->accumulate = (mode & CITRUS_MODE_ACCUMULATE) != 0;
+    c->deferred = (mode & CITRUS_MODE_DEFERRED_LM) != 0;
+    c->cap[0] = budget_k + (c->deferred ? chunk_s : 0);
+    c->cap[1] = budget_k;
     c->elt = fp32 ? 4 : 2;
     c->n_caches = c->individual ? 2 : 1;
-    c->score_stride = (budget_k + chunk_s + 3) & ~3;
+    c->score_stride = (c->cap[0] + chunk_s + 3) & ~3;
     c->use_tc = !fp32 && head_dim == 128;
     if (c->use_tc) {
         const char* dbg = std::getenv("CITRUS_DEBUG_SIMT");
@@ -336,8 +357,8 @@ int citrus_set_batch(citrus_handle h, int n_seq) {
 int citrus_reset(citrus_handle h) {
     if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
     for (Unit& u : h->units) {
-        u.m = 0; u.tokens_seen = 0; u.has_step = false;
-        u.last_n = u.last_kept = u.last_m = 0;
+        u.tokens_seen = 0; u.has_step = false;
+        for (int ci = 0; ci < 2; ++ci) u.m[ci] = u.last_n[ci] = u.last_kept[ci] = u.last_m[ci] = 0;
     }
     return CITRUS_OK;
 }
@@ -425,7 +446,7 @@ int citrus_cache_view(citrus_handle h, int layer, int which, int seq_slot,
     if (K) *K = cb.K[cb.cur];
     if (V) *V = cb.V[cb.cur];
     if (positions) *positions = cb.pos[cb.cur];
-    if (n_rows) *n_rows = u.m;
+    if (n_rows) *n_rows = u.m[which];
     return CITRUS_OK;
 }
 
@@ -435,10 +456,10 @@ int citrus_intersection_ratio(citrus_handle h, int layer, int seq_slot, float* r
     if (seq_slot < 0 || seq_slot >= h->n_slots) return CITRUS_ERR_INVALID_ARG;
     if (!h->individual || h->units.empty()) return CITRUS_ERR_STATE;
     const Unit& u = h->units[(size_t)layer * h->n_slots + seq_slot];
-    if (u.m < 1) return CITRUS_ERR_STATE;
+    if (u.m[0] < 1 || u.m[1] < 1) return CITRUS_ERR_STATE;
     const CacheBufs &lm = u.cache[0], &in = u.cache[1];
-    return cuda_rc(intersection_ratio(lm.pos[lm.cur], in.pos[in.cur], h->k, u.m, h->Hkv, ratio_dev,
-                                      reinterpret_cast<cudaStream_t>(stream)));
+    return cuda_rc(intersection_ratio(lm.pos[lm.cur], h->cap[0], u.m[0], in.pos[in.cur], h->cap[1], u.m[1], h->Hkv,
+                                      ratio_dev, reinterpret_cast<cudaStream_t>(stream)));
 }
 
 int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
@@ -452,10 +473,10 @@ int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
     if (!u.has_step) return CITRUS_ERR_STATE;
     if (scores) *scores = u.scores + (size_t)which * h->Hkv * h->score_stride;
     if (score_stride) *score_stride = h->score_stride;
-    if (idx) *idx = u.idx + (size_t)which * h->Hkv * h->k;
-    if (n_candidates) *n_candidates = u.last_n;
-    if (n_kept) *n_kept = u.last_kept;
-    if (m_before) *m_before = u.last_m;
+    if (idx) *idx = u.idx[which];
+    if (n_candidates) *n_candidates = u.last_n[which];
+    if (n_kept) *n_kept = u.last_kept[which];
+    if (m_before) *m_before = u.last_m[which];
     return CITRUS_OK;
 }
 

@@ -81,9 +81,12 @@ struct SelectJob {            // one per cache handled by the launch
     int pos_stride, m, chunk_pos0, start;
     // accumulative policy: importance carried by the old cache rows [kv_heads, pos_stride], or null
     const float* carried;
+    // sizes of this cache's step: n candidates, keep min(k, n); idx rows are idx_stride apart; candidates
+    // j >= forced_from always stay (deferred eviction: the chunk's own states), n when there are none
+    int n, k, idx_stride, forced_from;
 };
-// n candidates, keep min(k, n); layerwise: sum scores over heads first and give every head the same set.
-cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, int k, int layerwise, cudaStream_t s);
+// layerwise: sum scores over heads first and give every head the same set.
+cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int layerwise, cudaStream_t s);
 
 struct CompactJob {
     const void* srcK; const void* srcV; const int* srcPos;   // old cache buffers
@@ -92,13 +95,15 @@ struct CompactJob {
     int m;                                                    // rows in the old cache
     // accumulative policy: the kept candidates' accumulated scores become the new cache's carried importance
     const float* totals; int score_stride; float* dstCarried;  // null when the policy is off
+    int cap;                                                  // row capacity of this cache's buffers (old and new)
+    int kept;                                                 // rows of the new cache
 };
 cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
-                       int kv_heads, int cap, int row_bytes, int kept, int chunk_pos0, cudaStream_t s);
+                       int kv_heads, int row_bytes, int chunk_pos0, cudaStream_t s);
 // a3 + a4 in one launch (per-head granularity): clusters of CTAs per (cache, KV head).
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
-                           int kv_heads, int n, int k, int row_bytes, int kept, int chunk_pos0, cudaStream_t s);
-// ratio[g] = |{positions of a} intersect {positions of b}| / rows over two ascending position lists per head
-cudaError_t intersection_ratio(const int* pos_a, const int* pos_b, int pos_stride, int rows, int kv_heads, float* ratio,
-                               cudaStream_t s);
+                           int kv_heads, int row_bytes, int chunk_pos0, cudaStream_t s);
+// ratio[g] = |{positions of a} intersect {positions of b}| / rows_b over two ascending position lists per head
+cudaError_t intersection_ratio(const int* pos_a, int stride_a, int rows_a, const int* pos_b, int stride_b, int rows_b,
+                               int kv_heads, float* ratio, cudaStream_t s);
 }  // namespace citrus

@@ -35,8 +35,9 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 // `also(p, j)` is called for every kept candidate j with its place p in the ascending list (the fused kernel
 // uses it to hand the list to the gathering CTAs through shared memory).
 template <typename Also>
-__device__ __forceinline__ void select_body(const SelectJob& job, const int g, int kv_heads, int n, int k, int layerwise,
+__device__ __forceinline__ void select_body(const SelectJob& job, const int g, int kv_heads, int layerwise,
                                             uint32_t* keys /* shared, [n] */, Also also) {
+    const int n = job.n, k = job.k, ks = job.idx_stride;
     __shared__ uint32_t hist[256];
     __shared__ uint32_t s_prefix, s_remaining, s_bin_count, s_n_short;
     __shared__ uint32_t s_short[32];
@@ -44,11 +45,11 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
 
     const int tid = threadIdx.x;
     const int heads_out = layerwise ? kv_heads : 1;
-    int* idx0 = job.idx + (size_t)g * k;
+    int* idx0 = job.idx + (size_t)g * ks;
 
     if (n <= k) {                                  // nothing to evict: identity
         for (int j = tid; j < n; j += kSelThreads) {
-            for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * k + j] = j;
+            for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * ks + j] = j;
             also(j, j);
         }
         return;
@@ -78,6 +79,7 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
             const int pos = j < job.m ? job.pos[(size_t)(layerwise ? 0 : g) * job.pos_stride + j] : job.chunk_pos0 + (j - job.m);
             if (pos < job.start) key = 0xffffffffu;           // beats every score; ties among them keep index order
         }
+        if (j >= job.forced_from) key = 0xffffffffu;          // the chunk's own states all enter (deferred eviction)
         keys[j] = key;
     }
     if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; s_bin_count = (uint32_t)n; s_n_short = 0u; }
@@ -194,7 +196,7 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         bool keep = key > T || (key == T && eq_before < take_eq);
         if (keep) {
             uint32_t p = gt_before + min(eq_before, take_eq);
-            for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * k + p] = j;
+            for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * ks + p] = j;
             also((int)p, j);
         }
         gt_before += key > T;
@@ -204,17 +206,18 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
 }
 
 __global__ void __launch_bounds__(kSelThreads)
-select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int n, int k, int layerwise) {
-    extern __shared__ uint32_t keys[];            // [n]
+select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int layerwise) {
+    extern __shared__ uint32_t keys[];            // [largest n of the jobs]
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the scores are final after this
-    select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, n, k, layerwise, keys, [](int, int) {});
+    select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, layerwise, keys, [](int, int) {});
 }
 
 // Rows [r_begin, r_end) of one (cache, head) are copied with 128-bit accesses, row_bytes/16 lanes per row.
 __device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4* __restrict__ chunkK,
-                                             const uint4* __restrict__ chunkV, const int g, int kv_heads, int cap,
+                                             const uint4* __restrict__ chunkV, const int g, int kv_heads,
                                              int row_vecs, int r_begin, int r_end, int chunk_pos0, const int* idx) {
+    const int cap = job.cap;
     // idx[r] = candidate kept in row r of this head (global list, or the CTA's slice in shared memory)
     const int rows_per_pass = blockDim.x / row_vecs;
     const int sub = threadIdx.x / row_vecs, v = threadIdx.x % row_vecs;
@@ -266,12 +269,13 @@ constexpr int kCompactRowsPerCta = 64;
 
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
-                  int kv_heads, int cap, int row_vecs, int kept, int chunk_pos0) {
+                  int kv_heads, int row_vecs, int chunk_pos0) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the index lists are final after this
+    const CompactJob& job = args.job[blockIdx.z];
     const int r0 = blockIdx.x * kCompactRowsPerCta;
-    compact_rows(args.job[blockIdx.z], chunkK, chunkV, blockIdx.y, kv_heads, cap, row_vecs,
-                 r0, min(kept, r0 + kCompactRowsPerCta), chunk_pos0, args.job[blockIdx.z].idx + (size_t)blockIdx.y * cap);
+    compact_rows(job, chunkK, chunkV, blockIdx.y, kv_heads, row_vecs,
+                 r0, min(job.kept, r0 + kCompactRowsPerCta), chunk_pos0, job.idx + (size_t)blockIdx.y * job.cap);
 }
 
 // a3 + a4 in one launch: a cluster of kFusedCluster CTAs per (cache, KV head).  The first CTA of the cluster
@@ -283,11 +287,12 @@ constexpr int kFusedCluster = 8;
 
 __global__ void __launch_bounds__(kSelThreads)
 select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_constant__ CompactArgs cmp, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
-                      int kv_heads, int n, int k, int row_vecs, int kept, int chunk_pos0) {
-    extern __shared__ uint32_t keys[];            // [n] order keys (selecting CTA only), then this CTA's slice of the list
+                      int kv_heads, int n_max, int row_vecs, int chunk_pos0) {
+    extern __shared__ uint32_t keys[];            // [n_max] order keys (selecting CTA only), then this CTA's slice of the list
     const int g = blockIdx.y;
+    const int kept = cmp.job[blockIdx.z].kept;
     const int per = (kept + kFusedCluster - 1) / kFusedCluster;
-    int* s_idx = reinterpret_cast<int*>(keys + n);     // [per]
+    int* s_idx = reinterpret_cast<int*>(keys + n_max);     // [per]
     // programmatic dependent launch: let the next kernel start its prologue, then wait for the scores
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     CITRUS_SPAN_MIN(0);
@@ -299,7 +304,7 @@ select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_const
     CITRUS_TR(9);
     if (blockIdx.x == 0) {
         const uint32_t slice = (uint32_t)__cvta_generic_to_shared(s_idx);
-        select_body(sel.job[blockIdx.z], g, kv_heads, n, k, 0, keys, [&](int p, int j) {
+        select_body(sel.job[blockIdx.z], g, kv_heads, 0, keys, [&](int p, int j) {
             uint32_t remote;
             asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(slice + 4u * (uint32_t)(p % per)), "r"(p / per));
             asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(j) : "memory");
@@ -311,7 +316,7 @@ select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_const
     CITRUS_SPAN_MAX(3);
     CITRUS_TR(16);
     const int r0 = blockIdx.x * per;
-    compact_rows(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, k, row_vecs, r0, min(kept, r0 + per), chunk_pos0, s_idx - r0);
+    compact_rows(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, row_vecs, r0, min(kept, r0 + per), chunk_pos0, s_idx - r0);
     CITRUS_SPAN_MAX(2);
     CITRUS_TR(17);
 }
@@ -319,22 +324,23 @@ select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_const
 // One CTA per KV head: thread t looks element t, t + 256, ... of list b up in list a (both strictly ascending) by
 // binary search; the hits are counted with a warp reduction and one shared-memory atomic per warp.
 __global__ void __launch_bounds__(256)
-intersection_kernel(const int* __restrict__ pos_a, const int* __restrict__ pos_b, int pos_stride, int rows, float* __restrict__ ratio) {
+intersection_kernel(const int* __restrict__ pos_a, int stride_a, int rows_a, const int* __restrict__ pos_b, int stride_b, int rows,
+                    float* __restrict__ ratio) {
     __shared__ int hits;
     const int g = blockIdx.x;
-    const int* a = pos_a + (size_t)g * pos_stride;
-    const int* b = pos_b + (size_t)g * pos_stride;
+    const int* a = pos_a + (size_t)g * stride_a;
+    const int* b = pos_b + (size_t)g * stride_b;
     if (threadIdx.x == 0) hits = 0;
     __syncthreads();
     int mine = 0;
     for (int i = threadIdx.x; i < rows; i += blockDim.x) {
         const int x = b[i];
-        int lo = 0, hi = rows;                    // first index with a[idx] >= x
+        int lo = 0, hi = rows_a;                  // first index with a[idx] >= x
         while (lo < hi) {
             const int mid = (lo + hi) >> 1;
             if (a[mid] < x) lo = mid + 1; else hi = mid;
         }
-        mine += lo < rows && a[lo] == x;
+        mine += lo < rows_a && a[lo] == x;
     }
     mine = __reduce_add_sync(0xffffffffu, mine);
     if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&hits, mine);
@@ -344,16 +350,17 @@ intersection_kernel(const int* __restrict__ pos_a, const int* __restrict__ pos_b
 
 }  // namespace
 
-cudaError_t intersection_ratio(const int* pos_a, const int* pos_b, int pos_stride, int rows, int kv_heads, float* ratio,
-                               cudaStream_t s) {
-    intersection_kernel<<<kv_heads, 256, 0, s>>>(pos_a, pos_b, pos_stride, rows, ratio);
+cudaError_t intersection_ratio(const int* pos_a, int stride_a, int rows_a, const int* pos_b, int stride_b, int rows_b,
+                               int kv_heads, float* ratio, cudaStream_t s) {
+    intersection_kernel<<<kv_heads, 256, 0, s>>>(pos_a, stride_a, rows_a, pos_b, stride_b, rows_b, ratio);
     return cudaGetLastError();
 }
 
-cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, int k, int layerwise, cudaStream_t s) {
+cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int layerwise, cudaStream_t s) {
     if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
     SelectArgs a;
-    for (int i = 0; i < n_jobs; ++i) a.job[i] = jobs[i];
+    int n = 0;
+    for (int i = 0; i < n_jobs; ++i) { a.job[i] = jobs[i]; n = jobs[i].n > n ? jobs[i].n : n; }
     static bool attr_set = false;
     size_t smem = (size_t)n * sizeof(uint32_t);
     if (!attr_set) {
@@ -371,14 +378,19 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int n, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     before_launch(s);
-    return cudaLaunchKernelEx(&cfg, select_topk_kernel, a, kv_heads, n, k, layerwise);
+    return cudaLaunchKernelEx(&cfg, select_topk_kernel, a, kv_heads, layerwise);
 }
 
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
-                           int kv_heads, int n, int k, int row_bytes, int kept, int chunk_pos0, cudaStream_t s) {
+                           int kv_heads, int row_bytes, int chunk_pos0, cudaStream_t s) {
     if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
     SelectArgs sa; CompactArgs ca;
-    for (int i = 0; i < n_jobs; ++i) { sa.job[i] = sjobs[i]; ca.job[i] = cjobs[i]; }
+    int n = 0, kept = 0;
+    for (int i = 0; i < n_jobs; ++i) {
+        sa.job[i] = sjobs[i]; ca.job[i] = cjobs[i];
+        n = sjobs[i].n > n ? sjobs[i].n : n;
+        kept = cjobs[i].kept > kept ? cjobs[i].kept : kept;
+    }
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -398,14 +410,15 @@ cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int 
     cfg.attrs = attr; cfg.numAttrs = 2;
     before_launch(s);
     return cudaLaunchKernelEx(&cfg, select_compact_kernel, sa, ca, reinterpret_cast<const uint4*>(chunkK),
-                              reinterpret_cast<const uint4*>(chunkV), kv_heads, n, k, row_bytes / 16, kept, chunk_pos0);
+                              reinterpret_cast<const uint4*>(chunkV), kv_heads, n, row_bytes / 16, chunk_pos0);
 }
 
 cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
-                       int kv_heads, int cap, int row_bytes, int kept, int chunk_pos0, cudaStream_t s) {
+                       int kv_heads, int row_bytes, int chunk_pos0, cudaStream_t s) {
     if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
     CompactArgs a;
-    for (int i = 0; i < n_jobs; ++i) a.job[i] = jobs[i];
+    int kept = 0;
+    for (int i = 0; i < n_jobs; ++i) { a.job[i] = jobs[i]; kept = jobs[i].kept > kept ? jobs[i].kept : kept; }
     int row_vecs = row_bytes / 16;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((kept + kCompactRowsPerCta - 1) / kCompactRowsPerCta, kv_heads, n_jobs);
@@ -417,7 +430,7 @@ cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, c
     cfg.attrs = attr; cfg.numAttrs = 1;
     before_launch(s);
     return cudaLaunchKernelEx(&cfg, compact_kv_kernel, a, reinterpret_cast<const uint4*>(chunkK),
-                              reinterpret_cast<const uint4*>(chunkV), kv_heads, cap, row_vecs, kept, chunk_pos0);
+                              reinterpret_cast<const uint4*>(chunkV), kv_heads, row_vecs, chunk_pos0);
 }
 
 }  // namespace citrus

@@ -48,6 +48,7 @@ class Workload:
     min_tokens: int = 0        # ragged: lengths ~ U{min_tokens..doc_tokens}
     start_size: int = 0        # initial tokens that are never evicted (paper's appendix variant: 4)
     accumulate: bool = False   # accumulative score policy: importance carried across steps
+    deferred_lm: bool = False  # language-modelling cache evicted by the next chunk (Section 4.1 order)
 
     @property
     def torch_dtype(self):

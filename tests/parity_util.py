@@ -25,14 +25,14 @@ SWAP_REL = 1e-5
 def make_pair(w: wl.Workload, layers=1, layerwise=False):
     ctx = Citrus(layers, w.q_heads, w.kv_heads, w.head_dim, w.budget_k, w.chunk_s, mode=w.mode, dtype=w.dtype,
                  lm_window=w.lm_window, layerwise=layerwise, n_seqs=w.n_seqs, start_size=w.start_size,
-                 accumulate=w.accumulate)
+                 accumulate=w.accumulate, deferred_lm=w.deferred_lm)
     return ctx
 
 
 def make_oracle(w: wl.Workload, layerwise=False):
     return CitrusOracle(w.q_heads, w.kv_heads, w.head_dim, w.budget_k, w.mode,
                         lm_window=(w.lm_window or None), layerwise=layerwise, start_size=w.start_size,
-                        accumulate=w.accumulate)
+                        accumulate=w.accumulate, deferred_lm=w.deferred_lm)
 
 
 def check_index_rule(own, gpu, scores, n, k):
@@ -66,13 +66,17 @@ def load_oracle_from_library(orc: CitrusOracle, ctx: Citrus, layer: int, slot: i
     orc.tokens_seen = tokens_seen
 
 
-def check_cache_properties(ctx: Citrus, doc: wl.Document, layer: int, slot: int, tokens_seen: int, Kdev, Vdev):
+def check_cache_properties(ctx: Citrus, doc: wl.Document, layer: int, slot: int, tokens_seen: int, Kdev, Vdev,
+                           expected_rows=None):
     """Properties that hold at any size: row count, ascending positions, rows are the
     document's rows at those positions (bit-exact)."""
     n_caches = 2 if ctx.individual else 1
     for cid in range(n_caches):
         K, V, P = ctx.cache_view(layer, cid, slot)
-        assert K.shape[1] == min(ctx.budget_k, tokens_seen)
+        if expected_rows is not None:
+            assert K.shape[1] == expected_rows[cid]
+        else:
+            assert K.shape[1] == min(ctx.budget_k, tokens_seen)
         if P.shape[1] > 1:
             assert bool((P[:, 1:] > P[:, :-1]).all())
         assert int(P.min()) >= 0 and int(P.max()) < tokens_seen
@@ -108,6 +112,7 @@ def run_document(w: wl.Workload, ctx: Citrus, layer=0, slot=0, seq=0, n_tokens=N
     st.setdefault("max_out_err", 0.0); st.setdefault("max_score_err", 0.0)
     st.setdefault("max_score_rel", 0.0); st.setdefault("flips", 0); st.setdefault("checked_chunks", 0)
     tokens_seen = 0
+    rows = [0, 0]            # expected rows of each cache (tracked here only for deferred eviction)
     oracle_synced = True     # oracle's caches equal the library's
     for ci, (a, b) in enumerate(bounds):
         L = b - a
@@ -127,13 +132,13 @@ def run_document(w: wl.Workload, ctx: Citrus, layer=0, slot=0, seq=0, n_tokens=N
             forced = {cid: views[cid][1].cpu().numpy().astype(np.int64) for cid in range(n_caches)}
             res = orc.process_chunk(wl.to_f64(doc.Q[a:b]), wl.to_f64(doc.K[a:b]), wl.to_f64(doc.V[a:b]),
                                     Qi64 if with_instr else None, forced)
-            n = res.m_before + L
             err = float(np.abs(out.to(torch.float64).cpu().numpy() - res.out).max())
             st["max_out_err"] = max(st["max_out_err"], err)
             assert err <= tol, f"chunk {ci}: attention output error {err}"
             for cid in range(n_caches):
                 S_gpu = views[cid][0].to(torch.float64).cpu().numpy()
-                assert views[cid][2] == res.m_before
+                assert views[cid][2] == res.m_by_cache[cid]
+                n = res.m_by_cache[cid] + L
                 S_or = res.scores[cid]
                 if (ctx.individual and cid == 0) or not with_instr:
                     wrows = L if not w.lm_window else min(w.lm_window, L)
@@ -162,5 +167,11 @@ def run_document(w: wl.Workload, ctx: Citrus, layer=0, slot=0, seq=0, n_tokens=N
             st["checked_chunks"] += 1
         else:
             oracle_synced = False
-        check_cache_properties(ctx, doc, layer, slot, tokens_seen, Kd, Vd)
+        expected = None
+        if w.deferred_lm:
+            lm_scored = w.mode == "individual" or not with_instr
+            rows[0] = (min(rows[0], w.budget_k) + L) if lm_scored else min(rows[0] + L, w.budget_k)
+            rows[1] = min(rows[1] + L, w.budget_k)
+            expected = list(rows)
+        check_cache_properties(ctx, doc, layer, slot, tokens_seen, Kd, Vd, expected)
     return doc, st

@@ -105,6 +105,28 @@ def test_accumulative_score_policy(mode, layerwise, dtype):
     ctx.close()
 
 
+@pytest.mark.parametrize("mode,dtype,lm_window", [("standard", "bf16", 0), ("standard", "fp32", 0), ("individual", "bf16", 0),
+                                                   ("individual", "bf16", 24)])
+def test_deferred_eviction_of_the_language_modelling_cache(mode, dtype, lm_window):
+    # Section 4.1 order: cache 0 keeps budget_k states plus the previous chunk; the next chunk's attention evicts them
+    w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=2, head_dim=128, budget_k=200, chunk_s=160, doc_tokens=1100,
+                  n_instr=12, dtype=dtype, mode=mode, lm_window=lm_window, n_planted=4, deferred_lm=True)
+    ctx = pu.make_pair(w)
+    _, st = pu.run_document(w, ctx, chunk_lengths=[160, 160, 160, 97, 160, 160, 160, 43])
+    _report(f"deferred {mode} {dtype} w={lm_window}", st)
+    K0 = ctx.cache_view(0, 0)[0]
+    assert K0.shape[1] == (200 if mode == "standard" else 200 + 43)     # standard: the last call evicts by the instruction
+    if mode == "individual":
+        assert ctx.cache_view(0, 1)[0].shape[1] == 200
+        r = ctx.intersection_ratio(0)
+        assert r.shape == (2,) and 0.0 <= float(r.min()) <= float(r.max()) <= 1.0
+    ctx.close()
+    with pytest.raises(CitrusError):
+        Citrus(1, 8, 2, 128, 200, 160, mode="shared", deferred_lm=True)  # no language-modelling cache to defer
+    with pytest.raises(CitrusError):
+        Citrus(1, 8, 2, 128, 40000, 5000, mode="standard", deferred_lm=True)   # budget + 2 chunks exceeds the limit
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_layerwise_granularity(dtype):
     w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=4, head_dim=128, budget_k=96, chunk_s=160, doc_tokens=640,
