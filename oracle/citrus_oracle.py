@@ -139,6 +139,22 @@ def kth_gap(score: np.ndarray, k: int):
 
 
 # --------------------------------------------------------------------------
+# Position shift (Section "Hyperparameters": positional embeddings follow the place in the cache, not the place in
+# the document).  Rotary embedding in the half-split layout of the Llama / Mistral backbones: element d pairs with
+# element d + D/2 and the pair turns by pos * base^(-2d/D).
+# --------------------------------------------------------------------------
+def rope(x: np.ndarray, pos: np.ndarray, base: float = 10000.0) -> np.ndarray:
+    """x [..., D]; pos broadcastable to x.shape[:-1]."""
+    D = x.shape[-1]
+    half = D // 2
+    theta = base ** (-2.0 * np.arange(half, dtype=np.float64) / D)
+    ang = np.asarray(pos, dtype=np.float64)[..., None] * theta
+    c, s_ = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s_, x2 * c + x1 * s_], axis=-1)
+
+
+# --------------------------------------------------------------------------
 # Diagnostic of the appendix "Details for the Intersection Probing Experiments":
 # |C_context  intersect  C_instruction| / |C_instruction| for two sets of retained states
 # --------------------------------------------------------------------------
@@ -198,7 +214,8 @@ class CitrusOracle:
 
     def __init__(self, q_heads, kv_heads, head_dim, budget_k, mode=SHARED,
                  lm_window: Optional[int] = None, layerwise: bool = False, start_size: int = 0,
-                 accumulate: bool = False, deferred_lm: bool = False):
+                 accumulate: bool = False, deferred_lm: bool = False, rope_shift: bool = False,
+                 rope_base: float = 10000.0):
         assert q_heads % kv_heads == 0
         self.Hq, self.Hkv, self.D, self.k = q_heads, kv_heads, head_dim, budget_k
         self.mode = mode
@@ -214,6 +231,12 @@ class CitrusOracle:
         # compete for the k places at once.
         self.deferred_lm = deferred_lm
         assert not deferred_lm or mode in (INDIVIDUAL, STANDARD)
+        # position shift: Q, K and the instruction queries arrive without rotary embedding; every step embeds them by
+        # their place in [cache ; chunk ; instruction] (cache row r -> r, chunk token i -> m + i, instruction token
+        # i -> m + L + i).  The caches keep the un-rotated keys.
+        self.rope_shift = rope_shift
+        self.rope_base = rope_base
+        assert not (rope_shift and deferred_lm)
         self.tokens_seen = 0
         n_caches = 2 if mode == INDIVIDUAL else 1
         self.caches = [CacheState(np.zeros((kv_heads, 0, head_dim)),
@@ -231,20 +254,31 @@ class CitrusOracle:
         m = c0.K.shape[1]
         chunk_pos = self.tokens_seen + np.arange(L, dtype=np.int64)
 
+        raw_Kc = Kc
+        cacheK = {cid: st.K for cid, st in enumerate(self.caches)}
+        if self.rope_shift:
+            b = self.rope_base
+            Qc = rope(Qc, (m + np.arange(L))[:, None], b)
+            Kc = rope(Kc, (m + np.arange(L))[:, None], b)
+            if Qi is not None:
+                Qi = rope(Qi, (m + L + np.arange(Qi.shape[0]))[:, None], b)
+            cacheK = {cid: rope(st.K, np.arange(st.K.shape[1])[None, :], b) for cid, st in enumerate(self.caches)}
+        c0K = cacheK[0]
+
         scores: Dict[int, np.ndarray] = {}
         if self.mode == STANDARD and Qi is None:
             # Eq. 1 with s = the chunk: its last w queries vote on [cache ; chunk]
             w = L if self.lm_window is None else min(self.lm_window, L)
-            out, s_lm = chunk_attention(Qc, c0.K, c0.V, Kc, Vc, lm_window=w)
+            out, s_lm = chunk_attention(Qc, c0K, c0.V, Kc, Vc, lm_window=w)
             scores[0] = s_lm
         elif self.mode in (SHARED, STANDARD):
-            out, _ = chunk_attention(Qc, c0.K, c0.V, Kc, Vc, lm_window=0)
-            scores[0] = importance_sum(Qi, c0.K, Kc)
+            out, _ = chunk_attention(Qc, c0K, c0.V, Kc, Vc, lm_window=0)
+            scores[0] = importance_sum(Qi, c0K, Kc)
         else:
             w = L if self.lm_window is None else min(self.lm_window, L)
-            out, s_lm = chunk_attention(Qc, c0.K, c0.V, Kc, Vc, lm_window=w)
+            out, s_lm = chunk_attention(Qc, c0K, c0.V, Kc, Vc, lm_window=w)
             scores[0] = s_lm
-            scores[1] = importance_sum(Qi, self.caches[1].K, Kc)
+            scores[1] = importance_sum(Qi, cacheK[1], Kc)
 
         rows = {cid: self.caches[cid].K.shape[1] for cid in scores}
         lm_scored = self.mode == INDIVIDUAL or (self.mode == STANDARD and Qi is None)   # cache 0 scored by the chunk
@@ -280,7 +314,7 @@ class CitrusOracle:
             c = self.caches[cid]
             newK, newV, newP = [], [], []
             for g in range(self.Hkv):
-                kk, vv, pp = compact(c.K[g], c.V[g], c.pos[g], Kc[:, g, :], Vc[:, g, :], chunk_pos, use[g])
+                kk, vv, pp = compact(c.K[g], c.V[g], c.pos[g], raw_Kc[:, g, :], Vc[:, g, :], chunk_pos, use[g])
                 newK.append(kk); newV.append(vv); newP.append(pp)
             new_acc = np.stack([S_total[g][use[g]] for g in range(self.Hkv)]) if self.accumulate else None
             self.caches[cid] = CacheState(np.stack(newK), np.stack(newV), np.stack(newP), new_acc)

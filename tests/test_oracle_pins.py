@@ -470,6 +470,66 @@ def test_deferred_lm_eviction_with_unit_chunks_is_tova():
         assert orc.caches[0].pos[0].tolist() == held
 
 
+def test_rope_is_a_rotation_of_complex_pairs_and_depends_on_relative_position_only():
+    from oracle import rope
+    rng = np.random.default_rng(41)
+    D = 16
+    q, k = rng.normal(size=D), rng.normal(size=D)
+    theta = 10000.0 ** (-2.0 * np.arange(D // 2) / D)
+    for a, b in [(0, 0), (3, 3), (5, 2), (1000, 977), (7, 40)]:
+        # complex form: pair (x_d, x_{d+D/2}) is the number x_d + i x_{d+D/2}, turned by exp(i pos theta_d)
+        qa = (q[:D // 2] + 1j * q[D // 2:]) * np.exp(1j * a * theta)
+        kb = (k[:D // 2] + 1j * k[D // 2:]) * np.exp(1j * b * theta)
+        assert np.allclose(rope(q, np.array(a)), np.concatenate([qa.real, qa.imag]), atol=1e-12)
+        dot = float(rope(q, np.array(a)) @ rope(k, np.array(b)))
+        assert abs(dot - float(np.real(np.sum(qa * np.conj(kb))))) < 1e-10
+        assert abs(dot - float(rope(q, np.array(a - b)) @ k)) < 1e-9          # relative position only
+    assert np.allclose(rope(q, np.array(0)), q)
+    assert abs(np.linalg.norm(rope(q, np.array(123))) - np.linalg.norm(q)) < 1e-12
+
+
+def test_position_shift_without_eviction_is_ordinary_rope_by_document_position():
+    # budget larger than the document: every state keeps its place, so cache slot = document position and the shifted
+    # run must equal a plain run on inputs that were embedded up front
+    from oracle import rope
+    rng = np.random.default_rng(42)
+    N, Hq, Hkv, D, ls, nI = 48, 4, 2, 8, 16, 5
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, nI, Hq, D)
+    shifted = CitrusOracle(Hq, Hkv, D, 1000, SHARED, rope_shift=True)
+    plain = CitrusOracle(Hq, Hkv, D, 1000, SHARED)
+    pos = np.arange(N)[:, None]
+    Qr, Kr = rope(Q, pos), rope(K, pos)
+    for c in range(0, N, ls):
+        a = shifted.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        Qir = rope(Qi, (c + ls + np.arange(nI))[:, None])           # the instruction follows what has been read
+        b = plain.process_chunk(Qr[c:c + ls], Kr[c:c + ls], V[c:c + ls], Qir)
+        assert np.allclose(a.out, b.out, atol=1e-12) and np.allclose(a.scores[0], b.scores[0], atol=1e-12)
+    assert np.array_equal(shifted.caches[0].K, np.transpose(K, (1, 0, 2)))     # the cache keeps un-rotated keys
+
+
+def test_position_shift_with_eviction_embeds_by_cache_slot():
+    # after eviction a kept state sits in a lower slot and is embedded by that slot: brute force for one query
+    import math
+    from oracle import rope
+    rng = np.random.default_rng(43)
+    N, Hq, Hkv, D, k, ls = 40, 1, 1, 8, 6, 8
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, 2, Hq, D)
+    orc = CitrusOracle(Hq, Hkv, D, k, SHARED, rope_shift=True)
+    for c in range(0, N, ls):
+        held = orc.caches[0].pos[0].tolist()
+        res = orc.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        m = len(held)
+        t = ls - 1                                            # last token of the chunk sees everything
+        keys = [rope(K[p, 0], np.array(slot)) for slot, p in enumerate(held)] + \
+               [rope(K[c + i, 0], np.array(m + i)) for i in range(ls)]
+        vals = [V[p, 0] for p in held] + [V[c + i, 0] for i in range(ls)]
+        qv = rope(Q[c + t, 0], np.array(m + t))
+        logits = [float(qv @ kk) / math.sqrt(D) for kk in keys]
+        mx = max(logits); w = [math.exp(x - mx) for x in logits]; den = sum(w)
+        expect = sum(wi / den * v for wi, v in zip(w, vals))
+        assert np.allclose(res.out[t, 0], expect, atol=1e-12)
+
+
 def test_forced_selection_is_adopted():
     rng = np.random.default_rng(16)
     N, Hq, Hkv, D, k = 10, 2, 1, 4, 3
