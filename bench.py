@@ -199,7 +199,7 @@ def run_ours(args, rank, world, local_rank):
     Q, K, V, Qi = doc.Q.cuda(), doc.K.cuda(), doc.V.cuda(), doc.Q_instr.cuda()
     out = torch.empty_like(Q)
     ctx = Citrus(1, w.q_heads, w.kv_heads, w.head_dim, w.budget_k, w.chunk_s, mode=w.mode, dtype=w.dtype,
-                 lm_window=w.lm_window)
+                 lm_window=w.lm_window, position_shift=w.position_shift)
     stream = torch.cuda.Stream()
 
     def one_document():

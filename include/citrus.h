@@ -75,6 +75,17 @@ typedef struct CUstream_st* citrus_stream_t;
                                              instruction queries (the final eviction) evicts [C ; chunk] to budget_k.
                                              budget_k + 2 chunk_s <= CITRUS_MAX_CANDIDATES. */
 
+#define CITRUS_MODE_POSITION_SHIFT 0x80000000u /* position shift (Section "Hyperparameters"): positional embeddings follow
+                                             the place in the cache, not the place in the document.  Q_chunk, K_chunk
+                                             and Q_instr are passed WITHOUT rotary embedding; every step embeds them
+                                             by their place in [cache ; chunk ; instruction] (cache row r -> r, chunk
+                                             token i -> rows + i, instruction token i -> rows + n_tokens + i; half-split
+                                             layout: element d pairs with d + head_dim/2 and turns by
+                                             pos * base^(-2d/head_dim), base 10000 unless citrus_set_rope_base is
+                                             called).  The caches keep the un-rotated keys (that is what
+                                             citrus_cache_view shows) next to a copy embedded by slot, which the
+                                             compaction rewrites as rows move.  Not together with DEFERRED_LM. */
+
 #define CITRUS_OK                 0
 #define CITRUS_ERR_INVALID_ARG   -1
 #define CITRUS_ERR_SHAPE         -2
@@ -196,7 +207,8 @@ int citrus_step_view(citrus_handle h, int layer, int which, int seq_slot,
 #define CITRUS_KERNEL_COLSUM    2   /* a2, column sums (instruction and LM) */
 #define CITRUS_KERNEL_SELECT    3   /* a3 (separate launch only with CITRUS_MODE_LAYERWISE) */
 #define CITRUS_KERNEL_COMPACT   4   /* a4 (per-head granularity: one launch with a3) */
-#define CITRUS_N_KERNELS        5
+#define CITRUS_KERNEL_ROPE      5   /* embedding pre-pass of CITRUS_MODE_POSITION_SHIFT */
+#define CITRUS_N_KERNELS        6
 int citrus_profile(citrus_handle h, int enable);
 int citrus_profile_read(citrus_handle h, double* ms, long long* launches);
 
@@ -246,6 +258,10 @@ int citrus_importance_static(const void* Q_s, int n_s, const void* K, int n_keys
  * process call of that unit.
  */
 int citrus_intersection_ratio(citrus_handle h, int layer, int seq_slot, float* ratio_dev, citrus_stream_t stream);
+
+/* Base of the rotary embedding of a CITRUS_MODE_POSITION_SHIFT context (default 10000; Llama-3 uses 500000).
+ * Only before the context's first step (CITRUS_ERR_STATE afterwards); base > 1. */
+int citrus_set_rope_base(citrus_handle h, double base);
 
 /* Reads the device status word (0, or CITRUS_ERR_TIMEOUT if a bounded wait in a
  * kernel gave up). Synchronises the device. */

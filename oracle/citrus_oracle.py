@@ -154,6 +154,14 @@ def rope(x: np.ndarray, pos: np.ndarray, base: float = 10000.0) -> np.ndarray:
     return np.concatenate([x1 * c - x2 * s_, x2 * c + x1 * s_], axis=-1)
 
 
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest bfloat16 (ties to even), returned as fp64: the precision in which a bf16 model holds
+    its rotary-embedded queries and keys."""
+    b = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    b = ((b + 0x7FFF + ((b >> 16) & 1)) & 0xFFFF0000).astype(np.uint32)
+    return b.view(np.float32).astype(np.float64)
+
+
 # --------------------------------------------------------------------------
 # Diagnostic of the appendix "Details for the Intersection Probing Experiments":
 # |C_context  intersect  C_instruction| / |C_instruction| for two sets of retained states
@@ -215,7 +223,7 @@ class CitrusOracle:
     def __init__(self, q_heads, kv_heads, head_dim, budget_k, mode=SHARED,
                  lm_window: Optional[int] = None, layerwise: bool = False, start_size: int = 0,
                  accumulate: bool = False, deferred_lm: bool = False, rope_shift: bool = False,
-                 rope_base: float = 10000.0):
+                 rope_base: float = 10000.0, embedded_dtype: Optional[str] = None):
         assert q_heads % kv_heads == 0
         self.Hq, self.Hkv, self.D, self.k = q_heads, kv_heads, head_dim, budget_k
         self.mode = mode
@@ -236,6 +244,9 @@ class CitrusOracle:
         # i -> m + L + i).  The caches keep the un-rotated keys.
         self.rope_shift = rope_shift
         self.rope_base = rope_base
+        # "bf16": the embedded queries and keys exist as bf16 tensors (one rounding of the fp64 rotation), as they do
+        # in a bf16 model; None keeps them in fp64
+        self.embedded_dtype = embedded_dtype
         assert not (rope_shift and deferred_lm)
         self.tokens_seen = 0
         n_caches = 2 if mode == INDIVIDUAL else 1
@@ -263,6 +274,10 @@ class CitrusOracle:
             if Qi is not None:
                 Qi = rope(Qi, (m + L + np.arange(Qi.shape[0]))[:, None], b)
             cacheK = {cid: rope(st.K, np.arange(st.K.shape[1])[None, :], b) for cid, st in enumerate(self.caches)}
+            if self.embedded_dtype == "bf16":
+                Qc, Kc = round_bf16(Qc), round_bf16(Kc)
+                Qi = None if Qi is None else round_bf16(Qi)
+                cacheK = {cid: round_bf16(x) for cid, x in cacheK.items()}
         c0K = cacheK[0]
 
         scores: Dict[int, np.ndarray] = {}

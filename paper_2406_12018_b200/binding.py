@@ -22,15 +22,17 @@ MODE_LAYERWISE = 4
 MODE_STANDARD = 8
 MODE_ACCUMULATE = 0x20000000
 MODE_DEFERRED_LM = 0x40000000
+MODE_POSITION_SHIFT = 0x80000000
 MAX_INSTR = 4096
 MAX_CANDIDATES = 49152
 
-KERNEL_NAMES = ["attention", "score_lse", "colsum", "select", "compact"]
+KERNEL_NAMES = ["attention", "score_lse", "colsum", "select", "compact", "rope"]
 
 EXPORTS = [
     "citrus_create", "citrus_set_batch", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
     "citrus_process_chunk_host", "citrus_process_chunk_batch", "citrus_cache_view", "citrus_step_view", "citrus_profile",
-    "citrus_profile_read", "citrus_importance_static", "citrus_intersection_ratio", "citrus_poll_status",
+    "citrus_profile_read", "citrus_importance_static", "citrus_intersection_ratio", "citrus_set_rope_base",
+    "citrus_poll_status",
     "citrus_destroy", "citrus_strerror",
 ]
 
@@ -64,6 +66,7 @@ def load() -> C.CDLL:
     lib.citrus_step_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(i), C.POINTER(vp),
                                      C.POINTER(i), C.POINTER(i), C.POINTER(i)]
     lib.citrus_intersection_ratio.argtypes = [vp, i, i, vp, vp]
+    lib.citrus_set_rope_base.argtypes = [vp, C.c_double]
     lib.citrus_profile.argtypes = [vp, i]
     lib.citrus_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     lib.citrus_importance_static.argtypes = [vp, i, vp, i, i, i, i, C.c_uint, vp, i, vp, vp]
@@ -118,7 +121,8 @@ class Citrus:
     """One eviction context (all layers and sequence slots of one geometry)."""
 
     def __init__(self, layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, mode="shared", dtype="bf16",
-                 lm_window=0, layerwise=False, n_seqs=1, start_size=0, accumulate=False, deferred_lm=False):
+                 lm_window=0, layerwise=False, n_seqs=1, start_size=0, accumulate=False, deferred_lm=False, position_shift=False,
+                 rope_base=None):
         lib = load()
         bits = {"individual": MODE_INDIVIDUAL, "standard": MODE_STANDARD}.get(mode, MODE_SHARED)
         bits |= MODE_FP32 if dtype == "fp32" else 0
@@ -127,6 +131,7 @@ class Citrus:
         bits |= (int(start_size) & 0xF) << 24
         bits |= MODE_ACCUMULATE if accumulate else 0
         bits |= MODE_DEFERRED_LM if deferred_lm else 0
+        bits |= MODE_POSITION_SHIFT if position_shift else 0
         self._h = C.c_void_p()
         rc = lib.citrus_create(C.byref(self._h), layers, q_heads, kv_heads, head_dim, budget_k, chunk_s, bits)
         if rc != 0:
@@ -138,6 +143,11 @@ class Citrus:
         # row capacity of each cache's buffers: with deferred eviction cache 0 also holds the previous chunk
         self.cap = (budget_k + (chunk_s if deferred_lm else 0), budget_k)
         self.torch_dtype = torch.float32 if dtype == "fp32" else torch.bfloat16
+        if rope_base is not None:
+            rc = lib.citrus_set_rope_base(self._h, float(rope_base))
+            if rc != 0:
+                self.close()
+                raise CitrusError(rc, "citrus_set_rope_base")
         if n_seqs != 1:
             rc = lib.citrus_set_batch(self._h, n_seqs)
             if rc != 0:

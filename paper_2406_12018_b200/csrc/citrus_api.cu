@@ -3,6 +3,7 @@
 #include "../../include/citrus.h"
 #include "citrus_internal.h"
 
+#include <cmath>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -19,6 +20,7 @@ struct CacheBufs {
     void* V[2] = {nullptr, nullptr};
     int* pos[2] = {nullptr, nullptr};
     float* carried[2] = {nullptr, nullptr};      // accumulative policy: importance carried by the rows
+    void* Kraw[2] = {nullptr, nullptr};          // position shift: the un-rotated keys (K[] then holds them embedded by slot)
     int cur = 0;
 };
 
@@ -46,6 +48,9 @@ struct citrus_ctx {
     bool accumulate = false;        // scores carried across steps
     bool deferred = false;          // cache 0 holds k states + the previous chunk and is evicted by the next chunk
     int cap[2] = {0, 0};            // row capacity of each cache's buffers
+    bool shift = false;             // position shift: rotary embedding by cache slot
+    RopeTable rope;                 // its angles per pair
+    void *rotQ = nullptr, *rotK = nullptr, *rotQi = nullptr;   // the step's embedded chunk queries / keys / instruction queries
     int elt = 2;
     int n_caches = 1;
     int n_slots = 1;
@@ -106,6 +111,7 @@ int alloc_units(citrus_ctx* c) {
             for (int b = 0; b < 2; ++b) {
                 if ((rc = dev_alloc(c, &u.cache[ci].K[b], kv_bytes, true))) return rc;
                 if ((rc = dev_alloc(c, &u.cache[ci].V[b], kv_bytes, true))) return rc;
+                if (c->shift && (rc = dev_alloc(c, &u.cache[ci].Kraw[b], kv_bytes, true))) return rc;
                 if ((rc = dev_alloc(c, (void**)&u.cache[ci].pos[b], (size_t)c->Hkv * c->cap[ci] * sizeof(int), true))) return rc;
                 if (c->accumulate &&
                     (rc = dev_alloc(c, (void**)&u.cache[ci].carried[b], (size_t)c->Hkv * c->cap[ci] * sizeof(float), true))) return rc;
@@ -182,13 +188,23 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         cand[ci] = Candidates{cb.K[cb.cur], cb.V[cb.cur], Kc, Vc, mc[ci], L, c->cap[ci], c->Hkv};
     }
     const int m = mc[0];
+    cudaError_t e;
+    const void* Kc_raw = Kc;                                      // what the compaction gathers
+    if (c->shift) {
+        // position shift: embed the chunk's queries and keys at rows m .. m+L-1 and the instruction queries behind them
+        RopeRows jobs[3] = {{Qc, c->rotQ, L, c->Hq, mc[0]}, {Kc, c->rotK, L, c->Hkv, mc[0]}, {Qi, c->rotQi, nI, c->Hq, mc[0] + L}};
+        LaunchTimer t(c, CITRUS_KERNEL_ROPE, st);
+        e = rope_rows(jobs, instr_scoring ? 3 : 2, c->D, c->elt, c->rope, st);
+        if (e != cudaSuccess) return cuda_rc(e);
+        Qc = c->rotQ; Kc = c->rotK; if (instr_scoring) Qi = c->rotQi;
+        for (int ci = 0; ci < c->n_caches; ++ci) cand[ci].chunkK = Kc;
+    }
     QueryRows q_chunk{Qc, L, c->Hq, 1, 0};
     QueryRows q_instr{Qi, nI, c->Hq, 0, 0};
     float* scores[2] = {u.scores, u.scores + (size_t)c->Hkv * c->score_stride};
     const int ic = c->individual ? 1 : 0;     // the cache scored by the instruction text
     if (!instr_scoring) q_instr.rows = 0;
 
-    cudaError_t e;
     float* lse_chunk = lm_scoring ? u.lse_chunk : nullptr;        // only a2-L reads a1's row log-sum-exp
     int splits = 1;
     if (c->use_tc) {
@@ -241,7 +257,8 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
                             cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, mc[ci],
                             c->accumulate ? scores[ci] : nullptr, c->score_stride,
-                            c->accumulate ? cb.carried[cb.cur ^ 1] : nullptr, c->cap[ci], kept[ci]};
+                            c->accumulate ? cb.carried[cb.cur ^ 1] : nullptr, c->cap[ci], kept[ci],
+                            c->shift ? cb.Kraw[cb.cur] : nullptr, c->shift ? cb.Kraw[cb.cur ^ 1] : nullptr};
         gather_bytes += (size_t)c->Hkv * kept[ci] * c->D * c->elt * 2;
     }
     // Small steps (a few MB to move) are latency-bound: one cluster launch does a3 and a4.  Large steps want every
@@ -249,7 +266,8 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     if (!c->layerwise && gather_bytes <= ((size_t)8 << 20)) {
         // one cluster launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-        e = select_compact(sj, cj, c->n_caches, Kc, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen, st);
+        e = select_compact(sj, cj, c->n_caches, Kc_raw, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen,
+                           c->shift ? &c->rope : nullptr, c->elt, st);
         if (e != cudaSuccess) return cuda_rc(e);
     } else {
         {
@@ -259,7 +277,8 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         if (e != cudaSuccess) return cuda_rc(e);
         {
             LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-            e = compact_kv(cj, c->n_caches, Kc, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen, st);
+            e = compact_kv(cj, c->n_caches, Kc_raw, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen,
+                           c->shift ? &c->rope : nullptr, c->elt, st);
         }
         if (e != cudaSuccess) return cuda_rc(e);
     }
@@ -290,7 +309,8 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     if (out == nullptr) return CITRUS_ERR_INVALID_ARG;
     *out = nullptr;
     if (layers < 1 || q_heads < 1 || kv_heads < 1 || budget_k < 1 || chunk_s < 1) return CITRUS_ERR_INVALID_ARG;
-    if (mode & ~(0xFu | 0xFFFF00u | 0xF000000u | CITRUS_MODE_ACCUMULATE | CITRUS_MODE_DEFERRED_LM)) return CITRUS_ERR_INVALID_ARG;
+    if (mode & ~(0xFu | 0xFFFF00u | 0xF000000u | CITRUS_MODE_ACCUMULATE | CITRUS_MODE_DEFERRED_LM | CITRUS_MODE_POSITION_SHIFT)) return CITRUS_ERR_INVALID_ARG;
+    if ((mode & CITRUS_MODE_POSITION_SHIFT) && (mode & CITRUS_MODE_DEFERRED_LM)) return CITRUS_ERR_INVALID_ARG;
     if ((mode & CITRUS_MODE_DEFERRED_LM) && !(mode & (CITRUS_MODE_INDIVIDUAL | CITRUS_MODE_STANDARD))) return CITRUS_ERR_INVALID_ARG;
     if ((mode & CITRUS_MODE_STANDARD) && (mode & CITRUS_MODE_INDIVIDUAL)) return CITRUS_ERR_INVALID_ARG;
     if (q_heads % kv_heads != 0) return CITRUS_ERR_SHAPE;
@@ -312,6 +332,8 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     c->start_size = (int)((mode >> 24) & 0xFu);
     c->accumulate = (mode & CITRUS_MODE_ACCUMULATE) != 0;
     c->deferred = (mode & CITRUS_MODE_DEFERRED_LM) != 0;
+    c->shift = (mode & CITRUS_MODE_POSITION_SHIFT) != 0;
+    for (int d = 0; d < 64; ++d) c->rope.theta[d] = std::pow(10000.0, -2.0 * d / head_dim);
     c->cap[0] = budget_k + (c->deferred ? chunk_s : 0);
     c->cap[1] = budget_k;
     c->elt = fp32 ? 4 : 2;
@@ -324,6 +346,12 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     }
     int rc = dev_alloc(c, (void**)&c->status, sizeof(int), true, true);
     if (rc == CITRUS_OK && c->use_tc && tc_init() != cudaSuccess) rc = CITRUS_ERR_UNSUPPORTED;
+    if (rc == CITRUS_OK && c->shift) {
+        const size_t row = (size_t)head_dim * c->elt;
+        rc = dev_alloc(c, &c->rotQ, (size_t)chunk_s * q_heads * row, false, true);
+        if (rc == CITRUS_OK) rc = dev_alloc(c, &c->rotK, (size_t)chunk_s * kv_heads * row, false, true);
+        if (rc == CITRUS_OK) rc = dev_alloc(c, &c->rotQi, (size_t)CITRUS_MAX_INSTR * q_heads * row, false, true);
+    }
     if (rc == CITRUS_OK) rc = alloc_units(c);
     if (rc != CITRUS_OK) { free_all(c); delete c; return rc; }
     {
@@ -351,6 +379,13 @@ int citrus_set_batch(citrus_handle h, int n_seq) {
             return rc;
         }
     }
+    return CITRUS_OK;
+}
+
+int citrus_set_rope_base(citrus_handle h, double base) {
+    if (h == nullptr || !is_live(h) || !(base > 1.0)) return CITRUS_ERR_INVALID_ARG;
+    if (!h->shift || h->used) return CITRUS_ERR_STATE;
+    for (int d = 0; d < 64; ++d) h->rope.theta[d] = std::pow(base, -2.0 * d / h->D);
     return CITRUS_OK;
 }
 
@@ -443,7 +478,7 @@ int citrus_cache_view(citrus_handle h, int layer, int which, int seq_slot,
     if (h->units.empty()) return CITRUS_ERR_STATE;
     const Unit& u = h->units[(size_t)layer * h->n_slots + seq_slot];
     const CacheBufs& cb = u.cache[which];
-    if (K) *K = cb.K[cb.cur];
+    if (K) *K = h->shift ? cb.Kraw[cb.cur] : cb.K[cb.cur];
     if (V) *V = cb.V[cb.cur];
     if (positions) *positions = cb.pos[cb.cur];
     if (n_rows) *n_rows = u.m[which];

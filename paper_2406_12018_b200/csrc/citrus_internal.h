@@ -97,12 +97,21 @@ struct CompactJob {
     const float* totals; int score_stride; float* dstCarried;  // null when the policy is off
     int cap;                                                  // row capacity of this cache's buffers (old and new)
     int kept;                                                 // rows of the new cache
+    // position shift: the un-rotated keys are what is gathered (old raw cache, caller's chunk K) and kept in
+    // dstKraw; dstK receives them embedded by their new slot.  Null when the mode is off.
+    const void* srcKraw; void* dstKraw;
 };
+// Rotary embedding in the half-split layout: element d pairs with d + D/2, the pair turns by pos * theta[d].
+struct RopeTable { double theta[64]; };
+// One tensor of the embedding pre-pass: token-major [rows, heads, D], row i embedded at position pos0 + i.
+struct RopeRows { const void* in; void* out; int rows, heads, pos0; };
+cudaError_t rope_rows(const RopeRows* jobs, int n_jobs, int D, int elt, const RopeTable& table, cudaStream_t s);
+// rope: table of the position shift, or null (the jobs' raw pointers are then null too); elt = bytes per element
 cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
-                       int kv_heads, int row_bytes, int chunk_pos0, cudaStream_t s);
+                       int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s);
 // a3 + a4 in one launch (per-head granularity): clusters of CTAs per (cache, KV head).
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
-                           int kv_heads, int row_bytes, int chunk_pos0, cudaStream_t s);
+                           int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s);
 // ratio[g] = |{positions of a} intersect {positions of b}| / rows_b over two ascending position lists per head
 cudaError_t intersection_ratio(const int* pos_a, int stride_a, int rows_a, const int* pos_b, int stride_b, int rows_b,
                                int kv_heads, float* ratio, cudaStream_t s);

@@ -19,7 +19,37 @@ constexpr int kSelThreads = 1024;
 constexpr int kMaxJobs = 2;
 
 struct SelectArgs { SelectJob job[kMaxJobs]; };
-struct CompactArgs { CompactJob job[kMaxJobs]; };
+struct CompactArgs { CompactJob job[kMaxJobs]; RopeTable rope; int elt; };
+
+// A 16-byte piece of a key row embedded at position `pos`: `mine` holds elements [d0, d0 + E) of one half of the head
+// dimension, `other` the same elements of the other half (E = 8 bf16 or 4 fp32); lower: `mine` is the first half.
+// first' = first cos - second sin, second' = second cos + first sin, angle = pos * theta[d].
+__device__ __forceinline__ uint4 rope_piece(uint4 mine, uint4 other, int pos, int d0, bool lower, const RopeTable& t, int elt) {
+    const uint32_t* a = reinterpret_cast<const uint32_t*>(&mine);
+    const uint32_t* b = reinterpret_cast<const uint32_t*>(&other);
+    uint4 out;
+    uint32_t* o = reinterpret_cast<uint32_t*>(&out);
+    auto turn = [&](float x, float y, int d) {
+        double ang = (double)pos * t.theta[d];
+        ang -= 6.283185307179586 * floor(ang * 0.15915494309189535);     // into [0, 2 pi) before the fp32 sincos
+        float sn, cs;
+        sincosf((float)ang, &sn, &cs);
+        return lower ? x * cs - y * sn : x * cs + y * sn;
+    };
+    if (elt == 2) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float x0 = __uint_as_float(a[w] << 16), x1 = __uint_as_float(a[w] & 0xffff0000u);
+            const float y0 = __uint_as_float(b[w] << 16), y1 = __uint_as_float(b[w] & 0xffff0000u);
+            __nv_bfloat162 r = __floats2bfloat162_rn(turn(x0, y0, d0 + 2 * w), turn(x1, y1, d0 + 2 * w + 1));
+            o[w] = *reinterpret_cast<uint32_t*>(&r);
+        }
+    } else {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) o[w] = __float_as_uint(turn(__uint_as_float(a[w]), __uint_as_float(b[w]), d0 + w));
+    }
+    return out;
+}
 
 // Order-preserving map from fp32 to uint32 (larger float <=> larger key).
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -216,20 +246,23 @@ select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int la
 // Rows [r_begin, r_end) of one (cache, head) are copied with 128-bit accesses, row_bytes/16 lanes per row.
 __device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4* __restrict__ chunkK,
                                              const uint4* __restrict__ chunkV, const int g, int kv_heads,
-                                             int row_vecs, int r_begin, int r_end, int chunk_pos0, const int* idx) {
+                                             int row_vecs, int r_begin, int r_end, int chunk_pos0, const int* idx,
+                                             const RopeTable& rope, int elt) {
     const int cap = job.cap;
+    const bool shift = job.dstKraw != nullptr;        // position shift: gather un-rotated keys, embed by the new slot
     // idx[r] = candidate kept in row r of this head (global list, or the CTA's slice in shared memory)
     const int rows_per_pass = blockDim.x / row_vecs;
     const int sub = threadIdx.x / row_vecs, v = threadIdx.x % row_vecs;
-    const uint4* srcK = reinterpret_cast<const uint4*>(job.srcK);
+    const uint4* srcK = reinterpret_cast<const uint4*>(shift ? job.srcKraw : job.srcK);
     const uint4* srcV = reinterpret_cast<const uint4*>(job.srcV);
-    uint4* dstK = reinterpret_cast<uint4*>(job.dstK);
+    uint4* dstK = reinterpret_cast<uint4*>(shift ? job.dstKraw : job.dstK);
+    uint4* dstKrot = reinterpret_cast<uint4*>(job.dstK);
     uint4* dstV = reinterpret_cast<uint4*>(job.dstV);
     // four rows per thread in flight: first every index, then every load, then the stores
     constexpr int kInFlight = 4;
     for (int rb = r_begin + sub; rb < r_end; rb += kInFlight * rows_per_pass) {
         int j[kInFlight];
-        uint4 a[kInFlight], b[kInFlight];
+        uint4 a[kInFlight] = {}, b[kInFlight] = {};
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
             const int r = rb + u * rows_per_pass;
@@ -247,6 +280,21 @@ __device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4*
                 pk = chunkK + off; pv = chunkV + off;
             }
             a[u] = __ldg(pk); b[u] = __ldg(pv);
+        }
+        if (shift) {
+            // the other half of the head dimension sits half a row away, in a lane of the same warp; every lane
+            // takes part in the exchange, rows past the end only skip the store
+            const int half_vecs = row_vecs >> 1, per_vec = 16 / elt;
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) {
+                uint4 other;
+                other.x = __shfl_xor_sync(0xffffffffu, a[u].x, half_vecs); other.y = __shfl_xor_sync(0xffffffffu, a[u].y, half_vecs);
+                other.z = __shfl_xor_sync(0xffffffffu, a[u].z, half_vecs); other.w = __shfl_xor_sync(0xffffffffu, a[u].w, half_vecs);
+                if (j[u] < 0) continue;
+                const int r = rb + u * rows_per_pass;
+                dstKrot[((size_t)g * cap + r) * row_vecs + v] =
+                    rope_piece(a[u], other, r, (v % half_vecs) * per_vec, v < half_vecs, rope, elt);
+            }
         }
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
@@ -275,7 +323,7 @@ compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restr
     const CompactJob& job = args.job[blockIdx.z];
     const int r0 = blockIdx.x * kCompactRowsPerCta;
     compact_rows(job, chunkK, chunkV, blockIdx.y, kv_heads, row_vecs,
-                 r0, min(job.kept, r0 + kCompactRowsPerCta), chunk_pos0, job.idx + (size_t)blockIdx.y * job.cap);
+                 r0, min(job.kept, r0 + kCompactRowsPerCta), chunk_pos0, job.idx + (size_t)blockIdx.y * job.cap, args.rope, args.elt);
 }
 
 // a3 + a4 in one launch: a cluster of kFusedCluster CTAs per (cache, KV head).  The first CTA of the cluster
@@ -316,7 +364,8 @@ select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_const
     CITRUS_SPAN_MAX(3);
     CITRUS_TR(16);
     const int r0 = blockIdx.x * per;
-    compact_rows(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, row_vecs, r0, min(kept, r0 + per), chunk_pos0, s_idx - r0);
+    compact_rows(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, row_vecs, r0, min(kept, r0 + per), chunk_pos0, s_idx - r0,
+                 cmp.rope, cmp.elt);
     CITRUS_SPAN_MAX(2);
     CITRUS_TR(17);
 }
@@ -348,7 +397,56 @@ intersection_kernel(const int* __restrict__ pos_a, int stride_a, int rows_a, con
     if (threadIdx.x == 0) ratio[g] = (float)hits / (float)rows;
 }
 
+constexpr int kMaxRopeJobs = 3;
+struct RopeArgs { RopeRows job[kMaxRopeJobs]; RopeTable table; int n_jobs, row_vecs, elt; };
+
+// Embedding pre-pass of the position shift: every 16-byte piece of the listed token-major tensors is turned by the
+// position of its row.  grid.y = tensor, grid-stride over its pieces.
+__global__ void __launch_bounds__(256)
+rope_rows_kernel(const __grid_constant__ RopeArgs args) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // the outputs are scratch that the previous step's kernels may still be reading
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const RopeRows& job = args.job[blockIdx.y];
+    const int row_vecs = args.row_vecs, half_vecs = row_vecs >> 1, per_vec = 16 / args.elt;
+    const long long total = (long long)job.rows * job.heads * row_vecs;          // a multiple of 32
+    const uint4* in = reinterpret_cast<const uint4*>(job.in);
+    uint4* out = reinterpret_cast<uint4*>(job.out);
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int v = (int)(i % row_vecs);
+        const int row = (int)(i / ((long long)row_vecs * job.heads));
+        const uint4 mine = __ldg(in + i);
+        uint4 other;
+        other.x = __shfl_xor_sync(0xffffffffu, mine.x, half_vecs); other.y = __shfl_xor_sync(0xffffffffu, mine.y, half_vecs);
+        other.z = __shfl_xor_sync(0xffffffffu, mine.z, half_vecs); other.w = __shfl_xor_sync(0xffffffffu, mine.w, half_vecs);
+        out[i] = rope_piece(mine, other, job.pos0 + row, (v % half_vecs) * per_vec, v < half_vecs, args.table, args.elt);
+    }
+}
+
 }  // namespace
+
+cudaError_t rope_rows(const RopeRows* jobs, int n_jobs, int D, int elt, const RopeTable& table, cudaStream_t s) {
+    if (n_jobs < 1 || n_jobs > kMaxRopeJobs) return cudaErrorInvalidValue;
+    RopeArgs a;
+    a.table = table; a.n_jobs = n_jobs; a.row_vecs = D * elt / 16; a.elt = elt;
+    long long most = 0;
+    for (int i = 0; i < n_jobs; ++i) {
+        a.job[i] = jobs[i];
+        const long long t = (long long)jobs[i].rows * jobs[i].heads * a.row_vecs;
+        most = t > most ? t : most;
+    }
+    cudaLaunchConfig_t cfg = {};
+    long long blocks = (most + 255) / 256;
+    cfg.gridDim = dim3((unsigned)(blocks > 592 ? 592 : (blocks < 1 ? 1 : blocks)), n_jobs);
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    before_launch(s);
+    return cudaLaunchKernelEx(&cfg, rope_rows_kernel, a);
+}
 
 cudaError_t intersection_ratio(const int* pos_a, int stride_a, int rows_a, const int* pos_b, int stride_b, int rows_b,
                                int kv_heads, float* ratio, cudaStream_t s) {
@@ -382,9 +480,11 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int lay
 }
 
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
-                           int kv_heads, int row_bytes, int chunk_pos0, cudaStream_t s) {
+                           int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s) {
     if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
     SelectArgs sa; CompactArgs ca;
+    ca.elt = elt;
+    if (rope != nullptr) ca.rope = *rope;
     int n = 0, kept = 0;
     for (int i = 0; i < n_jobs; ++i) {
         sa.job[i] = sjobs[i]; ca.job[i] = cjobs[i];
@@ -414,9 +514,11 @@ cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int 
 }
 
 cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
-                       int kv_heads, int row_bytes, int chunk_pos0, cudaStream_t s) {
+                       int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s) {
     if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
     CompactArgs a;
+    a.elt = elt;
+    if (rope != nullptr) a.rope = *rope;
     int kept = 0;
     for (int i = 0; i < n_jobs; ++i) { a.job[i] = jobs[i]; kept = jobs[i].kept > kept ? jobs[i].kept : kept; }
     int row_vecs = row_bytes / 16;

@@ -49,6 +49,8 @@ class Workload:
     start_size: int = 0        # initial tokens that are never evicted (paper's appendix variant: 4)
     accumulate: bool = False   # accumulative score policy: importance carried across steps
     deferred_lm: bool = False  # language-modelling cache evicted by the next chunk (Section 4.1 order)
+    position_shift: bool = False   # inputs without rotary embedding; embedded by cache slot every step
+    rope_base: float = 10000.0
 
     @property
     def torch_dtype(self):
@@ -78,6 +80,9 @@ CONFIGS = {
 PAPER_SHAPES = {
     "paper_mistral7b": Workload("paper_mistral7b", 11, 1, 32, 8, 128, 768, 256, 16384, 64, "bf16", "shared",
                                 n_planted=32, n_sinks=1),
+    # the same with the position shift the paper applies (inputs without rotary embedding, embedded by cache slot)
+    "paper_mistral7b_shift": Workload("paper_mistral7b_shift", 11, 1, 32, 8, 128, 768, 256, 16384, 64, "bf16", "shared",
+                                      n_planted=32, n_sinks=1, position_shift=True),
     "paper_llama2_13b": Workload("paper_llama2_13b", 12, 1, 40, 40, 128, 768, 256, 16384, 64, "bf16", "shared",
                                  n_planted=32, n_sinks=1),
     "paper_llama3_8b": Workload("paper_llama3_8b", 13, 1, 32, 8, 128, 768, 256, 16384, 64, "bf16", "individual",

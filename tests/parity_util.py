@@ -25,14 +25,17 @@ SWAP_REL = 1e-5
 def make_pair(w: wl.Workload, layers=1, layerwise=False):
     ctx = Citrus(layers, w.q_heads, w.kv_heads, w.head_dim, w.budget_k, w.chunk_s, mode=w.mode, dtype=w.dtype,
                  lm_window=w.lm_window, layerwise=layerwise, n_seqs=w.n_seqs, start_size=w.start_size,
-                 accumulate=w.accumulate, deferred_lm=w.deferred_lm)
+                 accumulate=w.accumulate, deferred_lm=w.deferred_lm, position_shift=w.position_shift,
+                 rope_base=w.rope_base if w.position_shift else None)
     return ctx
 
 
 def make_oracle(w: wl.Workload, layerwise=False):
     return CitrusOracle(w.q_heads, w.kv_heads, w.head_dim, w.budget_k, w.mode,
                         lm_window=(w.lm_window or None), layerwise=layerwise, start_size=w.start_size,
-                        accumulate=w.accumulate, deferred_lm=w.deferred_lm)
+                        accumulate=w.accumulate, deferred_lm=w.deferred_lm, rope_shift=w.position_shift,
+                        rope_base=w.rope_base,
+                        embedded_dtype="bf16" if (w.position_shift and w.dtype == "bf16") else None)
 
 
 def check_index_rule(own, gpu, scores, n, k):

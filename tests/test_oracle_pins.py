@@ -488,6 +488,16 @@ def test_rope_is_a_rotation_of_complex_pairs_and_depends_on_relative_position_on
     assert abs(np.linalg.norm(rope(q, np.array(123))) - np.linalg.norm(q)) < 1e-12
 
 
+def test_round_bf16_is_round_to_nearest_even_on_the_upper_sixteen_bits():
+    from oracle import round_bf16
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, 1.0 + 3 * 2.0 ** -8, -0.3, 3.0e-40, 65504.0])
+    r = round_bf16(x)
+    # 1 + 2^-8 is half way between 1 and 1 + 2^-7: ties go to the even mantissa (1.0); just above goes up;
+    # 1 + 3 * 2^-8 is half way between 1 + 2^-7 and 1 + 2^-6: the even one is 1 + 2^-6
+    assert r[0] == 1.0 and r[1] == 1.0 and r[2] == 1.0 + 2.0 ** -7 and r[3] == 1.0 + 2.0 ** -6
+    assert np.array_equal(r, torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy())
+
+
 def test_position_shift_without_eviction_is_ordinary_rope_by_document_position():
     # budget larger than the document: every state keeps its place, so cache slot = document position and the shifted
     # run must equal a plain run on inputs that were embedded up front

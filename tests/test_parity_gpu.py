@@ -4,7 +4,7 @@ import pytest
 import torch
 
 from paper_2406_12018_b200 import workloads as wl
-from paper_2406_12018_b200.binding import Citrus, CitrusError
+from paper_2406_12018_b200.binding import Citrus, CitrusError, load as load_lib
 import parity_util as pu
 
 pytestmark = pytest.mark.gpu
@@ -125,6 +125,29 @@ def test_deferred_eviction_of_the_language_modelling_cache(mode, dtype, lm_windo
         Citrus(1, 8, 2, 128, 200, 160, mode="shared", deferred_lm=True)  # no language-modelling cache to defer
     with pytest.raises(CitrusError):
         Citrus(1, 8, 2, 128, 40000, 5000, mode="standard", deferred_lm=True)   # budget + 2 chunks exceeds the limit
+
+
+@pytest.mark.parametrize("mode,dtype,D,base", [("shared", "bf16", 128, 10000.0), ("shared", "fp32", 64, 10000.0),
+                                                ("individual", "bf16", 128, 500000.0), ("shared", "fp32", 128, 10000.0)])
+def test_position_shift_embeds_by_cache_slot(mode, dtype, D, base):
+    # inputs arrive without rotary embedding; the library embeds chunk, instruction and cache rows by their slot
+    w = wl.scaled(C["tiny_fp32"], q_heads=8, kv_heads=2, head_dim=D, budget_k=200, chunk_s=160, doc_tokens=1000,
+                  n_instr=12, dtype=dtype, mode=mode, lm_window=16, n_planted=4, n_sinks=1, position_shift=True,
+                  rope_base=base)
+    ctx = pu.make_pair(w)
+    _, st = pu.run_document(w, ctx, chunk_lengths=[160, 160, 97, 160, 160, 160, 103])
+    _report(f"position shift {mode} {dtype} D{D}", st)
+    assert st["checked_chunks"] == 7
+    ctx.close()
+    with pytest.raises(CitrusError):
+        Citrus(1, 8, 2, 128, 200, 160, mode="individual", deferred_lm=True, position_shift=True)
+    plain = Citrus(1, 8, 2, 128, 200, 160)
+    with pytest.raises(CitrusError):
+        load_lib().citrus_set_rope_base  # noqa: B018  (symbol exists)
+        rc = load_lib().citrus_set_rope_base(plain._h, 10000.0)
+        if rc != 0:
+            raise CitrusError(rc, "citrus_set_rope_base")             # not a position-shift context
+    plain.close()
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
