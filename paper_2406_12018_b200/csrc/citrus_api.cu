@@ -263,7 +263,7 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     }
     // Small steps (a few MB to move) are latency-bound: one cluster launch does a3 and a4.  Large steps want every
     // SM streaming rows, which the clusters (idle while their first CTA selects) cannot give: two launches.
-    if (!c->layerwise && gather_bytes <= ((size_t)8 << 20)) {
+    if (!c->layerwise && !c->shift && gather_bytes <= ((size_t)8 << 20)) {
         // one cluster launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
         e = select_compact(sj, cj, c->n_caches, Kc_raw, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen,

@@ -244,12 +244,13 @@ select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int la
 }
 
 // Rows [r_begin, r_end) of one (cache, head) are copied with 128-bit accesses, row_bytes/16 lanes per row.
-__device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4* __restrict__ chunkK,
+template <bool SHIFT>
+__device__ __forceinline__ void compact_rows_t(const CompactJob& job, const uint4* __restrict__ chunkK,
                                              const uint4* __restrict__ chunkV, const int g, int kv_heads,
                                              int row_vecs, int r_begin, int r_end, int chunk_pos0, const int* idx,
                                              const RopeTable& rope, int elt) {
     const int cap = job.cap;
-    const bool shift = job.dstKraw != nullptr;        // position shift: gather un-rotated keys, embed by the new slot
+    constexpr bool shift = SHIFT;                     // position shift: gather un-rotated keys, embed by the new slot
     // idx[r] = candidate kept in row r of this head (global list, or the CTA's slice in shared memory)
     const int rows_per_pass = blockDim.x / row_vecs;
     const int sub = threadIdx.x / row_vecs, v = threadIdx.x % row_vecs;
@@ -262,7 +263,11 @@ __device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4*
     constexpr int kInFlight = 4;
     for (int rb = r_begin + sub; rb < r_end; rb += kInFlight * rows_per_pass) {
         int j[kInFlight];
-        uint4 a[kInFlight] = {}, b[kInFlight] = {};
+        uint4 a[kInFlight], b[kInFlight];
+        if (SHIFT) {
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) a[u] = make_uint4(0u, 0u, 0u, 0u);   // rows past the end still take part in the exchange
+        }
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
             const int r = rb + u * rows_per_pass;
@@ -311,10 +316,12 @@ __device__ __forceinline__ void compact_rows(const CompactJob& job, const uint4*
     }
 }
 
+// The position-shift variant is a separate instantiation (and a separate kernel) so that the plain gather stays lean.
 // grid: (row tiles, KV heads, caches)
 constexpr int kCompactThreads = 256;
 constexpr int kCompactRowsPerCta = 64;
 
+template <bool SHIFT>
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
                   int kv_heads, int row_vecs, int chunk_pos0) {
@@ -322,8 +329,8 @@ compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restr
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the index lists are final after this
     const CompactJob& job = args.job[blockIdx.z];
     const int r0 = blockIdx.x * kCompactRowsPerCta;
-    compact_rows(job, chunkK, chunkV, blockIdx.y, kv_heads, row_vecs,
-                 r0, min(job.kept, r0 + kCompactRowsPerCta), chunk_pos0, job.idx + (size_t)blockIdx.y * job.cap, args.rope, args.elt);
+    compact_rows_t<SHIFT>(job, chunkK, chunkV, blockIdx.y, kv_heads, row_vecs,
+                          r0, min(job.kept, r0 + kCompactRowsPerCta), chunk_pos0, job.idx + (size_t)blockIdx.y * job.cap, args.rope, args.elt);
 }
 
 // a3 + a4 in one launch: a cluster of kFusedCluster CTAs per (cache, KV head).  The first CTA of the cluster
@@ -364,8 +371,9 @@ select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_const
     CITRUS_SPAN_MAX(3);
     CITRUS_TR(16);
     const int r0 = blockIdx.x * per;
-    compact_rows(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, row_vecs, r0, min(kept, r0 + per), chunk_pos0, s_idx - r0,
-                 cmp.rope, cmp.elt);
+    // (the position shift always takes the two-kernel route: its rotation does not fit this kernel's 64 registers)
+    compact_rows_t<false>(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, row_vecs, r0, min(kept, r0 + per), chunk_pos0, s_idx - r0,
+                          cmp.rope, cmp.elt);
     CITRUS_SPAN_MAX(2);
     CITRUS_TR(17);
 }
@@ -481,10 +489,9 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int lay
 
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
                            int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s) {
-    if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
+    if (n_jobs < 1 || n_jobs > kMaxJobs || rope != nullptr) return cudaErrorInvalidValue;
     SelectArgs sa; CompactArgs ca;
     ca.elt = elt;
-    if (rope != nullptr) ca.rope = *rope;
     int n = 0, kept = 0;
     for (int i = 0; i < n_jobs; ++i) {
         sa.job[i] = sjobs[i]; ca.job[i] = cjobs[i];
@@ -531,7 +538,10 @@ cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     before_launch(s);
-    return cudaLaunchKernelEx(&cfg, compact_kv_kernel, a, reinterpret_cast<const uint4*>(chunkK),
+    if (rope != nullptr)
+        return cudaLaunchKernelEx(&cfg, compact_kv_kernel<true>, a, reinterpret_cast<const uint4*>(chunkK),
+                                  reinterpret_cast<const uint4*>(chunkV), kv_heads, row_vecs, chunk_pos0);
+    return cudaLaunchKernelEx(&cfg, compact_kv_kernel<false>, a, reinterpret_cast<const uint4*>(chunkK),
                               reinterpret_cast<const uint4*>(chunkV), kv_heads, row_vecs, chunk_pos0);
 }
 
