@@ -30,7 +30,7 @@ KERNEL_NAMES = ["attention", "score_lse", "colsum", "select", "compact", "rope"]
 
 EXPORTS = [
     "citrus_create", "citrus_set_batch", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
-    "citrus_process_chunk_host", "citrus_process_chunk_batch", "citrus_cache_view", "citrus_step_view", "citrus_profile",
+    "citrus_process_chunk_host", "citrus_process_document_host", "citrus_process_chunk_batch", "citrus_cache_view", "citrus_step_view", "citrus_profile",
     "citrus_profile_read", "citrus_importance_static", "citrus_intersection_ratio", "citrus_set_rope_base",
     "citrus_poll_status",
     "citrus_destroy", "citrus_strerror",
@@ -62,6 +62,7 @@ def load() -> C.CDLL:
     lib.citrus_process_chunk_slot.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, vp]
     lib.citrus_process_chunk_batch.argtypes = [vp, i, i, C.POINTER(i), C.POINTER(i), vp, vp, vp, C.POINTER(i), vp, vp, vp]
     lib.citrus_process_chunk_host.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, vp]
+    lib.citrus_process_document_host.argtypes = [vp, i, i, vp, vp, vp, C.c_longlong, vp, i, vp, vp]
     lib.citrus_cache_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(i)]
     lib.citrus_step_view.argtypes = [vp, i, i, i, C.POINTER(vp), C.POINTER(i), C.POINTER(vp),
                                      C.POINTER(i), C.POINTER(i), C.POINTER(i)]
@@ -194,6 +195,17 @@ class Citrus:
                                               _stream_ptr(stream))
         if rc != 0:
             raise CitrusError(rc, "citrus_process_chunk_host")
+        return out
+
+    def process_document_host(self, layer, Q, K, V, Qi, out, slot=0, stream=None):
+        """A whole document from host tensors; copies and steps overlap inside the library."""
+        for t in (Q, K, V, Qi, out):
+            self._check(t, False)
+        rc = load().citrus_process_document_host(self._h, layer, slot, Q.data_ptr(), K.data_ptr(), V.data_ptr(),
+                                                 Q.shape[0], Qi.data_ptr(), Qi.shape[0], out.data_ptr(),
+                                                 _stream_ptr(stream))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_process_document_host")
         return out
 
     def cache_view(self, layer, which=0, slot=0) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:

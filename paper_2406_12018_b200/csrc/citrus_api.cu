@@ -66,6 +66,10 @@ struct citrus_ctx {
     std::vector<Timed> timed;
     // staging of the host-buffer variant
     void *stQ = nullptr, *stK = nullptr, *stV = nullptr, *stQi = nullptr, *stOut = nullptr;
+    // whole-document host variant: a second staging set, two copy streams, events per set
+    void *st2Q = nullptr, *st2K = nullptr, *st2V = nullptr, *st2Out = nullptr;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_step[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr}, ev_qi = nullptr;
 };
 
 namespace {
@@ -94,6 +98,16 @@ void free_units(citrus_ctx* c) {
     for (void* p : c->allocs) cudaFree(p);
     c->allocs.clear();
     c->units.clear();
+}
+void free_copy_streams(citrus_ctx* c) {
+    for (int b = 0; b < 2; ++b) {
+        if (c->ev_in[b]) cudaEventDestroy(c->ev_in[b]);
+        if (c->ev_step[b]) cudaEventDestroy(c->ev_step[b]);
+        if (c->ev_out[b]) cudaEventDestroy(c->ev_out[b]);
+    }
+    if (c->ev_qi) cudaEventDestroy(c->ev_qi);
+    if (c->s_in) cudaStreamDestroy(c->s_in);
+    if (c->s_out) cudaStreamDestroy(c->s_out);
 }
 void free_all(citrus_ctx* c) {
     free_units(c);
@@ -470,6 +484,86 @@ int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,
     return cuda_rc(cudaStreamSynchronize(st));
 }
 
+int citrus_process_document_host(citrus_handle h, int layer, int seq_slot,
+                                 const void* Qh, const void* Kh, const void* Vh, long long n_tokens,
+                                 const void* Qih, int n_instr, void* out_h, citrus_stream_t stream) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    if (n_tokens < 1 || n_tokens > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
+    const int first = (int)(n_tokens < h->ls ? n_tokens : h->ls);
+    int rc = check_process_args(h, layer, seq_slot, Qh, Kh, Vh, first, Qih, n_instr, out_h);
+    if (rc) return rc;
+    if (n_instr < 1) return CITRUS_ERR_SHAPE;
+    {
+        const Unit& u = h->units[(size_t)layer * h->n_slots + seq_slot];
+        if (u.tokens_seen + n_tokens > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t qrow = (size_t)h->Hq * h->D * h->elt, krow = (size_t)h->Hkv * h->D * h->elt;
+    if (h->stQ == nullptr) {
+        if ((rc = dev_alloc(h, &h->stQ, qrow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->stOut, qrow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->stK, krow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->stV, krow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->stQi, qrow * CITRUS_MAX_INSTR, false, true))) return rc;
+    }
+    cudaError_t e = cudaSuccess;
+    if (h->s_in == nullptr) {
+        if ((rc = dev_alloc(h, &h->st2Q, qrow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->st2Out, qrow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->st2K, krow * h->ls, false, true))) return rc;
+        if ((rc = dev_alloc(h, &h->st2V, krow * h->ls, false, true))) return rc;
+        e = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking);
+        for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
+            e = cudaEventCreateWithFlags(&h->ev_in[b], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_step[b], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_out[b], cudaEventDisableTiming);
+        }
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_qi, cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_rc(e);
+    }
+    void* setQ[2] = {h->stQ, h->st2Q}; void* setK[2] = {h->stK, h->st2K};
+    void* setV[2] = {h->stV, h->st2V}; void* setO[2] = {h->stOut, h->st2Out};
+    const char *q = reinterpret_cast<const char*>(Qh), *k = reinterpret_cast<const char*>(Kh), *v = reinterpret_cast<const char*>(Vh);
+    char* o = reinterpret_cast<char*>(out_h);
+    // the copy streams start behind whatever the caller's stream already holds
+    if ((e = cudaEventRecord(h->ev_qi, st)) != cudaSuccess) return cuda_rc(e);
+    if ((e = cudaStreamWaitEvent(h->s_in, h->ev_qi, 0)) != cudaSuccess) return cuda_rc(e);
+    if ((e = cudaStreamWaitEvent(h->s_out, h->ev_qi, 0)) != cudaSuccess) return cuda_rc(e);
+    if ((e = cudaMemcpyAsync(h->stQi, Qih, qrow * n_instr, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) return cuda_rc(e);
+    const long long n_chunks = (n_tokens + h->ls - 1) / h->ls;
+    for (long long c = 0; c < n_chunks && rc == CITRUS_OK; ++c) {
+        const int b = (int)(c & 1);
+        const long long t0 = c * h->ls;
+        const int L = (int)(n_tokens - t0 < h->ls ? n_tokens - t0 : h->ls);
+        // inputs of chunk c into set b, once the step that last read the set (chunk c-2) is done
+        if (c >= 2 && (e = cudaStreamWaitEvent(h->s_in, h->ev_step[b], 0)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(setQ[b], q + qrow * t0, qrow * L, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(setK[b], k + krow * t0, krow * L, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(setV[b], v + krow * t0, krow * L, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
+        if ((e = cudaEventRecord(h->ev_in[b], h->s_in)) != cudaSuccess) break;
+        // the step, once its inputs are there and the output buffer of the set has been copied back (chunk c-2)
+        if ((e = cudaStreamWaitEvent(st, h->ev_in[b], 0)) != cudaSuccess) break;
+        if (c >= 2 && (e = cudaStreamWaitEvent(st, h->ev_out[b], 0)) != cudaSuccess) break;
+        const bool with_instr = !h->standard || c == n_chunks - 1;
+        rc = run_step(h, layer, seq_slot, setQ[b], setK[b], setV[b], L, with_instr ? h->stQi : nullptr, with_instr ? n_instr : 0,
+                      setO[b], st);
+        if (rc != CITRUS_OK) break;
+        if ((e = cudaEventRecord(h->ev_step[b], st)) != cudaSuccess) break;
+        // its output back to the host
+        if ((e = cudaStreamWaitEvent(h->s_out, h->ev_step[b], 0)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(o + qrow * t0, setO[b], qrow * L, cudaMemcpyDeviceToHost, h->s_out)) != cudaSuccess) break;
+        if ((e = cudaEventRecord(h->ev_out[b], h->s_out)) != cudaSuccess) break;
+    }
+    // whatever was enqueued is drained before returning, also after an error
+    cudaError_t e1 = cudaStreamSynchronize(h->s_in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(h->s_out);
+    if (rc != CITRUS_OK) return rc;
+    if (e != cudaSuccess) return cuda_rc(e);
+    if (e1 != cudaSuccess) return cuda_rc(e1);
+    if (e2 != cudaSuccess) return cuda_rc(e2);
+    return cuda_rc(e3);
+}
+
 int citrus_cache_view(citrus_handle h, int layer, int which, int seq_slot,
                       const void** K, const void** V, const int** positions, int* n_rows) {
     if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
@@ -554,6 +648,7 @@ int citrus_destroy(citrus_handle h) {
     }
     cudaDeviceSynchronize();
     for (const citrus_ctx::Timed& t : h->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+    free_copy_streams(h);
     free_all(h);
     cudaGetLastError();
     delete h;

@@ -343,6 +343,29 @@ def test_host_buffer_variant_matches_device_variant():
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("mode", ["shared", "standard"])
+def test_whole_document_host_call_matches_chunk_by_chunk_device_calls(mode):
+    # copies of chunk c+1 and c-1 overlap the step of chunk c inside the library; results must not notice
+    w = wl.scaled(C["mistral7b_layer"], doc_tokens=5 * 512 + 77, mode=mode)
+    doc = wl.make_document(w)
+    a, b = pu.make_pair(w), pu.make_pair(w)
+    N = doc.Q.shape[0]
+    bounds = [(s, min(N, s + w.chunk_s)) for s in range(0, N, w.chunk_s)]
+    outs = []
+    for i, (s, e) in enumerate(bounds):
+        qi = doc.Q_instr.cuda() if (mode != "standard" or i == len(bounds) - 1) else None
+        outs.append(a.process_chunk(0, doc.Q[s:e].cuda(), doc.K[s:e].cuda(), doc.V[s:e].cuda(), qi).cpu())
+    oh = torch.empty_like(doc.Q).pin_memory()
+    for rep in range(2):                                   # the second document reuses the copy streams and events
+        b.reset()
+        oh.zero_()
+        b.process_document_host(0, doc.Q.pin_memory(), doc.K.pin_memory(), doc.V.pin_memory(), doc.Q_instr.pin_memory(), oh)
+        assert torch.equal(torch.cat(outs), oh)
+        for x, y in zip(a.cache_view(0), b.cache_view(0)):
+            assert torch.equal(x, y)
+    a.close(); b.close()
+
+
 def test_reset_and_rerun_is_deterministic():
     # back-to-back replays of the same document must agree bit for bit (no float atomics, no
     # timing-dependent waits); many repeats, because a missed wait only shows up now and then
