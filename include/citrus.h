@@ -174,9 +174,9 @@ int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,
  * (any number: the document is cut into chunks of chunk_s tokens, the last one shorter), Qih the n_instr
  * instruction queries that score every chunk (STANDARD contexts: only the last chunk, as in citrus_process_chunk
  * with n_instr = 0 before it).  The unit continues from its current state (citrus_reset starts a new document).
- * Chunk c+1's inputs are copied to the device and chunk c-1's output is copied back while chunk c is computed:
- * two staging sets and two copy streams owned by the context, created by the first call (make that call outside any
- * stream capture).  Returns when out_h is complete.  Errors: as citrus_process_chunk; nothing is enqueued if the
+ * The document moves in blocks of four chunks: the next block's inputs are copied to the device and the previous
+ * block's output is copied back while the current block is computed - two staging sets and two copy streams owned
+ * by the context, created by the first call (make that call outside any stream capture).  Returns when out_h is complete.  Errors: as citrus_process_chunk; nothing is enqueued if the
  * arguments are rejected.
  */
 int citrus_process_document_host(citrus_handle h, int layer, int seq_slot,

@@ -66,8 +66,9 @@ struct citrus_ctx {
     std::vector<Timed> timed;
     // staging of the host-buffer variant
     void *stQ = nullptr, *stK = nullptr, *stV = nullptr, *stQi = nullptr, *stOut = nullptr;
-    // whole-document host variant: a second staging set, two copy streams, events per set
-    void *st2Q = nullptr, *st2K = nullptr, *st2V = nullptr, *st2Out = nullptr;
+    // whole-document host variant: two staging sets of a few chunks each, two copy streams, events per set
+    void *docQ[2] = {nullptr, nullptr}, *docK[2] = {nullptr, nullptr}, *docV[2] = {nullptr, nullptr}, *docOut[2] = {nullptr, nullptr};
+    void* docQi = nullptr;
     cudaStream_t s_in = nullptr, s_out = nullptr;
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_step[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr}, ev_qi = nullptr;
 };
@@ -499,19 +500,18 @@ int citrus_process_document_host(citrus_handle h, int layer, int seq_slot,
     }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const size_t qrow = (size_t)h->Hq * h->D * h->elt, krow = (size_t)h->Hkv * h->D * h->elt;
-    if (h->stQ == nullptr) {
-        if ((rc = dev_alloc(h, &h->stQ, qrow * h->ls, false, true))) return rc;
-        if ((rc = dev_alloc(h, &h->stOut, qrow * h->ls, false, true))) return rc;
-        if ((rc = dev_alloc(h, &h->stK, krow * h->ls, false, true))) return rc;
-        if ((rc = dev_alloc(h, &h->stV, krow * h->ls, false, true))) return rc;
-        if ((rc = dev_alloc(h, &h->stQi, qrow * CITRUS_MAX_INSTR, false, true))) return rc;
-    }
+    // Copies move kDocBlock chunks at a time: a few large transfers use the link better than many small ones.
+    constexpr int kDocBlock = 4;
+    const size_t blk_rows = (size_t)h->ls * kDocBlock;
     cudaError_t e = cudaSuccess;
     if (h->s_in == nullptr) {
-        if ((rc = dev_alloc(h, &h->st2Q, qrow * h->ls, false, true))) return rc;
-        if ((rc = dev_alloc(h, &h->st2Out, qrow * h->ls, false, true))) return rc;
-        if ((rc = dev_alloc(h, &h->st2K, krow * h->ls, false, true))) return rc;
-        if ((rc = dev_alloc(h, &h->st2V, krow * h->ls, false, true))) return rc;
+        for (int b = 0; b < 2; ++b) {
+            if ((rc = dev_alloc(h, &h->docQ[b], qrow * blk_rows, false, true))) return rc;
+            if ((rc = dev_alloc(h, &h->docOut[b], qrow * blk_rows, false, true))) return rc;
+            if ((rc = dev_alloc(h, &h->docK[b], krow * blk_rows, false, true))) return rc;
+            if ((rc = dev_alloc(h, &h->docV[b], krow * blk_rows, false, true))) return rc;
+        }
+        if ((rc = dev_alloc(h, &h->docQi, qrow * CITRUS_MAX_INSTR, false, true))) return rc;
         e = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking);
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking);
         for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
@@ -522,37 +522,40 @@ int citrus_process_document_host(citrus_handle h, int layer, int seq_slot,
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_qi, cudaEventDisableTiming);
         if (e != cudaSuccess) return cuda_rc(e);
     }
-    void* setQ[2] = {h->stQ, h->st2Q}; void* setK[2] = {h->stK, h->st2K};
-    void* setV[2] = {h->stV, h->st2V}; void* setO[2] = {h->stOut, h->st2Out};
     const char *q = reinterpret_cast<const char*>(Qh), *k = reinterpret_cast<const char*>(Kh), *v = reinterpret_cast<const char*>(Vh);
     char* o = reinterpret_cast<char*>(out_h);
     // the copy streams start behind whatever the caller's stream already holds
     if ((e = cudaEventRecord(h->ev_qi, st)) != cudaSuccess) return cuda_rc(e);
     if ((e = cudaStreamWaitEvent(h->s_in, h->ev_qi, 0)) != cudaSuccess) return cuda_rc(e);
     if ((e = cudaStreamWaitEvent(h->s_out, h->ev_qi, 0)) != cudaSuccess) return cuda_rc(e);
-    if ((e = cudaMemcpyAsync(h->stQi, Qih, qrow * n_instr, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) return cuda_rc(e);
+    if ((e = cudaMemcpyAsync(h->docQi, Qih, qrow * n_instr, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) return cuda_rc(e);
     const long long n_chunks = (n_tokens + h->ls - 1) / h->ls;
-    for (long long c = 0; c < n_chunks && rc == CITRUS_OK; ++c) {
-        const int b = (int)(c & 1);
-        const long long t0 = c * h->ls;
-        const int L = (int)(n_tokens - t0 < h->ls ? n_tokens - t0 : h->ls);
-        // inputs of chunk c into set b, once the step that last read the set (chunk c-2) is done
-        if (c >= 2 && (e = cudaStreamWaitEvent(h->s_in, h->ev_step[b], 0)) != cudaSuccess) break;
-        if ((e = cudaMemcpyAsync(setQ[b], q + qrow * t0, qrow * L, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
-        if ((e = cudaMemcpyAsync(setK[b], k + krow * t0, krow * L, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
-        if ((e = cudaMemcpyAsync(setV[b], v + krow * t0, krow * L, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
+    const long long n_blocks = (n_chunks + kDocBlock - 1) / kDocBlock;
+    for (long long blk = 0; blk < n_blocks && rc == CITRUS_OK && e == cudaSuccess; ++blk) {
+        const int b = (int)(blk & 1);
+        const long long t0 = blk * (long long)blk_rows;
+        const long long rows = n_tokens - t0 < (long long)blk_rows ? n_tokens - t0 : (long long)blk_rows;
+        // inputs of the block into set b, once the steps that last read the set (block blk-2) are done
+        if (blk >= 2 && (e = cudaStreamWaitEvent(h->s_in, h->ev_step[b], 0)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(h->docQ[b], q + qrow * t0, qrow * rows, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(h->docK[b], k + krow * t0, krow * rows, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(h->docV[b], v + krow * t0, krow * rows, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess) break;
         if ((e = cudaEventRecord(h->ev_in[b], h->s_in)) != cudaSuccess) break;
-        // the step, once its inputs are there and the output buffer of the set has been copied back (chunk c-2)
+        // the block's steps, once its inputs are there and the set's output buffer has been copied back (block blk-2)
         if ((e = cudaStreamWaitEvent(st, h->ev_in[b], 0)) != cudaSuccess) break;
-        if (c >= 2 && (e = cudaStreamWaitEvent(st, h->ev_out[b], 0)) != cudaSuccess) break;
-        const bool with_instr = !h->standard || c == n_chunks - 1;
-        rc = run_step(h, layer, seq_slot, setQ[b], setK[b], setV[b], L, with_instr ? h->stQi : nullptr, with_instr ? n_instr : 0,
-                      setO[b], st);
+        if (blk >= 2 && (e = cudaStreamWaitEvent(st, h->ev_out[b], 0)) != cudaSuccess) break;
+        for (long long r0 = 0; r0 < rows && rc == CITRUS_OK; r0 += h->ls) {
+            const int L = (int)(rows - r0 < h->ls ? rows - r0 : h->ls);
+            const bool last = t0 + r0 + L == n_tokens;
+            const bool with_instr = !h->standard || last;
+            rc = run_step(h, layer, seq_slot, (char*)h->docQ[b] + qrow * r0, (char*)h->docK[b] + krow * r0, (char*)h->docV[b] + krow * r0, L,
+                          with_instr ? h->docQi : nullptr, with_instr ? n_instr : 0, (char*)h->docOut[b] + qrow * r0, st);
+        }
         if (rc != CITRUS_OK) break;
         if ((e = cudaEventRecord(h->ev_step[b], st)) != cudaSuccess) break;
         // its output back to the host
         if ((e = cudaStreamWaitEvent(h->s_out, h->ev_step[b], 0)) != cudaSuccess) break;
-        if ((e = cudaMemcpyAsync(o + qrow * t0, setO[b], qrow * L, cudaMemcpyDeviceToHost, h->s_out)) != cudaSuccess) break;
+        if ((e = cudaMemcpyAsync(o + qrow * t0, h->docOut[b], qrow * rows, cudaMemcpyDeviceToHost, h->s_out)) != cudaSuccess) break;
         if ((e = cudaEventRecord(h->ev_out[b], h->s_out)) != cudaSuccess) break;
     }
     // whatever was enqueued is drained before returning, also after an error
