@@ -81,6 +81,13 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         for (int j = tid; j < n; j += kSelThreads) {
             for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * ks + j] = j;
             also(j, j);
+            if (job.carried != nullptr && j < job.m) {
+                // accumulative policy: the carried importance still has to be added to what is handed on
+                for (int ho = 0; ho < heads_out; ++ho) {
+                    const int gg = layerwise ? ho : g;
+                    job.scores[(size_t)gg * job.score_stride + j] += job.carried[(size_t)gg * job.pos_stride + j];
+                }
+            }
         }
         return;
     }

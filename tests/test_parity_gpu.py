@@ -266,6 +266,37 @@ def test_config5_long_document_sampled():
     ctx.close()
 
 
+@pytest.mark.parametrize("seed", range(32))
+def test_random_small_configurations(seed):
+    # seeded draws over head geometry, budget, chunk lengths, instruction length, mode and policy bits
+    rng = np.random.default_rng(1000 + seed)
+    kv = int(rng.choice([1, 2, 4]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    dtype = "bf16" if seed % 4 else "fp32"
+    D = 128 if dtype == "bf16" else int(rng.choice([64, 128]))
+    mode = str(rng.choice(["shared", "individual", "standard"]))
+    ls = int(rng.integers(40, 400))
+    k = int(rng.integers(20, 500))
+    n_chunks = int(rng.integers(3, 7))
+    lengths = [int(rng.integers(1, ls + 1)) for _ in range(n_chunks)]
+    lengths[int(rng.integers(0, n_chunks))] = ls
+    flags = dict(accumulate=bool(rng.integers(0, 2)), start_size=int(rng.choice([0, 0, 3])) if k >= 3 else 0)
+    variant = int(rng.integers(0, 3))
+    if variant == 1 and mode != "shared":
+        flags["deferred_lm"] = True
+    elif variant == 2:
+        flags["position_shift"] = True
+    layerwise = bool(rng.integers(0, 4) == 0)
+    w = wl.scaled(C["tiny_fp32"], seed=2000 + seed, q_heads=kv * G, kv_heads=kv, head_dim=D, budget_k=k, chunk_s=ls,
+                  doc_tokens=sum(lengths), n_instr=int(rng.integers(1, 150)), dtype=dtype, mode=mode,
+                  lm_window=int(rng.choice([0, 1, 17, 64])), n_planted=3, n_sinks=int(rng.integers(0, 2)), **flags)
+    ctx = pu.make_pair(w, layerwise=layerwise)
+    _, st = pu.run_document(w, ctx, chunk_lengths=lengths, layerwise=layerwise)
+    _report(f"random {seed}: {mode} {dtype} D{D} heads {kv * G}/{kv} k {k} l_s {ls} {flags} layerwise={layerwise}", st)
+    assert st["checked_chunks"] == n_chunks and ctx.poll_status() == 0
+    ctx.close()
+
+
 def test_maximum_candidates_and_instruction_rows():
     # the largest step the library accepts: budget + chunk = 49152 candidates, 4096 instruction queries.  Six full
     # chunks are property-checked (row counts, ascending positions, rows bit-equal to the document's); the sixth has
