@@ -297,6 +297,35 @@ def test_random_small_configurations(seed):
     ctx.close()
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_random_medium_configurations(seed):
+    # more heads, several instruction row tiles, budgets of a few key tiles with ragged edges (bf16 tensor-core path)
+    rng = np.random.default_rng(5000 + seed)
+    kv = int(rng.choice([2, 4, 8]))
+    G = int(rng.choice([1, 2, 4]))
+    mode = str(rng.choice(["shared", "individual", "standard"]))
+    ls = int(rng.choice([128, 256, 300, 512, 640]))
+    k = int(rng.integers(100, 1500))
+    n_chunks = int(rng.integers(3, 6))
+    lengths = [ls] * (n_chunks - 1) + [int(rng.integers(1, ls + 1))]
+    flags = {}
+    variant = int(rng.integers(0, 4))
+    if variant == 1 and mode != "shared":
+        flags["deferred_lm"] = True
+    elif variant == 2:
+        flags["position_shift"] = True
+    elif variant == 3:
+        flags["accumulate"] = True
+    w = wl.scaled(C["tiny_fp32"], seed=6000 + seed, q_heads=kv * G, kv_heads=kv, head_dim=128, budget_k=k, chunk_s=ls,
+                  doc_tokens=sum(lengths), n_instr=int(rng.choice([8, 64, 100, 128, 200, 520])), dtype="bf16", mode=mode,
+                  lm_window=int(rng.choice([0, 64, 200])), n_planted=8, n_sinks=1, **flags)
+    ctx = pu.make_pair(w)
+    _, st = pu.run_document(w, ctx, chunk_lengths=lengths)
+    _report(f"random medium {seed}: {mode} heads {kv * G}/{kv} k {k} l_s {ls} n_I {w.n_instr} w {w.lm_window} {flags}", st)
+    assert st["checked_chunks"] == n_chunks and ctx.poll_status() == 0
+    ctx.close()
+
+
 def test_maximum_candidates_and_instruction_rows():
     # the largest step the library accepts: budget + chunk = 49152 candidates, 4096 instruction queries.  Six full
     # chunks are property-checked (row counts, ascending positions, rows bit-equal to the document's); the sixth has
