@@ -29,12 +29,12 @@ __device__ __forceinline__ uint4 rope_piece(uint4 mine, uint4 other, int pos, in
     const uint32_t* b = reinterpret_cast<const uint32_t*>(&other);
     uint4 out;
     uint32_t* o = reinterpret_cast<uint32_t*>(&out);
+    // fp64 throughout, rounded once at the end: the embedded value is the correctly rounded rotation of the stored
+    // one (up to the last bit of sin / cos), whatever the position
     auto turn = [&](float x, float y, int d) {
-        double ang = (double)pos * t.theta[d];
-        ang -= 6.283185307179586 * floor(ang * 0.15915494309189535);     // into [0, 2 pi) before the fp32 sincos
-        float sn, cs;
-        sincosf((float)ang, &sn, &cs);
-        return lower ? x * cs - y * sn : x * cs + y * sn;
+        double sn, cs;
+        sincos((double)pos * t.theta[d], &sn, &cs);
+        return (float)(lower ? (double)x * cs - (double)y * sn : (double)x * cs + (double)y * sn);
     };
     if (elt == 2) {
 #pragma unroll
