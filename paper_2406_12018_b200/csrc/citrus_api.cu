@@ -214,8 +214,9 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         Qc = c->rotQ; Kc = c->rotK; if (instr_scoring) Qi = c->rotQi;
         for (int ci = 0; ci < c->n_caches; ++ci) cand[ci].chunkK = Kc;
     }
-    QueryRows q_chunk{Qc, L, c->Hq, 1, 0};
-    QueryRows q_instr{Qi, nI, c->Hq, 0, 0};
+    const int produced = c->shift ? 1 : 0;    // the embedding pre-pass above wrote Qc, Kc and Qi
+    QueryRows q_chunk{Qc, L, c->Hq, 1, 0, produced};
+    QueryRows q_instr{Qi, nI, c->Hq, 0, 0, produced};
     float* scores[2] = {u.scores, u.scores + (size_t)c->Hkv * c->score_stride};
     const int ic = c->individual ? 1 : 0;     // the cache scored by the instruction text
     if (!instr_scoring) q_instr.rows = 0;
@@ -244,7 +245,7 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     if (lm_scoring) {
         int w = c->lm_window > 0 && c->lm_window < L ? c->lm_window : L;
         const char* q0 = reinterpret_cast<const char*>(Qc) + (size_t)(L - w) * c->Hq * c->D * c->elt;
-        QueryRows q_lm{q0, w, c->Hq, 1, L - w};
+        QueryRows q_lm{q0, w, c->Hq, 1, L - w, produced};
         LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
         if (c->use_tc) e = tc_colsum(q_lm, cand[0], u.lse_chunk + (L - w), c->ls, 1, scores[0], c->score_stride, c->status, st);
         else e = simt_colsum(c->fp32, c->D, q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, st);

@@ -45,6 +45,8 @@ struct QueryRows {
     int q_heads;
     int causal;   // 1: row r sees chunk candidates u <= t0 + r only
     int t0;       // chunk index of row 0 (causal only)
+    int produced; // 1: Q and the chunk's keys were written by a kernel earlier in the stream (position shift), so a
+                  // kernel launched with programmatic serialization must wait for its predecessors before ANY load
 };
 
 // ---- SIMT (true fp32 arithmetic) path ------------------------------------

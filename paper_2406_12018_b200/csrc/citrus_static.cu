@@ -69,13 +69,13 @@ extern "C" int citrus_importance_static(const void* Q_s, int n_s, const void* K,
     }
     // all candidates are "chunk" rows of a token-major tensor; there is no retained cache (m = 0)
     Candidates cand{K, K, K, K, 0, n_keys, n_keys, kv_heads};
-    QueryRows q{Q_s, n_s, q_heads, 0, 0};
+    QueryRows q{Q_s, n_s, q_heads, 0, 0, 0};
     cudaError_t e;
     if (fp32) {
         e = simt_attention(true, head_dim, q, cand, nullptr, lse, lse_stride, st);
         if (e == cudaSuccess) e = simt_colsum(true, head_dim, q, cand, lse, lse_stride, scores, score_stride, st);
     } else {
-        const QueryRows none{nullptr, 0, q_heads, 0, 0};
+        const QueryRows none{nullptr, 0, q_heads, 0, 0, 0};
         e = tc_attention_lse(none, cand, nullptr, nullptr, 0, q, cand, lse, nullptr, lse_stride, 1, status, st);
         if (e == cudaSuccess) e = tc_colsum(q, cand, lse, lse_stride, 1, scores, score_stride, status, st);
     }

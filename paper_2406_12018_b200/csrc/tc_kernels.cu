@@ -233,6 +233,7 @@ struct TcParams {
     float* scores;   // colsum: [kv_heads, score_stride]
     int score_stride;
     int* status;
+    int dep_first;   // the queries and the chunk's keys come from a preceding kernel: wait for it before the first load
 };
 
 // Load one 128x128 bf16 tile as two swizzled halves.  token_major: coordinates (d, head, row);
@@ -379,6 +380,8 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
     // still does.  The chunk's own tiles come first in the sweep and need nothing from it, so only two things
     // wait for the predecessor (griddepcontrol.wait): the first load of a retained-cache tile, and the
     // log-sum-exp writes of the epilogue (the previous chunk's column-sum kernel may still be reading them).
+    // Exception (p.dep_first): with the position shift the queries and the chunk's keys are written by the
+    // embedding pre-pass launched just before, so the Q/K producer waits before its first load.
     // Sweep order: tile index jg(j) = chunk tiles first, then cache tiles.
     auto sweep_tile = [&](int j) {
         const int t = tile_begin + j;
@@ -392,6 +395,8 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
 
     if (warp == 8) {
         // ---------------------------------------------------------------- K (and Q) TMA producer (converged warp)
+        bool dep_waited = false;
+        if (p.dep_first) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
         if (!WITH_PV && p.pack > 1) {
             // several heads' scoring rows side by side in one tile (mapQ's box is pack_rows rows high)
             if (elect_one()) {
@@ -406,7 +411,6 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
         } else {
             load_tile(sQ, &mapQ, smem_u32(&bars->q_full), p.row0 + q_row0, h, true);
         }
-        bool dep_waited = false;
         for (int j = 0; j < nt; ++j) {
             const int s = j % kStagesK, jg = sweep_tile(j);
             const bool from_cache = jg < n_cache_tiles;
@@ -764,7 +768,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     // Programmatic dependent launch: the scoring queries and the chunk's keys are the caller's inputs and are loaded
-    // at once; what the preceding kernels produce is touched only after griddepcontrol.wait - a retained-cache
+    // at once (unless p.dep_first says that a preceding kernel wrote them: then the producer waits first); what the preceding kernels produce is touched only after griddepcontrol.wait - a retained-cache
     // tile (written by the previous chunk's compaction), the log-sum-exp values of pass 1, and the score vector
     // (still read by the previous chunk's select until that kernel has ended).
     const uint32_t tmem = bars->tmem_base;
@@ -782,8 +786,9 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         };
         bool ok = true;
         int it = 0;
+        if (p.dep_first) asm volatile("griddepcontrol.wait;" ::: "memory");
         for (; it < nb && it < kColStages && ok; ++it) ok = load_q(it);
-        if (from_cache) asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (from_cache && !p.dep_first) asm volatile("griddepcontrol.wait;" ::: "memory");
         load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
         for (; it < nb && ok; ++it) ok = load_q(it);
     } else if (warp == 9) {
@@ -977,7 +982,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t 
 TcParams base_params(const QueryRows& q, const Candidates& c, int* status) {
     TcParams p{};
     p.rows = q.rows; p.row0 = 0; p.q_heads = q.q_heads; p.kv_heads = c.kv_heads;
-    p.m = c.m; p.L = c.L; p.causal = q.causal; p.t0 = q.t0; p.status = status;
+    p.m = c.m; p.L = c.L; p.causal = q.causal; p.t0 = q.t0; p.status = status; p.dep_first = q.produced;
     return p;
 }
 

@@ -266,7 +266,8 @@ def test_config5_long_document_sampled():
     ctx.close()
 
 
-@pytest.mark.parametrize("seed", range(32))
+# (seeds past the first 32 / 12 are configurations on which a wider sweep once found a fault: kept as regressions)
+@pytest.mark.parametrize("seed", list(range(32)) + [182, 343])
 def test_random_small_configurations(seed):
     # seeded draws over head geometry, budget, chunk lengths, instruction length, mode and policy bits
     rng = np.random.default_rng(1000 + seed)
@@ -297,7 +298,7 @@ def test_random_small_configurations(seed):
     ctx.close()
 
 
-@pytest.mark.parametrize("seed", range(12))
+@pytest.mark.parametrize("seed", list(range(12)) + [16, 25, 115])
 def test_random_medium_configurations(seed):
     # more heads, several instruction row tiles, budgets of a few key tiles with ragged edges (bf16 tensor-core path)
     rng = np.random.default_rng(5000 + seed)
