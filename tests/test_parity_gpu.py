@@ -327,6 +327,43 @@ def test_random_medium_configurations(seed):
     ctx.close()
 
 
+@pytest.mark.parametrize("seed", [0, 2, 5, 18, 24, 30, 41, 47])
+def test_random_large_configurations(seed):
+    # several waves of attention items, split log-sum-exp passes, the two-kernel select / gather route; the oracle
+    # follows the last two chunks (every chunk under the accumulative policy, whose carried scores it has to track)
+    rng = np.random.default_rng(9000 + seed)
+    kv = int(rng.choice([4, 8, 16, 32]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    while kv * G > 64:
+        G //= 2
+    mode = str(rng.choice(["shared", "individual", "standard"]))
+    ls = int(rng.choice([700, 1024, 1500, 2048, 3000]))
+    k = int(rng.integers(500, 6000))
+    n_chunks = int(rng.integers(2, 5))
+    lengths = [ls] * (n_chunks - 1) + [int(rng.integers(1, ls + 1))]
+    flags = {}
+    variant = int(rng.integers(0, 5))
+    if variant == 1 and mode != "shared":
+        flags["deferred_lm"] = True
+    elif variant == 2:
+        flags["position_shift"] = True
+    elif variant == 3:
+        flags["accumulate"] = True
+    elif variant == 4:
+        flags["start_size"] = 4
+    layerwise = bool(rng.integers(0, 6) == 0)
+    n_instr = int(rng.choice([16, 64, 128, 256, 300, 1000]))
+    w = wl.scaled(C["tiny_fp32"], seed=9500 + seed, q_heads=kv * G, kv_heads=kv, head_dim=128, budget_k=k, chunk_s=ls,
+                  doc_tokens=sum(lengths), n_instr=n_instr, dtype="bf16", mode=mode,
+                  lm_window=int(rng.choice([0, 64, 500])), n_planted=16, n_sinks=2, **flags)
+    ctx = pu.make_pair(w, layerwise=layerwise)
+    followed = "all" if flags.get("accumulate") else {n_chunks - 2, n_chunks - 1}
+    _, st = pu.run_document(w, ctx, chunk_lengths=lengths, layerwise=layerwise, oracle_chunks=followed)
+    _report(f"random large {seed}: {mode} heads {kv * G}/{kv} k {k} l_s {ls} n_I {n_instr} {flags} layerwise={layerwise}", st)
+    assert st["checked_chunks"] >= min(2, n_chunks) and ctx.poll_status() == 0
+    ctx.close()
+
+
 def test_maximum_candidates_and_instruction_rows():
     # the largest step the library accepts: budget + chunk = 49152 candidates, 4096 instruction queries.  Six full
     # chunks are property-checked (row counts, ascending positions, rows bit-equal to the document's); the sixth has
@@ -425,6 +462,64 @@ def test_whole_document_host_call_matches_chunk_by_chunk_device_calls(mode):
         for x, y in zip(a.cache_view(0), b.cache_view(0)):
             assert torch.equal(x, y)
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_pipelined_replays_equal_the_synchronised_run(seed):
+    # Consecutive kernels overlap (programmatic dependent launch), so every mode and policy is replayed without host
+    # synchronisation between chunks and compared bit for bit with a run that synchronises after every chunk:
+    # outputs, both caches, positions, last scores and kept indices.
+    rng = np.random.default_rng(77000 + seed)
+    kv = int(rng.choice([2, 8, 16]))
+    G = int(rng.choice([1, 4]))
+    mode = str(rng.choice(["shared", "individual", "standard"]))
+    dtype = "bf16" if seed % 5 else "fp32"
+    ls = int(rng.choice([128, 256, 512, 640, 1024, 2048])) if dtype == "bf16" else int(rng.choice([64, 128, 200]))
+    k = int(rng.integers(100, 3000)) if dtype == "bf16" else int(rng.integers(50, 400))
+    n_chunks = int(rng.integers(4, 9))
+    lengths = [ls] * (n_chunks - 1) + [int(rng.integers(1, ls + 1))]
+    flags = {}
+    variant = int(rng.integers(0, 5))
+    if variant == 1 and mode != "shared":
+        flags["deferred_lm"] = True
+    elif variant == 2:
+        flags["position_shift"] = True
+    elif variant == 3:
+        flags["accumulate"] = True
+    elif variant == 4:
+        flags["start_size"] = 4
+    layerwise = bool(rng.integers(0, 5) == 0)
+    w = wl.scaled(C["tiny_fp32"], seed=77500 + seed, q_heads=kv * G, kv_heads=kv, head_dim=128, budget_k=k, chunk_s=ls,
+                  doc_tokens=sum(lengths), n_instr=int(rng.choice([16, 64, 128, 300])), dtype=dtype, mode=mode,
+                  lm_window=int(rng.choice([0, 64])), n_planted=4, n_sinks=1, **flags)
+    doc = wl.make_document(w)
+    ctx = pu.make_pair(w, layerwise=layerwise)
+    Q, K, V, Qi = doc.Q.cuda(), doc.K.cuda(), doc.V.cuda(), doc.Q_instr.cuda()
+    bounds = np.cumsum([0] + lengths)
+
+    def run(sync):
+        ctx.reset()
+        outs = []
+        for ci in range(n_chunks):
+            sl = slice(int(bounds[ci]), int(bounds[ci + 1]))
+            with_instr = mode != "standard" or ci == n_chunks - 1
+            outs.append(ctx.process_chunk(0, Q[sl], K[sl], V[sl], Qi if with_instr else None))
+            if sync:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        res = [torch.cat(outs).clone()]
+        for cid in range(2 if mode == "individual" else 1):
+            Kc, Vc, P = ctx.cache_view(0, cid)
+            S, I, _ = ctx.step_view(0, cid)
+            res += [Kc.clone(), Vc.clone(), P.clone(), S.clone(), I.clone()]
+        return res
+
+    ref = run(True)
+    for rep in range(12):
+        for i, (x, y) in enumerate(zip(ref, run(False))):
+            assert torch.equal(x, y), f"replay {rep}: tensor {i} differs"
+    assert ctx.poll_status() == 0
+    ctx.close()
 
 
 def test_reset_and_rerun_is_deterministic():
