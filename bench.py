@@ -57,7 +57,11 @@ class ClockSampler:
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, device_index: int):
-        self.idx = device_index
+        # nvidia-smi numbers the GPUs of the machine, CUDA those that are visible to the process: ask by UUID
+        try:
+            self.idx = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+        except Exception:
+            self.idx = device_index
         self.lines = []
         self.proc = None
 
@@ -72,9 +76,16 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
-    def stop(self):
+    def wait_first_sample(self, timeout_s: float = 10.0):
+        """nvidia-smi needs a moment to start: return once it has printed its first line."""
+        t_end = time.time() + timeout_s
+        while self.proc is not None and not self.lines and time.time() < t_end:
+            time.sleep(0.05)
+
+    def stop(self, t_begin: float = 0.0, t_end: float = float("inf")):
+        """Summary of the samples taken in [t_begin, t_end] (host clock), the timed region."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -84,7 +95,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for stamp, ln in self.lines:
+            if not (t_begin <= stamp <= t_end):
+                continue
             parts = [x.strip() for x in ln.split(",")]
             if len(parts) < 9:
                 continue
@@ -232,19 +245,21 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
 
     with torch.cuda.stream(stream):
-        for _ in range(args.warmup):
-            step()
-        barrier()
         sampler = ClockSampler(local_rank)
         if rank == 0:
             sampler.start()
+            sampler.wait_first_sample()
+        for _ in range(args.warmup):
+            step()
+        barrier()
+        t_begin = time.time()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record(stream)
         for _ in range(args.steps):
             step()
         ev1.record(stream)
         barrier()
-        clocks = sampler.stop() if rank == 0 else None
+        clocks = sampler.stop(t_begin, time.time()) if rank == 0 else None
     ms_total = ev0.elapsed_time(ev1)
     ms_total = max_over_ranks(ms_total, dist, "cuda")
     ms_per_step = ms_total / args.steps
@@ -346,7 +361,7 @@ def run_ours(args, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=WORKLOAD,
