@@ -29,7 +29,7 @@ MAX_CANDIDATES = 49152
 KERNEL_NAMES = ["attention", "score_lse", "colsum", "select", "compact", "rope"]
 
 EXPORTS = [
-    "citrus_create", "citrus_set_batch", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
+    "citrus_create", "citrus_set_batch", "citrus_set_batch_lanes", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
     "citrus_process_chunk_host", "citrus_process_document_host", "citrus_process_chunk_batch", "citrus_cache_view", "citrus_step_view", "citrus_profile",
     "citrus_profile_read", "citrus_importance_static", "citrus_intersection_ratio", "citrus_set_rope_base",
     "citrus_poll_status",
@@ -57,6 +57,7 @@ def load() -> C.CDLL:
     vp, i = C.c_void_p, C.c_int
     lib.citrus_create.argtypes = [C.POINTER(vp), i, i, i, i, i, i, C.c_uint]
     lib.citrus_set_batch.argtypes = [vp, i]
+    lib.citrus_set_batch_lanes.argtypes = [vp, i]
     lib.citrus_reset.argtypes = [vp]
     lib.citrus_process_chunk.argtypes = [vp, i, vp, vp, vp, i, vp, i, vp, vp]
     lib.citrus_process_chunk_slot.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, vp]
@@ -156,6 +157,12 @@ class Citrus:
                 raise CitrusError(rc, "citrus_set_batch")
 
     # -- calls -------------------------------------------------------------
+    def set_batch_lanes(self, n_lanes: int):
+        """Side streams of the packed batch call: 0 = chosen per call, 1 = the caller's stream only, up to 8."""
+        rc = load().citrus_set_batch_lanes(self._h, int(n_lanes))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_set_batch_lanes")
+
     def _check(self, t: torch.Tensor, cuda: bool):
         assert t.dtype == self.torch_dtype and t.is_contiguous() and t.is_cuda == cuda
 

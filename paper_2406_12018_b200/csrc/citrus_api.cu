@@ -2,6 +2,7 @@
 // checks, ping-pong cache bookkeeping and the launch sequence of one chunk step.
 #include "../../include/citrus.h"
 #include "citrus_internal.h"
+#include <algorithm>
 
 #include <cmath>
 #include <cstdlib>
@@ -71,6 +72,14 @@ struct citrus_ctx {
     void* docQi = nullptr;
     cudaStream_t s_in = nullptr, s_out = nullptr;
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_step[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr}, ev_qi = nullptr;
+    // ragged batches of small steps: the sequences of one call are dealt to side streams ("lanes") that fork from the
+    // caller's stream and join it again before the call returns, so that the latency chains of different sequences
+    // (a step of a few dozen CTAs leaves most SMs idle) overlap.  0 = chosen per call.
+    static constexpr int kMaxLanes = 8;
+    int lanes_wanted = 0;
+    cudaStream_t lane[kMaxLanes] = {};
+    cudaEvent_t lane_done[kMaxLanes] = {};
+    cudaEvent_t lane_fork = nullptr;
 };
 
 namespace {
@@ -109,6 +118,24 @@ void free_copy_streams(citrus_ctx* c) {
     if (c->ev_qi) cudaEventDestroy(c->ev_qi);
     if (c->s_in) cudaStreamDestroy(c->s_in);
     if (c->s_out) cudaStreamDestroy(c->s_out);
+    for (int i = 0; i < citrus_ctx::kMaxLanes; ++i) {
+        if (c->lane_done[i]) cudaEventDestroy(c->lane_done[i]);
+        if (c->lane[i]) cudaStreamDestroy(c->lane[i]);
+        c->lane_done[i] = nullptr; c->lane[i] = nullptr;
+    }
+    if (c->lane_fork) cudaEventDestroy(c->lane_fork);
+    c->lane_fork = nullptr;
+}
+// Side streams and events of the batch lanes (created once, by citrus_set_batch for more than one slot).
+int make_lanes(citrus_ctx* c) {
+    cudaError_t e = cudaSuccess;
+    if (c->lane_fork == nullptr) e = cudaEventCreateWithFlags(&c->lane_fork, cudaEventDisableTiming);
+    for (int i = 0; i < citrus_ctx::kMaxLanes && e == cudaSuccess; ++i) {
+        if (c->lane[i] == nullptr) e = cudaStreamCreateWithFlags(&c->lane[i], cudaStreamNonBlocking);
+        if (e == cudaSuccess && c->lane_done[i] == nullptr) e = cudaEventCreateWithFlags(&c->lane_done[i], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
+    return CITRUS_OK;
 }
 void free_all(citrus_ctx* c) {
     free_units(c);
@@ -395,6 +422,14 @@ int citrus_set_batch(citrus_handle h, int n_seq) {
             return rc;
         }
     }
+    if (h->n_slots > 1) return make_lanes(h);
+    return CITRUS_OK;
+}
+
+int citrus_set_batch_lanes(citrus_handle h, int n_lanes) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    if (n_lanes < 0 || n_lanes > citrus_ctx::kMaxLanes) return CITRUS_ERR_INVALID_ARG;
+    h->lanes_wanted = n_lanes;
     return CITRUS_OK;
 }
 
@@ -448,17 +483,43 @@ int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const i
         if (u.tokens_seen + L > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
     }
     const size_t qrow = (size_t)h->Hq * h->D * h->elt, krow = (size_t)h->Hkv * h->D * h->elt;   // multiples of 16 bytes
+    cudaStream_t caller = reinterpret_cast<cudaStream_t>(stream);
+    // Lanes: only where a step is small (its attention items fit the SMs at once), which is where a sequence's
+    // kernels wait for each other more than they compute.  The embedding scratch of the position shift is one per
+    // context and per-launch timing wants one stream, so those run in the caller's stream.
+    int n_lanes = 1;
+    if (n_active > 1 && h->lane_fork != nullptr && !h->shift && !h->profiling) {
+        int items = 0;
+        for (int i = 0; i < n_active; ++i) items = std::max(items, (tok_offset[i + 1] - tok_offset[i] + 127) / 128 * h->Hq);
+        n_lanes = h->lanes_wanted > 0 ? h->lanes_wanted : (items <= 148 ? 4 : 1);
+        n_lanes = std::min(n_lanes, n_active);
+    }
+    if (n_lanes > 1) {
+        cudaError_t e = cudaEventRecord(h->lane_fork, caller);
+        for (int l = 0; l < n_lanes && e == cudaSuccess; ++l) e = cudaStreamWaitEvent(h->lane[l], h->lane_fork, 0);
+        if (e != cudaSuccess) return cuda_rc(e);
+    }
+    int first_rc = CITRUS_OK;
     for (int i = 0; i < n_active; ++i) {
+        cudaStream_t st_i = n_lanes > 1 ? h->lane[i % n_lanes] : caller;
         const char* q = reinterpret_cast<const char*>(Q) + qrow * tok_offset[i];
         const char* k = reinterpret_cast<const char*>(K) + krow * tok_offset[i];
         const char* v = reinterpret_cast<const char*>(V) + krow * tok_offset[i];
         const char* qi = reinterpret_cast<const char*>(Q_instr) + qrow * instr_offset[i];
         char* o = reinterpret_cast<char*>(out) + qrow * tok_offset[i];
         int rc = run_step(h, layer, seq_slot[i], q, k, v, tok_offset[i + 1] - tok_offset[i], qi,
-                          instr_offset[i + 1] - instr_offset[i], o, reinterpret_cast<cudaStream_t>(stream));
-        if (rc != CITRUS_OK) return rc;     // only a launch failure can get here; earlier sequences have advanced
+                          instr_offset[i + 1] - instr_offset[i], o, st_i);
+        if (rc != CITRUS_OK) { first_rc = rc; break; }   // only a launch failure can get here; earlier sequences have advanced
     }
-    return CITRUS_OK;
+    if (n_lanes > 1) {
+        // the caller's stream continues only after every lane (also after a failure: nothing is left running unjoined)
+        for (int l = 0; l < n_lanes; ++l) {
+            cudaError_t e = cudaEventRecord(h->lane_done[l], h->lane[l]);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(caller, h->lane_done[l], 0);
+            if (e != cudaSuccess && first_rc == CITRUS_OK) first_rc = cuda_rc(e);
+        }
+    }
+    return first_rc;
 }
 
 int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,

@@ -386,12 +386,15 @@ def test_maximum_candidates_and_instruction_rows():
         Citrus(1, 8, 2, 128, k, ls + 1)                      # one candidate too many
 
 
-def test_ragged_batch_call_matches_per_sequence_calls_and_rejects_bad_batches():
+@pytest.mark.parametrize("lanes", [0, 1, 2])
+def test_ragged_batch_call_matches_per_sequence_calls_and_rejects_bad_batches(lanes):
     # three sequences of the serving mix advance in lock step through the packed call; finished ones drop out
+    # (lanes: 0 = the call deals these small steps to side streams by itself, 1 = caller's stream only, 2 = forced)
     w = wl.scaled(C["serving_mix"], n_seqs=3, budget_k=256, chunk_s=256, n_instr=24, doc_tokens=1024, min_tokens=300)
     lens = [700, 300, 1024]
     docs = [wl.make_document(w, seq=s, n_tokens=n) for s, n in enumerate(lens)]
     a, b = pu.make_pair(w), pu.make_pair(w)
+    a.set_batch_lanes(lanes)
     step = 0
     while True:
         active = [s for s in range(3) if step * w.chunk_s < lens[s]]
@@ -421,6 +424,62 @@ def test_ragged_batch_call_matches_per_sequence_calls_and_rejects_bad_batches():
     with pytest.raises(CitrusError) as e:
         a.process_chunk_batch(0, [0, 1], [0, 300, 310], Q, K, V, [0, 24, 48], Qi)       # chunk longer than chunk_s
     assert e.value.code == -2
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("mode", ["shared", "individual"])
+def test_batch_lanes_in_a_captured_graph_equal_the_single_stream_run(mode):
+    # six ragged sequences through the packed call: once on the caller's stream alone, once dealt to four side
+    # streams and captured into a CUDA graph that is replayed twice; outputs, positions and caches must be identical
+    w = wl.scaled(C["serving_mix"], n_seqs=6, budget_k=300, chunk_s=200, n_instr=40, doc_tokens=1000, min_tokens=150,
+                  mode=mode, lm_window=32)
+    lens = [1000, 431, 777, 150, 999, 600]
+    docs = [wl.make_document(w, seq=s, n_tokens=n) for s, n in enumerate(lens)]
+    steps, step = [], 0
+    while True:
+        active = [s for s in range(len(lens)) if step * w.chunk_s < lens[s]]
+        if not active:
+            break
+        sl = [slice(step * w.chunk_s, min(lens[s], (step + 1) * w.chunk_s)) for s in active]
+        tok = [0]
+        for x in sl:
+            tok.append(tok[-1] + (x.stop - x.start))
+        steps.append((active, tok, torch.cat([docs[s].Q[x] for s, x in zip(active, sl)]).cuda(),
+                      torch.cat([docs[s].K[x] for s, x in zip(active, sl)]).cuda(),
+                      torch.cat([docs[s].V[x] for s, x in zip(active, sl)]).cuda(),
+                      [w.n_instr * i for i in range(len(active) + 1)], torch.cat([docs[s].Q_instr for s in active]).cuda()))
+        step += 1
+    a, b = pu.make_pair(w), pu.make_pair(w)
+    a.set_batch_lanes(1)
+    b.set_batch_lanes(4)
+    ref = [a.process_chunk_batch(0, act, tok, Q, K, V, ins, Qi) for act, tok, Q, K, V, ins, Qi in steps]
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    outs = [torch.empty_like(r) for r in ref]
+
+    def document():
+        b.reset()
+        for (act, tok, Q, K, V, ins, Qi), o in zip(steps, outs):
+            b.process_chunk_batch(0, act, tok, Q, K, V, ins, Qi, out=o, stream=stream)
+
+    with torch.cuda.stream(stream):
+        document()                                   # one-time set-up happens outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        document()
+    for _ in range(2):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for o, r in zip(outs, ref):
+            assert torch.equal(o, r)
+        for s in range(len(lens)):
+            for which in range(2 if mode == "individual" else 1):
+                for x, y in zip(a.cache_view(0, which, s), b.cache_view(0, which, s)):
+                    assert torch.equal(x, y)
+    assert a.poll_status() == 0 and b.poll_status() == 0
     a.close(); b.close()
 
 
