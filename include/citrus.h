@@ -119,7 +119,7 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
 int citrus_set_batch(citrus_handle h, int n_seq);
 
 /* Side streams used by citrus_process_chunk_batch (Section 4 has no counterpart: the paper processes one document at
- * a time).  n_lanes = 0 (default) lets each call choose (four for small steps, one otherwise); 1 enqueues every
+ * a time).  n_lanes = 0 (default) lets each call choose (four for the smallest steps, two for medium ones, one otherwise); 1 enqueues every
  * sequence on the caller's stream; up to 8.  May be changed between calls.  Errors: INVALID_ARG. */
 int citrus_set_batch_lanes(citrus_handle h, int n_lanes);
 
@@ -157,8 +157,8 @@ int citrus_process_chunk_slot(citrus_handle h, int layer, int seq_slot,
  * (n_active, n_active + 1 and n_active + 1 ints); the tensors are device pointers as in citrus_process_chunk.
  * Every sequence's chunk obeys the single-call rules (1..chunk_s tokens, 1..CITRUS_MAX_INSTR instruction rows,
  * distinct slots).  All arguments are validated before anything is enqueued; sequences are independent (no state
- * is shared between slots).  Where every sequence's step is small (its attention items fit the SMs at once) the
- * sequences are dealt to side streams owned by the context, which fork from `stream` when the call starts and join
+ * is shared between slots).  Where every sequence's step is small (its attention items make at most about three
+ * waves over the SMs) the sequences are dealt to side streams owned by the context, which fork from `stream` when the call starts and join
  * it again before the call returns: to the caller the call is still one piece of work on `stream` (it can be captured
  * in a CUDA graph through `stream`), but the steps of different sequences overlap.  Larger steps, position-shift
  * contexts and profiled runs are enqueued one after the other on `stream` itself.  See citrus_set_batch_lanes.

@@ -484,14 +484,15 @@ int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const i
     }
     const size_t qrow = (size_t)h->Hq * h->D * h->elt, krow = (size_t)h->Hkv * h->D * h->elt;   // multiples of 16 bytes
     cudaStream_t caller = reinterpret_cast<cudaStream_t>(stream);
-    // Lanes: only where a step is small (its attention items fit the SMs at once), which is where a sequence's
-    // kernels wait for each other more than they compute.  The embedding scratch of the position shift is one per
+    // Lanes: only where a step is small (its attention items make a few waves over the SMs at most), which is where a
+    // sequence's kernels wait for each other more than they compute.  The embedding scratch of the position shift is one per
     // context and per-launch timing wants one stream, so those run in the caller's stream.
     int n_lanes = 1;
     if (n_active > 1 && h->lane_fork != nullptr && !h->shift && !h->profiling) {
         int items = 0;
         for (int i = 0; i < n_active; ++i) items = std::max(items, (tok_offset[i + 1] - tok_offset[i] + 127) / 128 * h->Hq);
-        n_lanes = h->lanes_wanted > 0 ? h->lanes_wanted : (items <= 148 ? 4 : 1);
+        // measured: four lanes pay up to one wave of attention items per sequence, two up to about three waves
+        n_lanes = h->lanes_wanted > 0 ? h->lanes_wanted : (items <= 148 ? 4 : (items <= 448 ? 2 : 1));
         n_lanes = std::min(n_lanes, n_active);
     }
     if (n_lanes > 1) {
