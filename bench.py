@@ -358,6 +358,68 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_batch(args, local_rank):
+    """Side measurement (not the headline): `--sequences N` documents of the workload advance together, one chunk
+    each per step, through the packed ragged-batch call; `--lanes` as in citrus_set_batch_lanes (0 = chosen per call).
+    Prints a reduced JSON line: whole-batch tokens/s from a CUDA graph of the run, inputs resident in HBM."""
+    from paper_2406_12018_b200.binding import Citrus
+    torch.cuda.set_device(local_rank)
+    w = {**wl.CONFIGS, **wl.PAPER_SHAPES}[args.workload]
+    n_tok = args.doc_tokens or w.doc_tokens
+    w = wl.scaled(w, doc_tokens=n_tok, n_seqs=args.sequences, min_tokens=0)
+    docs = [wl.make_document(w, seq=i, n_tokens=n_tok) for i in range(args.sequences)]
+    steps = []
+    for c in range(-(-n_tok // w.chunk_s)):
+        sl = slice(c * w.chunk_s, min(n_tok, (c + 1) * w.chunk_s))
+        rows = sl.stop - sl.start
+        Q, K, V = (torch.cat([getattr(d, name)[sl] for d in docs]).cuda() for name in ("Q", "K", "V"))
+        steps.append((list(range(args.sequences)), [rows * i for i in range(args.sequences + 1)], Q, K, V, torch.empty_like(Q)))
+    Qi = torch.cat([d.Q_instr for d in docs]).cuda()
+    ins = [w.n_instr * i for i in range(args.sequences + 1)]
+    ctx = Citrus(1, w.q_heads, w.kv_heads, w.head_dim, w.budget_k, w.chunk_s, mode=w.mode, dtype=w.dtype,
+                 lm_window=w.lm_window, position_shift=w.position_shift, n_seqs=args.sequences)
+    ctx.set_batch_lanes(args.lanes)
+    stream = torch.cuda.Stream()
+
+    def all_documents():
+        ctx.reset()
+        for slots, tok, Q, K, V, out in steps:
+            ctx.process_chunk_batch(0, slots, tok, Q, K, V, ins, Qi, out=out, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(1, args.warmup)):
+            all_documents()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        all_documents()
+    n_steps = max(1, min(args.steps, 200))
+    with torch.cuda.stream(stream):
+        sampler = ClockSampler(local_rank)
+        sampler.start(); sampler.wait_first_sample()
+        for _ in range(args.warmup):
+            graph.replay()
+        torch.cuda.synchronize()
+        t_begin = time.time()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(n_steps):
+            graph.replay()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        clocks = sampler.stop(t_begin, time.time())
+    ms = ev0.elapsed_time(ev1) / n_steps
+    assert ctx.poll_status() == 0, "a bounded device wait expired during the benchmark"
+    print(json.dumps({"metric": METRIC + " (batch of sequences, side measurement)", "value": args.sequences * n_tok / (ms / 1e3),
+                      "unit": UNIT, "n_gpus": 1, "steps": n_steps, "warmup": args.warmup, "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": args.workload, "sequences": args.sequences, "doc_tokens": n_tok,
+                                 "lanes": args.lanes, "budget_k": w.budget_k, "chunk_s": w.chunk_s, "mode": w.mode,
+                                 "launch": "cuda_graph"},
+                      "clocks": clocks}), flush=True)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -370,6 +432,9 @@ def main():
     ap.add_argument("--doc-tokens", type=int, default=0, help="truncate / set the document length")
     ap.add_argument("--no-graph", action="store_true", help="launch every chunk from the host instead of a CUDA graph")
     ap.add_argument("--skip-cpu", action="store_true", help="do not time the oracle (profiling runs)")
+    ap.add_argument("--sequences", type=int, default=1,
+                    help="side measurement: this many documents advance together through the ragged-batch call (1 GPU)")
+    ap.add_argument("--lanes", type=int, default=0, help="with --sequences: side streams of the batch call (0 = automatic)")
     ap.add_argument("--traffic", type=float, default=ATTN_DRAM_TRAFFIC_BYTES,
                     help="DRAM bytes per attention launch from the committed ncu summary (null if stale)")
     args = ap.parse_args()
@@ -382,6 +447,11 @@ def main():
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    if args.sequences > 1:
+        if world > 1:
+            raise SystemExit("--sequences is a single-GPU side measurement")
+        run_batch(args, local_rank)
+        return
     run_ours(args, rank, world, local_rank)
 
 
