@@ -605,3 +605,14 @@ def test_reset_and_rerun_is_deterministic():
                 assert torch.equal(x, y), f"replay {rep} differs"
     assert ctx.poll_status() == 0
     ctx.close()
+
+
+def test_bench_batch_side_measurement_runs():
+    # the --sequences option of bench.py (packed ragged-batch call, lanes chosen by the library) on a short run
+    import json, os, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--sequences", "3", "--doc-tokens", "1536",
+                        "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["config"]["sequences"] == 3 and line["value"] > 0 and line["unit"] == "tokens/s"
