@@ -160,8 +160,9 @@ int citrus_process_chunk_slot(citrus_handle h, int layer, int seq_slot,
  * is shared between slots).  Where every sequence's step is small (its attention items make at most about three
  * waves over the SMs) the sequences are dealt to side streams owned by the context, which fork from `stream` when the call starts and join
  * it again before the call returns: to the caller the call is still one piece of work on `stream` (it can be captured
- * in a CUDA graph through `stream`), but the steps of different sequences overlap.  Larger steps, position-shift
- * contexts and profiled runs are enqueued one after the other on `stream` itself.  See citrus_set_batch_lanes.
+ * in a CUDA graph through `stream`), but the steps of different sequences overlap.  Larger steps and profiled
+ * runs are enqueued one after the other on `stream` itself (a position-shift context keeps one embedding scratch per
+ * side stream: 8 x (chunk_s + CITRUS_MAX_INSTR) x q_heads rows more, allocated by citrus_set_batch).  See citrus_set_batch_lanes.
  * Errors: as citrus_process_chunk; INVALID_ARG for duplicate slots or non-increasing offsets.
  */
 int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const int* seq_slot, const int* tok_offset,

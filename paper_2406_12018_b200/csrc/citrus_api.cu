@@ -80,6 +80,8 @@ struct citrus_ctx {
     cudaStream_t lane[kMaxLanes] = {};
     cudaEvent_t lane_done[kMaxLanes] = {};
     cudaEvent_t lane_fork = nullptr;
+    // position shift: the embedding scratch of a step, one set per lane (the context's own set serves the caller's stream)
+    void *laneRotQ[kMaxLanes] = {}, *laneRotK[kMaxLanes] = {}, *laneRotQi[kMaxLanes] = {};
 };
 
 namespace {
@@ -135,6 +137,16 @@ int make_lanes(citrus_ctx* c) {
         if (e == cudaSuccess && c->lane_done[i] == nullptr) e = cudaEventCreateWithFlags(&c->lane_done[i], cudaEventDisableTiming);
     }
     if (e != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
+    if (c->shift) {
+        const size_t row = (size_t)c->D * c->elt;
+        for (int i = 0; i < citrus_ctx::kMaxLanes; ++i) {
+            if (c->laneRotQ[i] != nullptr) continue;
+            int rc = dev_alloc(c, &c->laneRotQ[i], (size_t)c->ls * c->Hq * row, false, true);
+            if (rc == CITRUS_OK) rc = dev_alloc(c, &c->laneRotK[i], (size_t)c->ls * c->Hkv * row, false, true);
+            if (rc == CITRUS_OK) rc = dev_alloc(c, &c->laneRotQi[i], (size_t)CITRUS_MAX_INSTR * c->Hq * row, false, true);
+            if (rc != CITRUS_OK) return rc;
+        }
+    }
     return CITRUS_OK;
 }
 void free_all(citrus_ctx* c) {
@@ -207,8 +219,12 @@ struct LaunchTimer {                 // brackets one kernel launch with events w
 
 // The launch sequence of one chunk step; all pointers are device pointers.
 int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc, const void* Vc, int L,
-             const void* Qi, int nI, void* out, cudaStream_t st) {
+             const void* Qi, int nI, void* out, cudaStream_t st, int lane = -1) {
     c->used = true;
+    // embedding scratch of this step (position shift): the lane's own set when the step runs on a side stream
+    void* const rotQ = lane >= 0 ? c->laneRotQ[lane] : c->rotQ;
+    void* const rotK = lane >= 0 ? c->laneRotK[lane] : c->rotK;
+    void* const rotQi = lane >= 0 ? c->laneRotQi[lane] : c->rotQi;
     Unit& u = c->units[(size_t)layer * c->n_slots + slot];
     if (u.tokens_seen + L > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
     const bool lm_scoring = c->individual || (c->standard && nI == 0);   // cache 0 is scored by the chunk's own queries
@@ -234,11 +250,11 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     const void* Kc_raw = Kc;                                      // what the compaction gathers
     if (c->shift) {
         // position shift: embed the chunk's queries and keys at rows m .. m+L-1 and the instruction queries behind them
-        RopeRows jobs[3] = {{Qc, c->rotQ, L, c->Hq, mc[0]}, {Kc, c->rotK, L, c->Hkv, mc[0]}, {Qi, c->rotQi, nI, c->Hq, mc[0] + L}};
+        RopeRows jobs[3] = {{Qc, rotQ, L, c->Hq, mc[0]}, {Kc, rotK, L, c->Hkv, mc[0]}, {Qi, rotQi, nI, c->Hq, mc[0] + L}};
         LaunchTimer t(c, CITRUS_KERNEL_ROPE, st);
         e = rope_rows(jobs, instr_scoring ? 3 : 2, c->D, c->elt, c->rope, st);
         if (e != cudaSuccess) return cuda_rc(e);
-        Qc = c->rotQ; Kc = c->rotK; if (instr_scoring) Qi = c->rotQi;
+        Qc = rotQ; Kc = rotK; if (instr_scoring) Qi = rotQi;
         for (int ci = 0; ci < c->n_caches; ++ci) cand[ci].chunkK = Kc;
     }
     const int produced = c->shift ? 1 : 0;    // the embedding pre-pass above wrote Qc, Kc and Qi
@@ -485,10 +501,11 @@ int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const i
     const size_t qrow = (size_t)h->Hq * h->D * h->elt, krow = (size_t)h->Hkv * h->D * h->elt;   // multiples of 16 bytes
     cudaStream_t caller = reinterpret_cast<cudaStream_t>(stream);
     // Lanes: only where a step is small (its attention items make a few waves over the SMs at most), which is where a
-    // sequence's kernels wait for each other more than they compute.  The embedding scratch of the position shift is one per
-    // context and per-launch timing wants one stream, so those run in the caller's stream.
+    // sequence's kernels wait for each other more than they compute.  Per-launch timing wants one stream, so profiled
+    // runs stay in the caller's stream; a position-shift context needs its per-lane embedding scratch.
     int n_lanes = 1;
-    if (n_active > 1 && h->lane_fork != nullptr && !h->shift && !h->profiling) {
+    if (n_active > 1 && h->lane_fork != nullptr && !h->profiling &&
+        (!h->shift || h->laneRotQi[citrus_ctx::kMaxLanes - 1] != nullptr)) {
         int items = 0;
         for (int i = 0; i < n_active; ++i) items = std::max(items, (tok_offset[i + 1] - tok_offset[i] + 127) / 128 * h->Hq);
         // measured: four lanes pay up to one wave of attention items per sequence, two up to about three waves
@@ -509,7 +526,7 @@ int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const i
         const char* qi = reinterpret_cast<const char*>(Q_instr) + qrow * instr_offset[i];
         char* o = reinterpret_cast<char*>(out) + qrow * tok_offset[i];
         int rc = run_step(h, layer, seq_slot[i], q, k, v, tok_offset[i + 1] - tok_offset[i], qi,
-                          instr_offset[i + 1] - instr_offset[i], o, st_i);
+                          instr_offset[i + 1] - instr_offset[i], o, st_i, n_lanes > 1 ? i % n_lanes : -1);
         if (rc != CITRUS_OK) { first_rc = rc; break; }   // only a launch failure can get here; earlier sequences have advanced
     }
     if (n_lanes > 1) {

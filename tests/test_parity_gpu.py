@@ -427,12 +427,12 @@ def test_ragged_batch_call_matches_per_sequence_calls_and_rejects_bad_batches(la
     a.close(); b.close()
 
 
-@pytest.mark.parametrize("mode", ["shared", "individual"])
-def test_batch_lanes_in_a_captured_graph_equal_the_single_stream_run(mode):
+@pytest.mark.parametrize("mode,shift", [("shared", False), ("individual", False), ("shared", True), ("individual", True)])
+def test_batch_lanes_in_a_captured_graph_equal_the_single_stream_run(mode, shift):
     # six ragged sequences through the packed call: once on the caller's stream alone, once dealt to four side
     # streams and captured into a CUDA graph that is replayed twice; outputs, positions and caches must be identical
     w = wl.scaled(C["serving_mix"], n_seqs=6, budget_k=300, chunk_s=200, n_instr=40, doc_tokens=1000, min_tokens=150,
-                  mode=mode, lm_window=32)
+                  mode=mode, lm_window=32, position_shift=shift)    # with the shift every lane embeds into its own scratch
     lens = [1000, 431, 777, 150, 999, 600]
     docs = [wl.make_document(w, seq=s, n_tokens=n) for s, n in enumerate(lens)]
     steps, step = [], 0
