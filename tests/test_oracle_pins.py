@@ -539,6 +539,121 @@ def test_position_shift_with_eviction_embeds_by_cache_slot():
         expect = sum(wi / den * v for wi, v in zip(w, vals))
         assert np.allclose(res.out[t, 0], expect, atol=1e-12)
 
+def _torch_bf16(x):
+    """Round with torch's own float32 -> bfloat16 conversion (not the oracle's bit arithmetic)."""
+    return torch.tensor(np.asarray(x), dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def test_bf16_embedding_branch_rounds_queries_and_keys_once_and_nothing_else():
+    # A bf16 model holds its rotary-embedded queries and keys as bf16 tensors.  With a budget larger than the document
+    # nothing moves, so the shifted run with embedded_dtype="bf16" must equal a plain run on inputs that were embedded
+    # up front and rounded by torch: the chunk's queries and keys and the instruction queries are rounded, V is not,
+    # and the cache keeps the un-rotated, un-rounded keys.
+    from oracle import rope
+    rng = np.random.default_rng(44)
+    N, Hq, Hkv, D, ls, nI = 48, 4, 2, 8, 16, 5
+    # inputs exactly representable in bf16, as the library receives them
+    Q, K, V, Qi = (_torch_bf16(rand(rng, *s)) for s in ((N, Hq, D), (N, Hkv, D), (N, Hkv, D), (nI, Hq, D)))
+    shifted = CitrusOracle(Hq, Hkv, D, 1000, SHARED, rope_shift=True, embedded_dtype="bf16")
+    plain = CitrusOracle(Hq, Hkv, D, 1000, SHARED)
+    pos = np.arange(N)[:, None]
+    Qr, Kr = _torch_bf16(rope(Q, pos)), _torch_bf16(rope(K, pos))
+    unrounded = CitrusOracle(Hq, Hkv, D, 1000, SHARED, rope_shift=True)
+    differs = False
+    for c in range(0, N, ls):
+        a = shifted.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        Qir = _torch_bf16(rope(Qi, (c + ls + np.arange(nI))[:, None]))
+        b = plain.process_chunk(Qr[c:c + ls], Kr[c:c + ls], V[c:c + ls], Qir)
+        assert np.allclose(a.out, b.out, rtol=0, atol=1e-12)
+        assert np.allclose(a.scores[0], b.scores[0], rtol=0, atol=1e-12)
+        u = unrounded.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        differs = differs or np.abs(a.out - u.out).max() > 1e-6
+    assert differs                                                  # the rounding is really applied
+    assert np.array_equal(shifted.caches[0].K, np.transpose(K, (1, 0, 2)))      # stored keys: un-rotated, un-rounded
+    assert np.array_equal(shifted.caches[0].V, np.transpose(V, (1, 0, 2)))
+
+
+def test_bf16_embedding_branch_after_eviction_rounds_the_keys_embedded_by_slot():
+    # After eviction every kept key is embedded again from its stored (un-rotated) value at its new slot and rounded
+    # once; the query likewise.  One query row by plain loops, rounding with torch.
+    import math
+    from oracle import rope
+    rng = np.random.default_rng(45)
+    N, Hq, Hkv, D, k, ls = 40, 1, 1, 8, 6, 8
+    Q, K, V, Qi = (_torch_bf16(rand(rng, *s)) for s in ((N, Hq, D), (N, Hkv, D), (N, Hkv, D), (3, Hq, D)))
+    orc = CitrusOracle(Hq, Hkv, D, k, SHARED, rope_shift=True, embedded_dtype="bf16")
+    for c in range(0, N, ls):
+        held = orc.caches[0].pos[0].tolist()
+        res = orc.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        m = len(held)
+        keys = [_torch_bf16(rope(K[p, 0], np.array(slot))) for slot, p in enumerate(held)] + \
+               [_torch_bf16(rope(K[c + i, 0], np.array(m + i))) for i in range(ls)]
+        vals = [V[p, 0] for p in held] + [V[c + i, 0] for i in range(ls)]
+        t = ls - 1
+        qv = _torch_bf16(rope(Q[c + t, 0], np.array(m + t)))
+        logits = [float(qv @ kk) / math.sqrt(D) for kk in keys]
+        mx = max(logits); w = [math.exp(x - mx) for x in logits]; den = sum(w)
+        assert np.allclose(res.out[t, 0], sum(wi / den * v for wi, v in zip(w, vals)), rtol=0, atol=1e-12)
+        # instruction scores (Eq. 1, s = I): instruction token i sits at slot m + L + i
+        score = [0.0] * len(keys)
+        for i in range(Qi.shape[0]):
+            qi = _torch_bf16(rope(Qi[i, 0], np.array(m + ls + i)))
+            lg = [float(qi @ kk) / math.sqrt(D) for kk in keys]
+            mx = max(lg); den = sum(math.exp(x - mx) for x in lg)
+            for j, x in enumerate(lg):
+                score[j] += math.exp(x - mx) / den
+        assert np.allclose(res.scores[0][0], score, rtol=0, atol=1e-12)
+
+
+def test_individual_caches_follow_the_two_eviction_rules_in_plain_python():
+    # Section 4.2, individual cache (Eq. 4-5): the language-modelling cache C is evicted by the chunk's own attention,
+    # the instruction cache C^I by the instruction's attention over C^I's OWN states plus the chunk; the chunk is
+    # encoded against C only.  Plain loops over original positions; K/V are looked up in the document by position.
+    import math
+    rng = np.random.default_rng(46)
+    N, Hq, Hkv, D, k, ls, nI, w = 60, 4, 2, 4, 7, 10, 3, 4
+    G = Hq // Hkv
+    Q, K, V, Qi = rand(rng, N, Hq, D), rand(rng, N, Hkv, D), rand(rng, N, Hkv, D), rand(rng, nI, Hq, D)
+    orc = CitrusOracle(Hq, Hkv, D, k, INDIVIDUAL, lm_window=w)
+
+    def softmax_over(qvec, g, keys):
+        lg = [sum(qvec[d] * K[j, g, d] for d in range(D)) / math.sqrt(D) for j in keys]
+        mx = max(lg); e = [math.exp(x - mx) for x in lg]; den = sum(e)
+        return [x / den for x in e]
+
+    C = [[] for _ in range(Hkv)]        # positions held by the language-modelling cache, per KV head
+    CI = [[] for _ in range(Hkv)]       # positions held by the instruction cache
+    caches_differ = False
+    for c in range(0, N, ls):
+        chunk = list(range(c, c + ls))
+        res = orc.process_chunk(Q[c:c + ls], K[c:c + ls], V[c:c + ls], Qi)
+        for g in range(Hkv):
+            cand_lm, cand_in = C[g] + chunk, CI[g] + chunk
+            s_lm = {j: 0.0 for j in cand_lm}
+            s_in = {j: 0.0 for j in cand_in}
+            for h in range(g * G, (g + 1) * G):
+                for t in chunk:
+                    keys = C[g] + [u for u in chunk if u <= t]
+                    p = softmax_over(Q[t, h], g, keys)
+                    # the output comes from the language-modelling cache
+                    expect = [sum(pj * V[j, g, d] for pj, j in zip(p, keys)) for d in range(D)]
+                    assert np.allclose(res.out[t - c, h], expect, rtol=0, atol=1e-12)
+                    if t >= c + ls - w:                       # the last w queries of the chunk vote on C
+                        for pj, j in zip(p, keys):
+                            s_lm[j] += pj
+                for i in range(nI):                           # every instruction token votes on C^I, unmasked
+                    for pj, j in zip(softmax_over(Qi[i, h], g, cand_in), cand_in):
+                        s_in[j] += pj
+            assert np.allclose(res.scores[0][g], [s_lm[j] for j in cand_lm], rtol=0, atol=1e-12)
+            assert np.allclose(res.scores[1][g], [s_in[j] for j in cand_in], rtol=0, atol=1e-12)
+            C[g] = sorted(sorted(cand_lm, key=lambda j: (-s_lm[j], j))[:k])
+            CI[g] = sorted(sorted(cand_in, key=lambda j: (-s_in[j], j))[:k])
+            assert orc.caches[0].pos[g].tolist() == C[g]
+            assert orc.caches[1].pos[g].tolist() == CI[g]
+            assert np.array_equal(orc.caches[1].K[g], K[CI[g], g]) and np.array_equal(orc.caches[1].V[g], V[CI[g], g])
+            caches_differ = caches_differ or C[g] != CI[g]
+    assert caches_differ                # otherwise scoring C^I with C's keys would go unnoticed
+
 
 def test_forced_selection_is_adopted():
     rng = np.random.default_rng(16)
