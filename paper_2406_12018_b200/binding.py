@@ -87,15 +87,18 @@ def strerror(code: int) -> str:
     return load().citrus_strerror(code).decode()
 
 
-def importance_static(Q_s: torch.Tensor, K: torch.Tensor, scores: torch.Tensor, stream=None) -> torch.Tensor:
+def importance_static(Q_s: torch.Tensor, K: torch.Tensor, scores: torch.Tensor, stream=None,
+                      status: Optional[torch.Tensor] = None) -> torch.Tensor:
     """Eq. 1 column sums of scoring rows Q_s [n_s, H_q, D] over keys K [n, H_kv, D] into the caller's
-    `scores` [H_kv, >= n] fp32, through the entry point that allocates nothing (see citrus.h)."""
+    `scores` [H_kv, >= n] fp32, through the entry point that allocates nothing (see citrus.h).
+    status: optional caller-owned int32 device word (zeroed by the caller), set to 1 if a bounded wait expires."""
     assert Q_s.is_cuda and K.is_cuda and scores.is_cuda and scores.dtype == torch.float32
+    assert status is None or (status.is_cuda and status.dtype == torch.int32)
     assert Q_s.is_contiguous() and K.is_contiguous() and scores.is_contiguous() and Q_s.dtype == K.dtype
     mode = MODE_FP32 if Q_s.dtype == torch.float32 else 0
     rc = load().citrus_importance_static(Q_s.data_ptr(), Q_s.shape[0], K.data_ptr(), K.shape[0], Q_s.shape[1],
                                          K.shape[1], Q_s.shape[2], mode, scores.data_ptr(), scores.shape[1],
-                                         None, _stream_ptr(stream))
+                                         None if status is None else status.data_ptr(), _stream_ptr(stream))
     if rc != 0:
         raise CitrusError(rc, "citrus_importance_static")
     return scores

@@ -4,14 +4,18 @@ Some users of this library cannot allocate device memory when they need scores -
 has given all of the GPU to its own pool, or they sit in a loop where cudaMalloc's device-wide
 synchronisation is not acceptable.  For them `citrus_importance_static` keeps its scratch in an
 array inside the library image.  This file checks, through the C ABI, that it returns what the
-first chunk of `citrus_process_chunk` computes for the same instruction queries and keys, twice in
-a row (the second call reuses the array the first one left dirty), and that oversized requests
-are refused.  It is named to be collected last.
+first chunk of `citrus_process_chunk` computes for the same instruction queries and keys and what
+the fp64 oracle's Eq. 1 column sums give, twice in a row (the second call reuses the array the
+first one left dirty), that the calls leave the amount of free device memory unchanged, and that
+oversized requests are refused.  It is named to be collected last.
 """
 import ctypes as C
 
+import numpy as np
 import pytest
 import torch
+
+import oracle
 
 from paper_2406_12018_b200 import binding, workloads as wl
 from paper_2406_12018_b200.binding import Citrus
@@ -32,11 +36,24 @@ def test_static_scores_match_regular_entry_point_twice(dtype, D):
         torch.cuda.synchronize()
         want = ctx.step_view(0)[0].clone()                      # [H_kv, L] scores of the existing entry point
         got = torch.full((w.kv_heads, L + 5), -1.0, device="cuda")
-        binding.importance_static(Qi, K, got)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        if call == 0:
+            binding.importance_static(Qi, K, got, status=status)   # the first call on a device does the one-time set-up
+            got.fill_(-1.0)
         torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]             # cudaMemGetInfo: the driver's view, not torch's cache
+        binding.importance_static(Qi, K, got, status=status)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before, "the allocation-free entry point changed free device memory"
+        assert int(status.item()) == 0                          # no bounded wait expired
         norm = n_instr * (w.q_heads // w.kv_heads)
         err = float((got[:, :L] - want).abs().max()) / norm
         assert err <= TOL[dtype], f"call {call}: normalised score error {err}"
+        # against the definition (Eq. 1, s = I, over exactly these keys; no retained cache)
+        S = oracle.importance_sum(wl.to_f64(doc.Q_instr), np.zeros((w.kv_heads, 0, D)), wl.to_f64(doc.K))
+        err_o = float(np.abs(got[:, :L].double().cpu().numpy() - S).max()) / norm
+        assert err_o <= TOL[dtype], f"call {call}: normalised score error against the oracle {err_o}"
+        assert np.allclose(got[:, :L].double().cpu().numpy().sum(axis=1), norm, rtol=2e-3)
         assert bool((got[:, L:] == -1.0).all())                 # nothing written past n_keys
         ctx.close()
 
