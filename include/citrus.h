@@ -123,6 +123,20 @@ int citrus_set_batch(citrus_handle h, int n_seq);
  * sequence on the caller's stream; up to 8.  May be changed between calls.  Errors: INVALID_ARG. */
 int citrus_set_batch_lanes(citrus_handle h, int n_lanes);
 
+/*
+ * Ordering of the caller's inputs (no counterpart in the paper; a property of how the kernels are launched).  The
+ * kernels of a call are launched with programmatic stream serialisation, which lets a kernel begin while its
+ * predecessor in the stream is still running.  By default (ready = 0) every kernel of a call waits for all earlier
+ * work in the stream before it first reads Q_chunk / K_chunk / V_chunk / Q_instr or writes `out`, so plain stream
+ * order holds whatever produced the inputs - also a kernel of the caller's that signals its dependents early.
+ * ready = 1 is the caller's promise that the inputs of every later call are complete before the call's first kernel
+ * can start executing (they were produced by copies, by work the stream has been synchronised with, or by kernels
+ * that do not signal their dependents early): the chunk's own tiles are then loaded while the previous call's
+ * compaction is still running.  The *_host variants order their own copies and always take the fast route.
+ * Errors: INVALID_ARG.
+ */
+int citrus_set_inputs_ready(citrus_handle h, int ready);
+
 /* Forget every cache of every layer and slot (start a new document). Host-only
  * bookkeeping; enqueues nothing. */
 int citrus_reset(citrus_handle h);
@@ -145,7 +159,10 @@ int citrus_process_chunk(citrus_handle h, int layer,
                          const void* Q_instr, int n_instr, void* out, citrus_stream_t stream);
 
 /* Same, for sequence slot `seq_slot` (ragged batches submit one call per active
- * sequence; slots are independent and may use different streams). */
+ * sequence; slots are independent and may use different streams).  A CITRUS_MODE_POSITION_SHIFT context has one
+ * embedding scratch: a step submitted on another stream than the context's previous step is ordered, by an event,
+ * behind everything enqueued on that stream so far (so such steps do not overlap; all of them must then belong to
+ * the same stream capture, or to none). */
 int citrus_process_chunk_slot(citrus_handle h, int layer, int seq_slot,
                               const void* Q_chunk, const void* K_chunk, const void* V_chunk, int n_tokens,
                               const void* Q_instr, int n_instr, void* out, citrus_stream_t stream);
@@ -262,9 +279,10 @@ int citrus_profile_read(citrus_handle h, double* ms, long long* launches);
  * tensor-map encoder and raises the kernels' shared-memory limits); make that first call
  * outside of any stream capture.  All calls on a device share the one array and overwrite it:
  * two calls whose GPU work overlaps (different streams, or different threads) race; run them
- * on one stream or order them with events.  device_status may be NULL; otherwise it is a
- * caller-owned device int, zeroed by the caller, set to 1 if a bounded wait inside a kernel
- * expires.
+ * on one stream or order them with events.  device_status is a caller-owned device int, zeroed by
+ * the caller, set to 1 if a bounded wait inside a kernel expires (the scores are then not valid).
+ * It may be NULL: the flag then goes to a word of the shared array that the next call clears and
+ * nothing reports, i.e. an expired wait goes unnoticed - pass a status word wherever that matters.
  */
 #define CITRUS_STATIC_MAX_LSE 65536
 int citrus_importance_static(const void* Q_s, int n_s, const void* K, int n_keys,
@@ -288,8 +306,16 @@ int citrus_intersection_ratio(citrus_handle h, int layer, int seq_slot, float* r
 int citrus_set_rope_base(citrus_handle h, double base);
 
 /* Reads the device status word (0, or CITRUS_ERR_TIMEOUT if a bounded wait in a
- * kernel gave up). Synchronises the device. */
+ * kernel gave up: every wait on an mbarrier inside the kernels ends after about one second, raises the word, and
+ * the kernel drains and returns).  Synchronises the device.  A raised word is cleared by the read; the caches of
+ * the steps that ran meanwhile are not valid (citrus_reset starts over). */
 int citrus_poll_status(citrus_handle h);
+
+/* Test aid for the time-out path (the paper has no counterpart): enqueues one warp that waits limit_ns nanoseconds
+ * (1 .. 100 000 000) on an mbarrier that nothing arms, with the same bounded wait the kernels use; the wait runs
+ * out, the kernel raises the context's status word and returns normally.  citrus_poll_status then reports
+ * CITRUS_ERR_TIMEOUT once.  Nothing else is touched.  Errors: INVALID_ARG, CUDA. */
+int citrus_debug_expire_wait(citrus_handle h, unsigned long long limit_ns, citrus_stream_t stream);
 
 /* Frees everything. NULL is a no-op; a handle that was already destroyed
  * returns CITRUS_ERR_STATE. */

@@ -32,7 +32,7 @@ EXPORTS = [
     "citrus_create", "citrus_set_batch", "citrus_set_batch_lanes", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
     "citrus_process_chunk_host", "citrus_process_document_host", "citrus_process_chunk_batch", "citrus_cache_view", "citrus_step_view", "citrus_profile",
     "citrus_profile_read", "citrus_importance_static", "citrus_intersection_ratio", "citrus_set_rope_base",
-    "citrus_poll_status",
+    "citrus_poll_status", "citrus_set_inputs_ready", "citrus_debug_expire_wait",
     "citrus_destroy", "citrus_strerror",
 ]
 
@@ -73,6 +73,8 @@ def load() -> C.CDLL:
     lib.citrus_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     lib.citrus_importance_static.argtypes = [vp, i, vp, i, i, i, i, C.c_uint, vp, i, vp, vp]
     lib.citrus_poll_status.argtypes = [vp]
+    lib.citrus_set_inputs_ready.argtypes = [vp, i]
+    lib.citrus_debug_expire_wait.argtypes = [vp, C.c_ulonglong, vp]
     lib.citrus_destroy.argtypes = [vp]
     lib.citrus_strerror.argtypes = [i]
     lib.citrus_strerror.restype = C.c_char_p
@@ -273,6 +275,18 @@ class Citrus:
 
     def poll_status(self) -> int:
         return load().citrus_poll_status(self._h)
+
+    def set_inputs_ready(self, ready: bool):
+        """Promise (or withdraw the promise) that every call's inputs are complete before its first kernel can run."""
+        rc = load().citrus_set_inputs_ready(self._h, 1 if ready else 0)
+        if rc != 0:
+            raise CitrusError(rc, "citrus_set_inputs_ready")
+
+    def debug_expire_wait(self, limit_ns: int = 1_000_000, stream=None):
+        """Test aid: let one bounded device wait run out (see citrus.h)."""
+        rc = load().citrus_debug_expire_wait(self._h, limit_ns, _stream_ptr(stream))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_debug_expire_wait")
 
     def close(self):
         if getattr(self, "_h", None) is not None and self._h.value is not None:

@@ -61,6 +61,14 @@ struct citrus_ctx {
     std::vector<void*> allocs;      // cache buffers and per-unit scratch
     std::vector<void*> misc;        // status word, host-variant staging
     int* status = nullptr;
+    // The caller has promised that the inputs of every call are complete before the call's first kernel can start
+    // (citrus_set_inputs_ready): the kernels may then load them ahead of griddepcontrol.wait.
+    bool inputs_ready = false;
+    // position shift: stream of the last step and an event to order a step on another stream behind it (the
+    // embedding scratch is one per context)
+    cudaStream_t shift_stream = nullptr;
+    bool shift_stream_set = false;
+    cudaEvent_t shift_done = nullptr;
     // optional per-launch timing: (kernel id, start, stop) event pairs recorded on the launching stream
     bool profiling = false;
     struct Timed { int id; cudaEvent_t a, b; };
@@ -127,6 +135,8 @@ void free_copy_streams(citrus_ctx* c) {
     }
     if (c->lane_fork) cudaEventDestroy(c->lane_fork);
     c->lane_fork = nullptr;
+    if (c->shift_done) cudaEventDestroy(c->shift_done);
+    c->shift_done = nullptr;
 }
 // Side streams and events of the batch lanes (created once, by citrus_set_batch for more than one slot).
 int make_lanes(citrus_ctx* c) {
@@ -219,8 +229,18 @@ struct LaunchTimer {                 // brackets one kernel launch with events w
 
 // The launch sequence of one chunk step; all pointers are device pointers.
 int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc, const void* Vc, int L,
-             const void* Qi, int nI, void* out, cudaStream_t st, int lane = -1) {
+             const void* Qi, int nI, void* out, cudaStream_t st, int lane = -1, bool inputs_ordered = false) {
     c->used = true;
+    if (c->shift && lane < 0) {
+        // One embedding scratch per context: a step on another stream than the last one is ordered behind everything
+        // enqueued there so far.  Steps that stay on one stream pay nothing.
+        if (c->shift_stream_set && c->shift_stream != st) {
+            cudaError_t ee = cudaEventRecord(c->shift_done, c->shift_stream);
+            if (ee == cudaSuccess) ee = cudaStreamWaitEvent(st, c->shift_done, 0);
+            if (ee != cudaSuccess) return cuda_rc(ee);
+        }
+        c->shift_stream = st; c->shift_stream_set = true;
+    }
     // embedding scratch of this step (position shift): the lane's own set when the step runs on a side stream
     void* const rotQ = lane >= 0 ? c->laneRotQ[lane] : c->rotQ;
     void* const rotK = lane >= 0 ? c->laneRotK[lane] : c->rotK;
@@ -245,7 +265,6 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         }
         cand[ci] = Candidates{cb.K[cb.cur], cb.V[cb.cur], Kc, Vc, mc[ci], L, c->cap[ci], c->Hkv};
     }
-    const int m = mc[0];
     cudaError_t e;
     const void* Kc_raw = Kc;                                      // what the compaction gathers
     if (c->shift) {
@@ -257,7 +276,11 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
         Qc = rotQ; Kc = rotK; if (instr_scoring) Qi = rotQi;
         for (int ci = 0; ci < c->n_caches; ++ci) cand[ci].chunkK = Kc;
     }
-    const int produced = c->shift ? 1 : 0;    // the embedding pre-pass above wrote Qc, Kc and Qi
+    // 1: the kernels wait for their predecessors in the stream before their first load of Q / K / Q_instr.  Needed when
+    // the embedding pre-pass above wrote them, and whenever the inputs may still be in the making: the call's first
+    // kernel is launched with programmatic stream serialisation, so a preceding kernel of the CALLER that signals
+    // its dependents early could otherwise still be writing them.
+    const int produced = (c->shift || !(c->inputs_ready || inputs_ordered)) ? 1 : 0;
     QueryRows q_chunk{Qc, L, c->Hq, 1, 0, produced};
     QueryRows q_instr{Qi, nI, c->Hq, 0, 0, produced};
     float* scores[2] = {u.scores, u.scores + (size_t)c->Hkv * c->score_stride};
@@ -354,6 +377,20 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
 
 }  // namespace
 
+int citrus::sm_count() {
+    static std::mutex mu;
+    static int count[DeviceOnce::kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= DeviceOnce::kMaxDevices) { cudaGetLastError(); return 148; }
+    std::lock_guard<std::mutex> lk(mu);
+    if (count[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) { cudaGetLastError(); n = 148; }
+        count[dev] = n;
+    }
+    return count[dev];
+}
+
 void citrus::before_launch(cudaStream_t s) {
     if (t_pending_start != nullptr) {
         cudaEventRecord(t_pending_start, s);
@@ -399,12 +436,12 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
     c->n_caches = c->individual ? 2 : 1;
     c->score_stride = (c->cap[0] + chunk_s + 3) & ~3;
     c->use_tc = !fp32 && head_dim == 128;
-    if (c->use_tc) {
-        const char* dbg = std::getenv("CITRUS_DEBUG_SIMT");
-        if (dbg != nullptr && dbg[0] == '1') c->use_tc = false;
-    }
     int rc = dev_alloc(c, (void**)&c->status, sizeof(int), true, true);
     if (rc == CITRUS_OK && c->use_tc && tc_init() != cudaSuccess) rc = CITRUS_ERR_UNSUPPORTED;
+    if (rc == CITRUS_OK && c->shift && cudaEventCreateWithFlags(&c->shift_done, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        rc = CITRUS_ERR_CUDA;
+    }
     if (rc == CITRUS_OK && c->shift) {
         const size_t row = (size_t)head_dim * c->elt;
         rc = dev_alloc(c, &c->rotQ, (size_t)chunk_s * q_heads * row, false, true);
@@ -412,7 +449,7 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
         if (rc == CITRUS_OK) rc = dev_alloc(c, &c->rotQi, (size_t)CITRUS_MAX_INSTR * q_heads * row, false, true);
     }
     if (rc == CITRUS_OK) rc = alloc_units(c);
-    if (rc != CITRUS_OK) { free_all(c); delete c; return rc; }
+    if (rc != CITRUS_OK) { if (c->shift_done) cudaEventDestroy(c->shift_done); free_all(c); delete c; return rc; }
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_live.insert(c);
@@ -446,6 +483,12 @@ int citrus_set_batch_lanes(citrus_handle h, int n_lanes) {
     if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
     if (n_lanes < 0 || n_lanes > citrus_ctx::kMaxLanes) return CITRUS_ERR_INVALID_ARG;
     h->lanes_wanted = n_lanes;
+    return CITRUS_OK;
+}
+
+int citrus_set_inputs_ready(citrus_handle h, int ready) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    h->inputs_ready = ready != 0;
     return CITRUS_OK;
 }
 
@@ -509,7 +552,7 @@ int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const i
         int items = 0;
         for (int i = 0; i < n_active; ++i) items = std::max(items, (tok_offset[i + 1] - tok_offset[i] + 127) / 128 * h->Hq);
         // measured: four lanes pay up to one wave of attention items per sequence, two up to about three waves
-        n_lanes = h->lanes_wanted > 0 ? h->lanes_wanted : (items <= 148 ? 4 : (items <= 448 ? 2 : 1));
+        n_lanes = h->lanes_wanted > 0 ? h->lanes_wanted : (items <= sm_count() ? 4 : (items <= 3 * sm_count() ? 2 : 1));
         n_lanes = std::min(n_lanes, n_active);
     }
     if (n_lanes > 1) {
@@ -526,7 +569,8 @@ int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const i
         const char* qi = reinterpret_cast<const char*>(Q_instr) + qrow * instr_offset[i];
         char* o = reinterpret_cast<char*>(out) + qrow * tok_offset[i];
         int rc = run_step(h, layer, seq_slot[i], q, k, v, tok_offset[i + 1] - tok_offset[i], qi,
-                          instr_offset[i + 1] - instr_offset[i], o, st_i, n_lanes > 1 ? i % n_lanes : -1);
+                          instr_offset[i + 1] - instr_offset[i], o, st_i, n_lanes > 1 ? i % n_lanes : -1,
+                          /*inputs_ordered=*/n_lanes > 1);    // a lane starts behind an event of the caller's stream
         if (rc != CITRUS_OK) { first_rc = rc; break; }   // only a launch failure can get here; earlier sequences have advanced
     }
     if (n_lanes > 1) {
@@ -559,7 +603,7 @@ int citrus_process_chunk_host(citrus_handle h, int layer, int seq_slot,
     if ((e = cudaMemcpyAsync(h->stK, Kh, krow * n_tokens, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
     if ((e = cudaMemcpyAsync(h->stV, Vh, krow * n_tokens, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
     if (n_instr > 0 && (e = cudaMemcpyAsync(h->stQi, Qih, qrow * n_instr, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_rc(e);
-    rc = run_step(h, layer, seq_slot, h->stQ, h->stK, h->stV, n_tokens, h->stQi, n_instr, h->stOut, st);
+    rc = run_step(h, layer, seq_slot, h->stQ, h->stK, h->stV, n_tokens, h->stQi, n_instr, h->stOut, st, -1, true);
     if (rc) return rc;
     if ((e = cudaMemcpyAsync(out_h, h->stOut, qrow * n_tokens, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_rc(e);
     return cuda_rc(cudaStreamSynchronize(st));
@@ -629,7 +673,7 @@ int citrus_process_document_host(citrus_handle h, int layer, int seq_slot,
             const bool last = t0 + r0 + L == n_tokens;
             const bool with_instr = !h->standard || last;
             rc = run_step(h, layer, seq_slot, (char*)h->docQ[b] + qrow * r0, (char*)h->docK[b] + krow * r0, (char*)h->docV[b] + krow * r0, L,
-                          with_instr ? h->docQi : nullptr, with_instr ? n_instr : 0, (char*)h->docOut[b] + qrow * r0, st);
+                          with_instr ? h->docQi : nullptr, with_instr ? n_instr : 0, (char*)h->docOut[b] + qrow * r0, st, -1, true);
         }
         if (rc != CITRUS_OK) break;
         if ((e = cudaEventRecord(h->ev_step[b], st)) != cudaSuccess) break;
@@ -718,7 +762,14 @@ int citrus_poll_status(citrus_handle h) {
     int v = 0;
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
     if (cudaMemcpy(&v, h->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
+    if (v != 0 && cudaMemset(h->status, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
     return v == 0 ? CITRUS_OK : CITRUS_ERR_TIMEOUT;
+}
+
+int citrus_debug_expire_wait(citrus_handle h, unsigned long long limit_ns, citrus_stream_t stream) {
+    if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
+    if (limit_ns < 1 || limit_ns > 100000000ull) return CITRUS_ERR_INVALID_ARG;       // at most 0.1 s
+    return cuda_rc(tc_expire_wait(h->status, limit_ns, reinterpret_cast<cudaStream_t>(stream)));
 }
 
 int citrus_destroy(citrus_handle h) {

@@ -34,6 +34,18 @@ struct Candidates {
     int kv_heads;
 };
 
+// One-time set-up that is per DEVICE (a kernel's shared-memory limit, the address of a __device__ symbol): which
+// devices of this process have had it.  Host bookkeeping only; the caller holds its own mutex around a
+// needs_setup / mark pair.
+struct DeviceOnce {
+    static constexpr int kMaxDevices = 64;
+    bool done[kMaxDevices] = {};
+    bool needs_setup(int dev) const { return dev < 0 || dev >= kMaxDevices || !done[dev]; }
+    void mark(int dev) { if (dev >= 0 && dev < kMaxDevices) done[dev] = true; }
+};
+// Streaming multiprocessors of the current device (cached per device).
+int sm_count();
+
 // Called by every launcher immediately before its kernel launch: when per-launch timing is on, this is where the
 // start event is recorded, so that host-side preparation (tensor-map encoding) is not counted as kernel time.
 void before_launch(cudaStream_t s);
@@ -59,7 +71,9 @@ cudaError_t simt_colsum(bool is_fp32, int D, const QueryRows& q, const Candidate
                         const float* lse2, int lse_stride, float* scores, int score_stride, cudaStream_t s);
 
 // ---- tensor-core (tcgen05 / TMEM / TMA) path: bf16, D = 128 ----------------
-cudaError_t tc_init();   // resolves the driver entry point for tensor-map encoding
+cudaError_t tc_init();   // resolves the driver entry point for tensor-map encoding; raises the kernels' shared-memory limits on the current device
+// Test aid: one warp waits limit_ns on an mbarrier nobody arms, raises *status and returns.
+cudaError_t tc_expire_wait(int* status, unsigned long long limit_ns, cudaStream_t s);
 // Number of key splits for pass 1 of a2-I (1 = the pass writes final log-sum-exp values).
 int tc_lse_splits(int n_rows, int q_heads, int kv_heads, int m, int L, int n_attn_items);
 constexpr int kTcMaxLseSplits = 8;

@@ -69,7 +69,7 @@ extern "C" int citrus_importance_static(const void* Q_s, int n_s, const void* K,
     }
     // all candidates are "chunk" rows of a token-major tensor; there is no retained cache (m = 0)
     Candidates cand{K, K, K, K, 0, n_keys, n_keys, kv_heads};
-    QueryRows q{Q_s, n_s, q_heads, 0, 0, 0};
+    QueryRows q{Q_s, n_s, q_heads, 0, 0, 1};   // produced = 1: wait for earlier stream work before the first load of Q_s or K
     cudaError_t e;
     if (fp32) {
         e = simt_attention(true, head_dim, q, cand, nullptr, lse, lse_stride, st);

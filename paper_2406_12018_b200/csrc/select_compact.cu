@@ -2,6 +2,8 @@
 // (ordered gather of K, V and positions into the other ping-pong buffer).
 #include "citrus_internal.h"
 
+#include <mutex>
+
 CITRUS_TRACE_EXPORT(_sc)
 #ifdef CITRUS_TRACE
 static __device__ __forceinline__ unsigned long long trace_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
@@ -268,7 +270,12 @@ __device__ __forceinline__ void compact_rows_t(const CompactJob& job, const uint
     uint4* dstV = reinterpret_cast<uint4*>(job.dstV);
     // four rows per thread in flight: first every index, then every load, then the stores
     constexpr int kInFlight = 4;
-    for (int rb = r_begin + sub; rb < r_end; rb += kInFlight * rows_per_pass) {
+    // The trip count is the same for every lane of a warp (the position-shift variant exchanges registers with a
+    // full-mask shuffle): the loop runs on the row of the warp's first lane, a lane whose own row lies past the end
+    // carries j = -1 and only skips its loads and stores.
+    const int sub_first = (int)(threadIdx.x & ~31u) / row_vecs;
+    for (int rb_w = r_begin + sub_first; rb_w < r_end; rb_w += kInFlight * rows_per_pass) {
+        const int rb = rb_w + (sub - sub_first);
         int j[kInFlight];
         uint4 a[kInFlight], b[kInFlight];
         if (SHIFT) {
@@ -424,18 +431,38 @@ rope_rows_kernel(const __grid_constant__ RopeArgs args) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const RopeRows& job = args.job[blockIdx.y];
     const int row_vecs = args.row_vecs, half_vecs = row_vecs >> 1, per_vec = 16 / args.elt;
-    const long long total = (long long)job.rows * job.heads * row_vecs;          // a multiple of 32
+    const long long total = (long long)job.rows * job.heads * row_vecs;          // a multiple of row_vecs, not always of 32
     const uint4* in = reinterpret_cast<const uint4*>(job.in);
     uint4* out = reinterpret_cast<uint4*>(job.out);
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int lane = threadIdx.x & 31;
+    // warp-uniform trip count (the exchange below is a full-mask shuffle): the loop runs on the warp's first piece
+    for (long long i_w = (long long)blockIdx.x * blockDim.x + (threadIdx.x - lane); i_w < total; i_w += (long long)gridDim.x * blockDim.x) {
+        const long long i = i_w + lane;
+        const bool active = i < total;
         const int v = (int)(i % row_vecs);
         const int row = (int)(i / ((long long)row_vecs * job.heads));
-        const uint4 mine = __ldg(in + i);
+        const uint4 mine = active ? __ldg(in + i) : make_uint4(0u, 0u, 0u, 0u);
         uint4 other;
         other.x = __shfl_xor_sync(0xffffffffu, mine.x, half_vecs); other.y = __shfl_xor_sync(0xffffffffu, mine.y, half_vecs);
         other.z = __shfl_xor_sync(0xffffffffu, mine.z, half_vecs); other.w = __shfl_xor_sync(0xffffffffu, mine.w, half_vecs);
-        out[i] = rope_piece(mine, other, job.pos0 + row, (v % half_vecs) * per_vec, v < half_vecs, args.table, args.elt);
+        if (active) out[i] = rope_piece(mine, other, job.pos0 + row, (v % half_vecs) * per_vec, v < half_vecs, args.table, args.elt);
     }
+}
+
+// The dynamic shared-memory limit of a kernel is a per-device attribute: raised once on every device that launches.
+std::mutex g_attr_mu;
+DeviceOnce g_attr_ready;
+cudaError_t raise_smem_limits() {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lk(g_attr_mu);
+    if (!g_attr_ready.needs_setup(dev)) return cudaSuccess;
+    e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    g_attr_ready.mark(dev);
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -474,12 +501,10 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int lay
     SelectArgs a;
     int n = 0;
     for (int i = 0; i < n_jobs; ++i) { a.job[i] = jobs[i]; n = jobs[i].n > n ? jobs[i].n : n; }
-    static bool attr_set = false;
     size_t smem = (size_t)n * sizeof(uint32_t);
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    {
+        cudaError_t e = raise_smem_limits();
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(layerwise ? 1 : kv_heads, n_jobs);
@@ -505,11 +530,9 @@ cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int 
         n = sjobs[i].n > n ? sjobs[i].n : n;
         kept = cjobs[i].kept > kept ? cjobs[i].kept : kept;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    {
+        cudaError_t e = raise_smem_limits();
         if (e != cudaSuccess) return e;
-        attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kFusedCluster, kv_heads, n_jobs);

@@ -15,6 +15,7 @@
 
 #include <cuda.h>
 
+#include <mutex>
 #include <utility>
 
 CITRUS_TRACE_EXPORT()
@@ -62,9 +63,9 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status, uint64_t limit_ns = kWaitLimitNs) {
     const uint64_t t0 = global_ns();
-    while (global_ns() - t0 < kWaitLimitNs) {
+    while (global_ns() - t0 < limit_ns) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try(bar, parity)) return true;
         __nanosleep(128);
@@ -72,14 +73,14 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* 
     atomicExch(status, 1);
     return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, uint64_t limit_ns = kWaitLimitNs) {
     for (int i = 0; i < 512; ++i)
         if (mbar_try(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, status);
+    return mbar_wait_slow(bar, parity, status, limit_ns);
 }
 // Same, with one outcome for the whole warp (the callers go on to warp-collective instructions).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, status));
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status, uint64_t limit_ns = kWaitLimitNs) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, status, limit_ns));
 }
 
 // One lane of a converged warp.  Loop control, addresses and descriptors are computed by the whole
@@ -927,6 +928,8 @@ typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeFn g_encode = nullptr;
+std::mutex g_init_mu;
+DeviceOnce g_device_ready;
 
 // Token-major tensor [rows, heads, 128] bf16: coordinates (d, head, row), box 64 x 1 x 128.
 bool map_token_major(CUtensorMap* map, const void* ptr, int rows, int heads, int box_rows = kTile) {
@@ -988,20 +991,45 @@ TcParams base_params(const QueryRows& q, const Candidates& c, int* status) {
 
 }  // namespace
 
+// A wait on an mbarrier that nothing ever arms: the bounded wait runs out after limit_ns, raises the status word and
+// the kernel returns normally.  Launched only by citrus_debug_expire_wait (the test of the time-out path).
+__global__ void expire_wait_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    mbar_wait_warp(smem_u32(&bar), 0, status, limit_ns);
+}
+
+cudaError_t tc_expire_wait(int* status, unsigned long long limit_ns, cudaStream_t s) {
+    expire_wait_kernel<<<1, 32, 0, s>>>(status, limit_ns);
+    return cudaGetLastError();
+}
+
 cudaError_t tc_init() {
-    if (g_encode != nullptr) return cudaSuccess;
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    // The driver entry point is per process; the kernels' shared-memory limits are per device.
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+    std::lock_guard<std::mutex> lk(g_init_mu);
+    if (g_encode == nullptr) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+        g_encode = reinterpret_cast<EncodeFn>(fn);
+    }
+    if (!g_device_ready.needs_setup(dev)) return cudaSuccess;
     e = cudaFuncSetAttribute(attn_lse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_lse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kColSmemBytes);
     if (e != cudaSuccess) return e;
-    g_encode = reinterpret_cast<EncodeFn>(fn);
+    g_device_ready.mark(dev);
     return cudaSuccess;
 }
 
@@ -1018,7 +1046,7 @@ int tc_lse_splits(int n_rows, int q_heads, int kv_heads, int m, int L, int n_att
     // The log-sum-exp items share a launch with the attention items.  When those leave SMs idle (fewer items than
     // SMs), split the key range so that there is about one short item per idle SM; otherwise keep whole sweeps,
     // because every extra item pays a CTA prologue.
-    const int kSMs = 148;
+    const int kSMs = sm_count();
     const int tiles = (m + kTile - 1) / kTile + (L + kTile - 1) / kTile;
     const int base_items = ((n_rows + kTile - 1) / kTile) * q_heads / lse_pack(n_rows, q_heads, kv_heads);
     const int idle = n_attn_items < kSMs ? kSMs - n_attn_items : 0;

@@ -51,6 +51,7 @@ class Workload:
     deferred_lm: bool = False  # language-modelling cache evicted by the next chunk (Section 4.1 order)
     position_shift: bool = False   # inputs without rotary embedding; embedded by cache slot every step
     rope_base: float = 10000.0
+    layerwise: bool = False    # one kept set per layer from head-summed scores (the paper's stated granularity)
 
     @property
     def torch_dtype(self):
@@ -87,6 +88,17 @@ PAPER_SHAPES = {
                                  n_planted=32, n_sinks=1),
     "paper_llama3_8b": Workload("paper_llama3_8b", 13, 1, 32, 8, 128, 768, 256, 16384, 64, "bf16", "individual",
                                 lm_window=64, n_planted=32, n_sinks=1),
+}
+
+
+# The other eviction policies of Section 4.1 on the Mistral-7B-shaped layer: standard chunked eviction (one cache,
+# scored by the chunk's own last 64 queries; the instruction only evicts in the last call) and the layer-wise
+# granularity (scores summed over the KV heads, one kept set for the whole layer).
+VARIANTS = {
+    "mistral7b_standard": Workload("mistral7b_standard", 2, 1, 32, 8, 128, 768, 512, 16384, 64, "bf16", "standard",
+                                   lm_window=64, n_planted=32, n_sinks=1),
+    "mistral7b_layerwise": Workload("mistral7b_layerwise", 2, 1, 32, 8, 128, 768, 512, 16384, 64, "bf16", "shared",
+                                    n_planted=32, n_sinks=1, layerwise=True),
 }
 
 

@@ -53,3 +53,25 @@ def test_reference_arm_under_torchrun_prints_one_line_from_rank0():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["cpu_baseline"]["kind"] == "oracle" and d["value"] > 0
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["unit"] == "tokens/s"
+
+
+def test_gpus_flag_without_a_launcher_starts_that_many_ranks():
+    # `python bench.py --gpus 2` with no launcher around it must become two ranks (one per GPU), not a silent 1-GPU
+    # run: the script re-executes itself under torch.distributed.run.  --dry-run stops each rank after the set-up,
+    # before any CUDA call, and prints the rank's share of the work.
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run", "--workload", "serving_mix"]
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=600, cwd=ROOT, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(ln) for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert sorted(d["rank"] for d in lines) == [0, 1]
+    assert all(d["n_gpus"] == 2 for d in lines)
+    shares = [d["sequences_of_this_rank"] for d in sorted(lines, key=lambda d: d["rank"])]
+    assert shares[0] == list(range(0, 16, 2)) and shares[1] == list(range(1, 16, 2))      # a slice of the 16 sequences each
+
+
+def test_rank_sequences_partition_the_batch():
+    import bench
+    for world in (1, 2, 3, 8):
+        parts = [bench.rank_sequences(16, r, world) for r in range(world)]
+        assert sorted(x for p in parts for x in p) == list(range(16))

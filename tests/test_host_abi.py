@@ -57,3 +57,37 @@ def test_null_and_unknown_handles(lib):
     assert lib.citrus_reset(bogus) == -1
     assert lib.citrus_poll_status(None) == -1
     assert lib.citrus_process_chunk(bogus, 0, None, None, None, 1, None, 1, None, None) == -1
+
+
+def test_per_device_setup_bookkeeping(tmp_path):
+    # The kernels' shared-memory limits and the static scratch address are per-device facts: the record of which
+    # devices have had their set-up (DeviceOnce in the library's internal header) is compiled here with the host
+    # compiler alone and driven as the launchers drive it.
+    import subprocess
+    src = tmp_path / "once.cpp"
+    src.write_text(r'''
+#include "citrus_internal.h"
+#include <cstdio>
+int main() {
+    citrus::DeviceOnce once;
+    int setups = 0;
+    const int order[] = {0, 0, 1, 0, 1, 63, 63};
+    for (int dev : order) {
+        if (once.needs_setup(dev)) { ++setups; once.mark(dev); }
+    }
+    if (setups != 3) { std::printf("setups %d\n", setups); return 1; }         // once per device, not once per process
+    if (once.needs_setup(0) || once.needs_setup(1) || once.needs_setup(63)) return 2;
+    if (!once.needs_setup(2)) return 3;                                         // an untouched device still needs it
+    // out-of-range ids are never recorded: the set-up simply runs every time
+    once.mark(64); once.mark(-1);
+    if (!once.needs_setup(64) || !once.needs_setup(-1)) return 4;
+    return 0;
+}
+''')
+    exe = tmp_path / "once"
+    inc = os.path.join(ROOT, "paper_2406_12018_b200", "csrc")
+    r = subprocess.run(["g++", "-std=c++17", "-I", inc, "-I", "/usr/local/cuda/include", str(src), "-o", str(exe)],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr[-2000:]
+    r = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert r.returncode == 0, (r.returncode, r.stdout)

@@ -628,7 +628,7 @@ def test_bench_batch_side_measurement_runs():
     # the --sequences option of bench.py (packed ragged-batch call, lanes chosen by the library) on a short run
     import json, os, subprocess, sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--sequences", "3", "--doc-tokens", "1536",
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--sequences", "3", "--doc-tokens", "1536", "--workload", "mistral7b_layer",
                         "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stderr[-2000:]
     line = json.loads(r.stdout.strip().splitlines()[-1])
