@@ -93,7 +93,7 @@ def check_cache_properties(ctx: Citrus, doc: wl.Document, layer: int, slot: int,
 
 
 def run_document(w: wl.Workload, ctx: Citrus, layer=0, slot=0, seq=0, n_tokens=None, oracle_chunks="all",
-                 layerwise=False, chunk_lengths=None, stats=None, unrounded=False, index_rule=True):
+                 layerwise=False, chunk_lengths=None, stats=None, unrounded=False, index_rule=True, out_tol=None):
     """Process one document through the library; compare with the oracle on `oracle_chunks`
     ("all" or a set of chunk numbers); property-check the cache after every chunk.
     index_rule=False: the kept sets are not compared (the oracle adopts the library's), only outputs, scores and the
@@ -141,7 +141,7 @@ def run_document(w: wl.Workload, ctx: Citrus, layer=0, slot=0, seq=0, n_tokens=N
                                     Qi64 if with_instr else None, forced)
             err = float(np.abs(out.to(torch.float64).cpu().numpy() - res.out).max())
             st["max_out_err"] = max(st["max_out_err"], err)
-            assert err <= tol, f"chunk {ci}: attention output error {err}"
+            assert err <= (tol if out_tol is None else out_tol), f"chunk {ci}: attention output error {err}"
             for cid in range(n_caches):
                 S_gpu = views[cid][0].to(torch.float64).cpu().numpy()
                 assert views[cid][2] == res.m_by_cache[cid]
