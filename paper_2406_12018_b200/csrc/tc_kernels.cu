@@ -724,7 +724,10 @@ struct ColSmem {
 };
 constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 8192;
 
-// grid: (candidate tiles, kv_heads).  Accumulator rows = 128 candidates, columns = scoring rows of one
+// grid: (kv_heads, candidate tiles) - the KV head varies fastest, so CTAs are dispatched in the order of their tile
+// index: the retained-cache tiles (which every scoring row sees) first, then the chunk's tiles, whose sweeps get
+// shorter and shorter under the causal mask; the short ones fill the tail of the last wave.
+// Accumulator rows = 128 candidates, columns = scoring rows of one
 // (head, row block); thread i owns candidate i and adds exp2(logit2 - lse2[row]) over its columns.
 __global__ void __launch_bounds__(kColThreads, 1)
 colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
@@ -740,7 +743,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     ColSmem* bars = reinterpret_cast<ColSmem*>(smem_raw + (sQ + kColStages * kTileBytes - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int kt = blockIdx.x, g = blockIdx.y;
+    const int kt = blockIdx.y, g = blockIdx.x;
     const int G = p.q_heads / p.kv_heads;
     const int n_cache_tiles = (p.m + kTile - 1) / kTile;
     const bool from_cache = kt < n_cache_tiles;
@@ -1101,7 +1104,7 @@ cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse_
     p.lse_in = lse_or_part; p.part = reinterpret_cast<float2*>(const_cast<float*>(lse_or_part));
     p.lse_stride = lse_stride; p.splits = splits; p.scores = scores; p.score_stride = score_stride;
     const int n_tiles = (c.m + kTile - 1) / kTile + (c.L + kTile - 1) / kTile;
-    dim3 grid(n_tiles, c.kv_heads);
+    dim3 grid(c.kv_heads, n_tiles);
     return launch_pdl(colsum_kernel, grid, kColThreads, kColSmemBytes, s, mp.Q, mp.CK, mp.SK, p);
 }
 
