@@ -284,7 +284,8 @@ constexpr int kStagesK = 2;             // K ring
 constexpr int kStagesV = 2;             // V ring
 constexpr int kVStageBytes = kTileBytes + kHalfBytes;   // a V tile and, right behind it, a [128 keys][64] block of ones
 constexpr int kAttnThreads = 352;       // 8 softmax warps, K-TMA warp, MMA warp, V-TMA warp
-constexpr int kColThreads = 320;        // 8 column-sum warps (two groups of four), 1 TMA warp, 1 MMA warp
+constexpr int kColGroups = 4;           // column-sum warp groups (four warps each), one S^T accumulator per group
+constexpr int kColThreads = (kColGroups * 4 + 2) * 32;   // the groups, 1 TMA warp, 1 MMA warp
 constexpr int kTmemCols = 512;
 constexpr uint32_t kTmemO = 256;        // O accumulator: 128 output columns + 16 columns that all hold the row sum of P
 constexpr uint32_t kTmemL = kTmemO + 128;
@@ -720,7 +721,7 @@ struct ColSmem {
     uint64_t k_full, q_full[kColStages], q_empty[kColStages], s_full[4], s_free[4], lse_full[8], drain;
     uint32_t tmem_base;
     alignas(16) float lse[8][kTile];          // log-sum-exp of the scoring rows of eight consecutive (head, row block)s
-    float acc_other[kTile];                   // partial column sums of the second warp group
+    float acc_other[kColGroups - 1][kTile];   // partial column sums of the other warp groups
 };
 constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 8192;
 
@@ -767,7 +768,8 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 9) tmem_alloc(smem_u32(&bars->tmem_base), kColTmemCols);
+    constexpr int kTmaWarp = kColGroups * 4, kMmaWarp = kColGroups * 4 + 1;
+    if (warp == kMmaWarp) tmem_alloc(smem_u32(&bars->tmem_base), kColTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -778,7 +780,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const uint32_t tmem = bars->tmem_base;
     auto tmS = [tmem](int b) { return tmem + (uint32_t)b * 128u; };
 
-    if (warp == 8) {
+    if (warp == kTmaWarp) {
         // TMA producer (converged warp)
         auto load_q = [&](int it) {
             const int s = it % kColStages;
@@ -795,7 +797,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (from_cache && !p.dep_first) asm volatile("griddepcontrol.wait;" ::: "memory");
         load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
         for (; it < nb && ok; ++it) ok = load_q(it);
-    } else if (warp == 9) {
+    } else if (warp == kMmaWarp) {
         // MMA issuer (converged warp)
         bool ok = mbar_wait_warp(smem_u32(&bars->k_full), 0, p.status);
         for (int it = 0; it < nb && ok; ++it) {
@@ -820,12 +822,15 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 #ifdef CITRUS_TRACE
         if (threadIdx.x == 0) atomicMax(&g_citrus_trace[246], ~global_ns());
 #endif
-        // Two groups of four warps: group 0 takes the even (head, row block) iterations (accumulators S[0], S[2]),
-        // group 1 the odd ones (S[1], S[3]); thread i of either group owns candidate i of the tile.
+        // kColGroups groups of four warps: group t takes the (head, row block) iterations it = t (mod kColGroups) and
+        // owns accumulator S[t]; thread i of every group owns candidate i of the tile.  With four warps per scheduler the
+        // exponentials of one group cover the tensor-memory loads, barrier round trips and Q.K^T latency of the others
+        // (two groups left the special-function pipe 40 % idle).
         const int group = warp >> 2;
         const int key_in_tile = (warp & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const float scale2 = kLog2e * rsqrtf((float)kD);
+        const uint64_t scale2x2 = pack_f32x2(scale2, scale2);
         const int j = kt < n_cache_tiles ? key_row0 + key_in_tile : p.m + key_row0 + key_in_tile;   // candidate index
         const int n_src = from_cache ? p.m : p.L;
         const bool key_ok = key_row0 + key_in_tile < n_src;
@@ -834,11 +839,12 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (p.causal && !from_cache) r_first = max(0, key_row0 + key_in_tile - p.t0);
         float acc = 0.f;
         bool ok = true;
-        // The log-sum-exp values of iteration `it2` (thread i brings row r0 + i) go to buffer it2 & 7.  The global
-        // load is issued one iteration of the group before its value is stored to shared memory, so its latency
-        // hides behind the exponentials in between.  A thread in iteration `it` publishes iteration it+2 into the
-        // buffer last read in iteration it-6; it has seen the MMA of `it`, which needed s_free of it-4 from all four
-        // warps of the group, so everybody has finished reading that buffer.
+        // The log-sum-exp values of iteration `it2` (thread i brings row r0 + i) go to buffer it2 & 7; a group reads
+        // only what it published itself.  The global load is issued one iteration of the group before its value is
+        // stored to shared memory, so its latency hides behind the exponentials in between.  A thread in iteration
+        // `it` publishes the group's next iteration into the buffer the group last read one iteration ago; it has
+        // seen the MMA of `it`, which needed s_free of that earlier iteration from all four warps of the group, so
+        // everybody has finished reading that buffer.
         auto fetch_lse = [&](int it2) -> float {
             const int h2 = g * G + it2 / rb_per_head;
             const int rr = (rb0 + it2 % rb_per_head) * kTile + key_in_tile;
@@ -863,13 +869,13 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             return lse;
         };
         auto publish_lse = [&](int it2, float lse) {
-            bars->lse[it2 & 7][key_in_tile] = lse;
+            bars->lse[it2 & 7][key_in_tile] = -lse;              // negated: the exponent is one fused multiply-add
             mbar_arrive_warp(smem_u32(&bars->lse_full[it2 & 7]));
         };
         float lse_next = INFINITY;
         if (nb > group) publish_lse(group, fetch_lse(group));
-        if (nb > group + 2) lse_next = fetch_lse(group + 2);
-        for (int it = group; it < nb; it += 2) {
+        if (nb > group + kColGroups) lse_next = fetch_lse(group + kColGroups);
+        for (int it = group; it < nb; it += kColGroups) {
             const int b = it & 3;
             const int rb = rb0 + it % rb_per_head;
             const int r0 = rb * kTile;
@@ -878,44 +884,69 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (it >> 2) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(160 + 3 * (it & 7));
-            if (it + 2 < nb) publish_lse(it + 2, lse_next);      // loaded one iteration ago
-            if (it + 4 < nb) lse_next = fetch_lse(it + 4);       // lands during this iteration's exponentials
+            if (it + kColGroups < nb) publish_lse(it + kColGroups, lse_next);      // loaded one iteration ago
+            if (it + 2 * kColGroups < nb) lse_next = fetch_lse(it + 2 * kColGroups);   // lands during this iteration's exponentials
             ok = mbar_wait_warp(smem_u32(&bars->lse_full[lb]), (it >> 3) & 1, p.status);
             if (!ok) break;
             if (warp == 0) CITRUS_TR(161 + 3 * (it & 7));
             tc_fence_after();
-            const float4* lse4 = reinterpret_cast<const float4*>(bars->lse[lb]);
+            const float4* nlse4 = reinterpret_cast<const float4*>(bars->lse[lb]);   // -lse (rows past the block end: -inf)
             const int c_lo = max(0, r_first - r0);                 // first column (scoring row) this candidate is visible to
             const int n_pieces = (ncols + 31) >> 5;                // the MMA wrote round_up(ncols, 32) columns
             float part[4] = {0.f, 0.f, 0.f, 0.f};
+            uint64_t part2[2] = {0ull, 0ull};
 #pragma unroll 1
             for (int c = 0; c < n_pieces; ++c) {
+                const int lo = c_lo - c * 32;                      // columns below lo do not see this candidate
+                if (__all_sync(0xffffffffu, lo >= 32)) continue;   // a piece that no candidate of the warp sees
                 uint32_t v[32];
                 tmem_ld32(tmS(b) + lane_base + c * 32, v);
                 tmem_wait_ld();
-                const int lo = c_lo - c * 32;                      // columns below lo do not see this candidate
+                if (__all_sync(0xffffffffu, lo <= 0)) {
+                    // every candidate of the warp sees the whole piece (always so away from the causal diagonal):
+                    // packed arithmetic, no predicates
 #pragma unroll
-                for (int q = 0; q < 32; q += 4) {
-                    const float4 l = lse4[c * 8 + (q >> 2)];        // rows past the block end carry +inf -> exp2 = 0
-                    float e0 = ex2(fmaf(__uint_as_float(v[q + 0]), scale2, -l.x));
-                    float e1 = ex2(fmaf(__uint_as_float(v[q + 1]), scale2, -l.y));
-                    float e2 = ex2(fmaf(__uint_as_float(v[q + 2]), scale2, -l.z));
-                    float e3 = ex2(fmaf(__uint_as_float(v[q + 3]), scale2, -l.w));
-                    part[0] += q + 0 >= lo ? e0 : 0.f;
-                    part[1] += q + 1 >= lo ? e1 : 0.f;
-                    part[2] += q + 2 >= lo ? e2 : 0.f;
-                    part[3] += q + 3 >= lo ? e3 : 0.f;
+                    for (int q = 0; q < 32; q += 4) {
+                        const float4 l = nlse4[c * 8 + (q >> 2)];
+                        float e0, e1, e2, e3;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[q + 0]), __uint_as_float(v[q + 1])), scale2x2, pack_f32x2(l.x, l.y)), e0, e1);
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[q + 2]), __uint_as_float(v[q + 3])), scale2x2, pack_f32x2(l.z, l.w)), e2, e3);
+                        part2[0] = add_f32x2(part2[0], pack_f32x2(ex2(e0), ex2(e1)));
+                        part2[1] = add_f32x2(part2[1], pack_f32x2(ex2(e2), ex2(e3)));
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 32; q += 4) {
+                        const float4 l = nlse4[c * 8 + (q >> 2)];
+                        float e0 = ex2(fmaf(__uint_as_float(v[q + 0]), scale2, l.x));
+                        float e1 = ex2(fmaf(__uint_as_float(v[q + 1]), scale2, l.y));
+                        float e2 = ex2(fmaf(__uint_as_float(v[q + 2]), scale2, l.z));
+                        float e3 = ex2(fmaf(__uint_as_float(v[q + 3]), scale2, l.w));
+                        part[0] += q + 0 >= lo ? e0 : 0.f;
+                        part[1] += q + 1 >= lo ? e1 : 0.f;
+                        part[2] += q + 2 >= lo ? e2 : 0.f;
+                        part[3] += q + 3 >= lo ? e3 : 0.f;
+                    }
                 }
+            }
+            {
+                float a0, a1, b0, b1;
+                unpack_f32x2(part2[0], a0, a1); unpack_f32x2(part2[1], b0, b1);
+                part[0] += a0; part[1] += a1; part[2] += b0; part[3] += b1;
             }
             tc_fence_before();
             mbar_arrive_warp(smem_u32(&bars->s_free[b]));
             acc += (part[0] + part[1]) + (part[2] + part[3]);
             if (warp == 0) CITRUS_TR(162 + 3 * (it & 7));
         }
-        // all eight column-sum warps arrive here, also after a wait that gave up
-        if (group == 1) bars->acc_other[key_in_tile] = acc;
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (group == 0 && ok && key_ok) p.scores[(size_t)g * p.score_stride + j] = acc + bars->acc_other[key_in_tile];
+        // all column-sum warps arrive here, also after a wait that gave up; the partial sums are added in group order
+        if (group > 0) bars->acc_other[group - 1][key_in_tile] = acc;
+        asm volatile("bar.sync 1, %0;" ::"n"(kColGroups * 128) : "memory");
+        if (group == 0 && ok && key_ok) {
+#pragma unroll
+            for (int t = 0; t < kColGroups - 1; ++t) acc += bars->acc_other[t][key_in_tile];
+            p.scores[(size_t)g * p.score_stride + j] = acc;
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -923,7 +954,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 #ifdef CITRUS_TRACE
     if (threadIdx.x == 0) atomicMax(&g_citrus_trace[247], global_ns());
 #endif
-    if (warp == 9) { __syncwarp(); tmem_dealloc(tmem, kColTmemCols); }
+    if (warp == kMmaWarp) { __syncwarp(); tmem_dealloc(tmem, kColTmemCols); }
 }
 
 // ------------------------------------------------------------------ host side
