@@ -25,6 +25,13 @@ struct CacheBufs {
     int cur = 0;
 };
 
+// The caches of one (layer, cache id) for all sequence slots and both ping-pong halves live in ONE tensor
+// [2 x n_slots x kv_heads, cap, D] (positions / carried importance: [2 x n_slots x kv_heads, cap]), so that a single
+// tensor map covers them and a batched launch reaches every sequence's cache through a head offset.
+struct LayerCache {
+    void* K = nullptr; void* V = nullptr; void* Kraw = nullptr; int* pos = nullptr; float* carried = nullptr;
+};
+
 struct Unit {                       // one (layer, sequence slot)
     CacheBufs cache[2];
     float* scores = nullptr;        // [n_caches, kv_heads, score_stride]
@@ -58,6 +65,7 @@ struct citrus_ctx {
     int score_stride = 0;
     bool used = false;
     std::vector<Unit> units;        // [layers * n_slots]
+    std::vector<LayerCache> layer_cache;   // [layers * 2]
     std::vector<void*> allocs;      // cache buffers and per-unit scratch
     std::vector<void*> misc;        // status word, host-variant staging
     int* status = nullptr;
@@ -118,6 +126,7 @@ void free_units(citrus_ctx* c) {
     for (void* p : c->allocs) cudaFree(p);
     c->allocs.clear();
     c->units.clear();
+    c->layer_cache.clear();
 }
 void free_copy_streams(citrus_ctx* c) {
     for (int b = 0; b < 2; ++b) {
@@ -168,20 +177,35 @@ void free_all(citrus_ctx* c) {
 int alloc_units(citrus_ctx* c) {
     const size_t row = (size_t)c->D * c->elt;
     c->units.assign((size_t)c->layers * c->n_slots, Unit());
-    for (Unit& u : c->units) {
-        int rc;
+    c->layer_cache.assign((size_t)c->layers * 2, LayerCache());
+    int rc;
+    for (int layer = 0; layer < c->layers; ++layer) {
         for (int ci = 0; ci < c->n_caches; ++ci) {
-            const size_t kv_bytes = (size_t)c->Hkv * c->cap[ci] * row;
-            for (int b = 0; b < 2; ++b) {
-                if ((rc = dev_alloc(c, &u.cache[ci].K[b], kv_bytes, true))) return rc;
-                if ((rc = dev_alloc(c, &u.cache[ci].V[b], kv_bytes, true))) return rc;
-                if (c->shift && (rc = dev_alloc(c, &u.cache[ci].Kraw[b], kv_bytes, true))) return rc;
-                if ((rc = dev_alloc(c, (void**)&u.cache[ci].pos[b], (size_t)c->Hkv * c->cap[ci] * sizeof(int), true))) return rc;
-                if (c->accumulate &&
-                    (rc = dev_alloc(c, (void**)&u.cache[ci].carried[b], (size_t)c->Hkv * c->cap[ci] * sizeof(float), true))) return rc;
+            LayerCache& lc = c->layer_cache[(size_t)layer * 2 + ci];
+            const size_t heads = (size_t)2 * c->n_slots * c->Hkv;           // ping-pong halves x slots x KV heads
+            const size_t kv_bytes = heads * c->cap[ci] * row;
+            if ((rc = dev_alloc(c, &lc.K, kv_bytes, true))) return rc;
+            if ((rc = dev_alloc(c, &lc.V, kv_bytes, true))) return rc;
+            if (c->shift && (rc = dev_alloc(c, &lc.Kraw, kv_bytes, true))) return rc;
+            if ((rc = dev_alloc(c, (void**)&lc.pos, heads * c->cap[ci] * sizeof(int), true))) return rc;
+            if (c->accumulate && (rc = dev_alloc(c, (void**)&lc.carried, heads * c->cap[ci] * sizeof(float), true))) return rc;
+            for (int slot = 0; slot < c->n_slots; ++slot) {
+                Unit& u = c->units[(size_t)layer * c->n_slots + slot];
+                for (int b = 0; b < 2; ++b) {
+                    const size_t first_head = ((size_t)b * c->n_slots + slot) * c->Hkv;
+                    const size_t off = first_head * c->cap[ci];
+                    u.cache[ci].K[b] = static_cast<char*>(lc.K) + off * row;
+                    u.cache[ci].V[b] = static_cast<char*>(lc.V) + off * row;
+                    if (c->shift) u.cache[ci].Kraw[b] = static_cast<char*>(lc.Kraw) + off * row;
+                    u.cache[ci].pos[b] = lc.pos + off;
+                    if (c->accumulate) u.cache[ci].carried[b] = lc.carried + off;
+                }
             }
-            if ((rc = dev_alloc(c, (void**)&u.idx[ci], (size_t)c->Hkv * c->cap[ci] * sizeof(int), true))) return rc;
         }
+    }
+    for (Unit& u : c->units) {
+        for (int ci = 0; ci < c->n_caches; ++ci)
+            if ((rc = dev_alloc(c, (void**)&u.idx[ci], (size_t)c->Hkv * c->cap[ci] * sizeof(int), true))) return rc;
         if ((rc = dev_alloc(c, (void**)&u.scores, (size_t)c->n_caches * c->Hkv * c->score_stride * sizeof(float), true))) return rc;
         if ((rc = dev_alloc(c, (void**)&u.lse_chunk, (size_t)c->Hq * c->ls * sizeof(float), true))) return rc;
         if ((rc = dev_alloc(c, (void**)&u.lse_instr, (size_t)c->Hq * CITRUS_MAX_INSTR * sizeof(float), true))) return rc;
@@ -227,10 +251,26 @@ struct LaunchTimer {                 // brackets one kernel launch with events w
     }
 };
 
-// The launch sequence of one chunk step; all pointers are device pointers.
-int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc, const void* Vc, int L,
-             const void* Qi, int nI, void* out, cudaStream_t st, int lane = -1, bool inputs_ordered = false) {
+// One sequence's chunk as the step launcher takes it; all pointers are device pointers to the sequence's own rows.
+struct StepIn {
+    int slot;
+    const void *Q, *K, *V, *Qi;
+    int L, nI;
+    void* out;
+};
+// The tensors that hold every sequence's rows of a batched call (null: a single sequence, its own tensors).
+struct PackedIn {
+    const void *Q, *K, *V, *Qi;
+    void* out;
+    int tok_rows, instr_rows;       // rows of Q / K / V / out and of Qi that the call spans
+};
+
+// The launch sequence of one chunk step for n sequences of one layer (n > 1: the tensor-core path without position
+// shift; every launch then covers all sequences).  The steps of different sequences are independent.
+int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn* packed, cudaStream_t st, int lane = -1,
+              bool inputs_ordered = false) {
     c->used = true;
+    if (n < 1 || n > kTcMaxBatch || (n > 1 && (!c->use_tc || c->shift || packed == nullptr))) return CITRUS_ERR_INVALID_ARG;
     if (c->shift && lane < 0) {
         // One embedding scratch per context: a step on another stream than the last one is ordered behind everything
         // enqueued there so far.  Steps that stay on one stream pay nothing.
@@ -245,134 +285,209 @@ int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc,
     void* const rotQ = lane >= 0 ? c->laneRotQ[lane] : c->rotQ;
     void* const rotK = lane >= 0 ? c->laneRotK[lane] : c->rotK;
     void* const rotQi = lane >= 0 ? c->laneRotQi[lane] : c->rotQi;
-    Unit& u = c->units[(size_t)layer * c->n_slots + slot];
-    if (u.tokens_seen + L > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
-    const bool lm_scoring = c->individual || (c->standard && nI == 0);   // cache 0 is scored by the chunk's own queries
-    const bool instr_scoring = nI > 0;
-
-    // sizes of each cache's step.  Deferred eviction (cache 0, when the chunk scores it): only the cache's own rows
-    // compete for the k places, all of the chunk's rows enter.
-    int mc[2], nc[2], kept[2], forced_from[2];
-    Candidates cand[2];
-    for (int ci = 0; ci < c->n_caches; ++ci) {
-        const CacheBufs& cb = u.cache[ci];
-        mc[ci] = u.m[ci]; nc[ci] = mc[ci] + L;
-        forced_from[ci] = nc[ci];
-        kept[ci] = nc[ci] < c->k ? nc[ci] : c->k;
-        if (c->deferred && ci == 0 && lm_scoring) {
-            kept[ci] = (mc[ci] < c->k ? mc[ci] : c->k) + L;
-            forced_from[ci] = mc[ci];
-        }
-        cand[ci] = Candidates{cb.K[cb.cur], cb.V[cb.cur], Kc, Vc, mc[ci], L, c->cap[ci], c->Hkv};
-    }
-    cudaError_t e;
-    const void* Kc_raw = Kc;                                      // what the compaction gathers
-    if (c->shift) {
-        // position shift: embed the chunk's queries and keys at rows m .. m+L-1 and the instruction queries behind them
-        RopeRows jobs[3] = {{Qc, rotQ, L, c->Hq, mc[0]}, {Kc, rotK, L, c->Hkv, mc[0]}, {Qi, rotQi, nI, c->Hq, mc[0] + L}};
-        LaunchTimer t(c, CITRUS_KERNEL_ROPE, st);
-        e = rope_rows(jobs, instr_scoring ? 3 : 2, c->D, c->elt, c->rope, st);
-        if (e != cudaSuccess) return cuda_rc(e);
-        Qc = rotQ; Kc = rotK; if (instr_scoring) Qi = rotQi;
-        for (int ci = 0; ci < c->n_caches; ++ci) cand[ci].chunkK = Kc;
-    }
+    const size_t qrow = (size_t)c->Hq * c->D * c->elt, krow = (size_t)c->Hkv * c->D * c->elt;
+    const int ic = c->individual ? 1 : 0;     // the cache scored by the instruction text
     // 1: the kernels wait for their predecessors in the stream before their first load of Q / K / Q_instr.  Needed when
-    // the embedding pre-pass above wrote them, and whenever the inputs may still be in the making: the call's first
+    // the embedding pre-pass wrote them, and whenever the inputs may still be in the making: the call's first
     // kernel is launched with programmatic stream serialisation, so a preceding kernel of the CALLER that signals
     // its dependents early could otherwise still be writing them.
     const int produced = (c->shift || !(c->inputs_ready || inputs_ordered)) ? 1 : 0;
-    QueryRows q_chunk{Qc, L, c->Hq, 1, 0, produced};
-    QueryRows q_instr{Qi, nI, c->Hq, 0, 0, produced};
-    float* scores[2] = {u.scores, u.scores + (size_t)c->Hkv * c->score_stride};
-    const int ic = c->individual ? 1 : 0;     // the cache scored by the instruction text
-    if (!instr_scoring) q_instr.rows = 0;
 
-    float* lse_chunk = lm_scoring ? u.lse_chunk : nullptr;        // only a2-L reads a1's row log-sum-exp
-    int splits = 1;
+    struct Sizes { int mc[2], nc[2], kept[2], forced_from[2]; bool lm_scoring, instr_scoring; };
+    std::vector<Sizes> sz(n);
+    std::vector<TcSeqStep> seq(n);
+    std::vector<SelectJob> sj;
+    std::vector<CompactJob> cj;
+    sj.reserve((size_t)n * c->n_caches); cj.reserve((size_t)n * c->n_caches);
+    bool any_lm = false, any_instr = false;
+    size_t gather_bytes = 0;
+    for (int i = 0; i < n; ++i) {
+        Unit& u = c->units[(size_t)layer * c->n_slots + in[i].slot];
+        const int L = in[i].L, nI = in[i].nI;
+        if (u.tokens_seen + L > 0x7fffffffLL) return CITRUS_ERR_SHAPE;
+        Sizes& z = sz[i];
+        z.lm_scoring = c->individual || (c->standard && nI == 0);   // cache 0 is scored by the chunk's own queries
+        z.instr_scoring = nI > 0;
+        any_lm |= z.lm_scoring; any_instr |= z.instr_scoring;
+        // sizes of each cache's step.  Deferred eviction (cache 0, when the chunk scores it): only the cache's own rows
+        // compete for the k places, all of the chunk's rows enter.
+        for (int ci = 0; ci < c->n_caches; ++ci) {
+            z.mc[ci] = u.m[ci]; z.nc[ci] = z.mc[ci] + L;
+            z.forced_from[ci] = z.nc[ci];
+            z.kept[ci] = z.nc[ci] < c->k ? z.nc[ci] : c->k;
+            if (c->deferred && ci == 0 && z.lm_scoring) {
+                z.kept[ci] = (z.mc[ci] < c->k ? z.mc[ci] : c->k) + L;
+                z.forced_from[ci] = z.mc[ci];
+            }
+        }
+        if (c->n_caches == 1) { z.mc[1] = z.mc[0]; z.nc[1] = z.nc[0]; z.kept[1] = z.kept[0]; z.forced_from[1] = z.forced_from[0]; }
+        TcSeqStep& q = seq[i];
+        q = TcSeqStep{};
+        q.L = L; q.nI = nI; q.ic = ic; q.produced = produced;
+        q.q_row0 = packed ? (int)((static_cast<const char*>(in[i].Q) - static_cast<const char*>(packed->Q)) / qrow) : 0;
+        q.kv_row0 = packed ? (int)((static_cast<const char*>(in[i].K) - static_cast<const char*>(packed->K)) / krow) : 0;
+        q.qi_row0 = (packed && nI > 0) ? (int)((static_cast<const char*>(in[i].Qi) - static_cast<const char*>(packed->Qi)) / qrow) : 0;
+        for (int ci = 0; ci < 2; ++ci) {
+            const int cc = ci < c->n_caches ? ci : 0;
+            q.m[ci] = z.mc[cc];
+            q.chead[ci] = (u.cache[cc].cur * c->n_slots + in[i].slot) * c->Hkv;
+            q.scores[ci] = u.scores + (size_t)cc * c->Hkv * c->score_stride;
+        }
+        q.score_stride = c->score_stride;
+        q.w = z.lm_scoring ? ((c->lm_window > 0 && c->lm_window < L) ? c->lm_window : L) : 0;
+        q.lse_chunk = z.lm_scoring ? u.lse_chunk : nullptr;           // only a2-L reads a1's row log-sum-exp
+        q.lse_instr = u.lse_instr; q.part = u.part;
+        q.splits = 1;
+        if (c->use_tc && z.instr_scoring)
+            // (chosen as for a call of this sequence alone, so that a batched step gives the same bits)
+            q.splits = tc_lse_splits(nI, c->Hq, c->Hkv, z.mc[ic], L, ((L + 127) / 128) * c->Hq);
+    }
+    // a batch shares one kernel template: either every sequence's a1 keeps its row log-sum-exp or none does
+    for (int i = 1; i < n; ++i)
+        if (sz[i].lm_scoring != sz[0].lm_scoring || sz[i].instr_scoring != sz[0].instr_scoring) return CITRUS_ERR_INVALID_ARG;
+
+    cudaError_t e = cudaSuccess;
+    const void *Qc = in[0].Q, *Kc = in[0].K, *Qi = in[0].Qi;       // single-sequence paths below (n == 1)
+    if (c->shift) {
+        // position shift: embed the chunk's queries and keys at rows m .. m+L-1 and the instruction queries behind them
+        const int m0 = sz[0].mc[0], L = in[0].L, nI = in[0].nI;
+        RopeRows jobs[3] = {{Qc, rotQ, L, c->Hq, m0}, {Kc, rotK, L, c->Hkv, m0}, {Qi, rotQi, nI, c->Hq, m0 + L}};
+        LaunchTimer t(c, CITRUS_KERNEL_ROPE, st);
+        e = rope_rows(jobs, sz[0].instr_scoring ? 3 : 2, c->D, c->elt, c->rope, st);
+        if (e != cudaSuccess) return cuda_rc(e);
+        Qc = rotQ; Kc = rotK; if (sz[0].instr_scoring) Qi = rotQi;
+    }
+
     if (c->use_tc) {
-        // a1 and pass 1 of a2-I (row log-sum-exp of the instruction queries, possibly split over key ranges): one launch
-        if (instr_scoring) splits = tc_lse_splits(nI, c->Hq, c->Hkv, mc[ic], L, ((L + 127) / 128) * c->Hq);
-        LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
-        e = tc_attention_lse(q_chunk, cand[0], out, lse_chunk, c->ls, q_instr, cand[ic], u.lse_instr, u.part,
-                             CITRUS_MAX_INSTR, splits, c->status, st);
+        TcTensors t{};
+        t.q_heads = c->Hq; t.kv_heads = c->Hkv;
+        if (packed != nullptr && !c->shift) {
+            t.Q = packed->Q; t.out = packed->out; t.q_rows = packed->tok_rows;
+            t.K = packed->K; t.V = packed->V; t.kv_rows = packed->tok_rows;
+            t.Qi = packed->Qi; t.qi_rows = packed->instr_rows;
+        } else {
+            t.Q = Qc; t.out = in[0].out; t.q_rows = in[0].L;
+            t.K = Kc; t.V = in[0].V; t.kv_rows = in[0].L;
+            t.Qi = Qi; t.qi_rows = in[0].nI;
+        }
+        for (int ci = 0; ci < 2; ++ci) {
+            const int cc = ci < c->n_caches ? ci : 0;
+            const LayerCache& lc = c->layer_cache[(size_t)layer * 2 + cc];
+            t.cacheK[ci] = lc.K; t.cacheV[ci] = lc.V; t.cap[ci] = c->cap[cc]; t.cache_heads[ci] = 2 * c->n_slots * c->Hkv;
+        }
+        {
+            // a1 and pass 1 of a2-I (row log-sum-exp of the instruction queries, possibly split over key ranges): one launch
+            LaunchTimer tm(c, CITRUS_KERNEL_ATTENTION, st);
+            e = tc_attention_lse(t, seq.data(), n, c->ls, CITRUS_MAX_INSTR, c->status, st);
+        }
+        if (e != cudaSuccess) return cuda_rc(e);
+        // a2-L (individual design, standard chunked eviction): votes of the chunk's last w queries on cache 0's candidates
+        if (any_lm) {
+            LaunchTimer tm(c, CITRUS_KERNEL_COLSUM, st);
+            e = tc_colsum(t, seq.data(), n, 0, c->ls, c->status, st);
+            if (e != cudaSuccess) return cuda_rc(e);
+        }
+        // a2-I pass 2: Eq. 1 column sums of the instruction queries over the instruction-side cache's candidates
+        if (any_instr) {
+            LaunchTimer tm(c, CITRUS_KERNEL_COLSUM, st);
+            e = tc_colsum(t, seq.data(), n, 1, CITRUS_MAX_INSTR, c->status, st);
+            if (e != cudaSuccess) return cuda_rc(e);
+        }
     } else {
+        Unit& u = c->units[(size_t)layer * c->n_slots + in[0].slot];
+        const Sizes& z = sz[0];
+        const int L = in[0].L, nI = in[0].nI;
+        Candidates cand[2];
+        for (int ci = 0; ci < c->n_caches; ++ci) {
+            const CacheBufs& cb = u.cache[ci];
+            cand[ci] = Candidates{cb.K[cb.cur], cb.V[cb.cur], Kc, in[0].V, z.mc[ci], L, c->cap[ci], c->Hkv};
+        }
+        QueryRows q_chunk{Qc, L, c->Hq, 1, 0, produced};
+        QueryRows q_instr{Qi, z.instr_scoring ? nI : 0, c->Hq, 0, 0, produced};
+        float* scores[2] = {u.scores, u.scores + (size_t)c->Hkv * c->score_stride};
+        float* lse_chunk = z.lm_scoring ? u.lse_chunk : nullptr;
         {
             LaunchTimer t(c, CITRUS_KERNEL_ATTENTION, st);
-            e = simt_attention(c->fp32, c->D, q_chunk, cand[0], out, lse_chunk, c->ls, st);
+            e = simt_attention(c->fp32, c->D, q_chunk, cand[0], in[0].out, lse_chunk, c->ls, st);
         }
-        if (e == cudaSuccess && instr_scoring) {
+        if (e == cudaSuccess && z.instr_scoring) {
             LaunchTimer t(c, CITRUS_KERNEL_SCORE_LSE, st);
             e = simt_attention(c->fp32, c->D, q_instr, cand[ic], nullptr, u.lse_instr, CITRUS_MAX_INSTR, st);
         }
-    }
-    if (e != cudaSuccess) return cuda_rc(e);
-
-    // a2-L (individual design, standard chunked eviction): votes of the chunk's last w queries on cache 0's candidates
-    if (lm_scoring) {
-        int w = c->lm_window > 0 && c->lm_window < L ? c->lm_window : L;
-        const char* q0 = reinterpret_cast<const char*>(Qc) + (size_t)(L - w) * c->Hq * c->D * c->elt;
-        QueryRows q_lm{q0, w, c->Hq, 1, L - w, produced};
-        LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
-        if (c->use_tc) e = tc_colsum(q_lm, cand[0], u.lse_chunk + (L - w), c->ls, 1, scores[0], c->score_stride, c->status, st);
-        else e = simt_colsum(c->fp32, c->D, q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, st);
         if (e != cudaSuccess) return cuda_rc(e);
+        if (z.lm_scoring) {
+            const int w = seq[0].w;
+            const char* q0 = reinterpret_cast<const char*>(Qc) + (size_t)(L - w) * qrow;
+            QueryRows q_lm{q0, w, c->Hq, 1, L - w, produced};
+            LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
+            e = simt_colsum(c->fp32, c->D, q_lm, cand[0], u.lse_chunk + (L - w), c->ls, scores[0], c->score_stride, st);
+            if (e != cudaSuccess) return cuda_rc(e);
+        }
+        if (z.instr_scoring) {
+            LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
+            e = simt_colsum(c->fp32, c->D, q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, st);
+            if (e != cudaSuccess) return cuda_rc(e);
+        }
     }
-    // a2-I pass 2: Eq. 1 column sums of the instruction queries over the instruction-side cache's candidates
-    if (instr_scoring) {
-        LaunchTimer t(c, CITRUS_KERNEL_COLSUM, st);
-        if (c->use_tc) e = tc_colsum(q_instr, cand[ic], splits > 1 ? u.part : u.lse_instr, CITRUS_MAX_INSTR, splits,
-                                     scores[ic], c->score_stride, c->status, st);
-        else e = simt_colsum(c->fp32, c->D, q_instr, cand[ic], u.lse_instr, CITRUS_MAX_INSTR, scores[ic], c->score_stride, st);
-    }
-    if (e != cudaSuccess) return cuda_rc(e);
 
-    // a3 + a4 for every cache
-    SelectJob sj[2];
-    CompactJob cj[2];
-    size_t gather_bytes = 0;
-    for (int ci = 0; ci < c->n_caches; ++ci) {
-        CacheBufs& cb = u.cache[ci];
-        int* idx = u.idx[ci];
-        sj[ci] = SelectJob{scores[ci], idx, c->score_stride, cb.pos[cb.cur], c->cap[ci], mc[ci], (int)u.tokens_seen,
-                           c->start_size, c->accumulate ? cb.carried[cb.cur] : nullptr,
-                           nc[ci], kept[ci], c->cap[ci], forced_from[ci]};
-        cj[ci] = CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
-                            cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, mc[ci],
-                            c->accumulate ? scores[ci] : nullptr, c->score_stride,
-                            c->accumulate ? cb.carried[cb.cur ^ 1] : nullptr, c->cap[ci], kept[ci],
-                            c->shift ? cb.Kraw[cb.cur] : nullptr, c->shift ? cb.Kraw[cb.cur ^ 1] : nullptr};
-        gather_bytes += (size_t)c->Hkv * kept[ci] * c->D * c->elt * 2;
+    // a3 + a4 for every cache of every sequence
+    for (int i = 0; i < n; ++i) {
+        Unit& u = c->units[(size_t)layer * c->n_slots + in[i].slot];
+        const Sizes& z = sz[i];
+        for (int ci = 0; ci < c->n_caches; ++ci) {
+            CacheBufs& cb = u.cache[ci];
+            int* idx = u.idx[ci];
+            float* scores = u.scores + (size_t)ci * c->Hkv * c->score_stride;
+            sj.push_back(SelectJob{scores, idx, c->score_stride, cb.pos[cb.cur], c->cap[ci], z.mc[ci], (int)u.tokens_seen,
+                                   c->start_size, c->accumulate ? cb.carried[cb.cur] : nullptr,
+                                   z.nc[ci], z.kept[ci], c->cap[ci], z.forced_from[ci]});
+            cj.push_back(CompactJob{cb.K[cb.cur], cb.V[cb.cur], cb.pos[cb.cur],
+                                    cb.K[cb.cur ^ 1], cb.V[cb.cur ^ 1], cb.pos[cb.cur ^ 1], idx, z.mc[ci],
+                                    c->accumulate ? scores : nullptr, c->score_stride,
+                                    c->accumulate ? cb.carried[cb.cur ^ 1] : nullptr, c->cap[ci], z.kept[ci],
+                                    c->shift ? cb.Kraw[cb.cur] : nullptr, c->shift ? cb.Kraw[cb.cur ^ 1] : nullptr,
+                                    in[i].K, in[i].V, (int)u.tokens_seen});       // the un-rotated chunk keys are what is gathered
+            gather_bytes += (size_t)c->Hkv * z.kept[ci] * c->D * c->elt * 2;
+        }
     }
+    const int n_jobs = (int)sj.size();
     // Small steps (a few MB to move) are latency-bound: one cluster launch does a3 and a4.  Large steps want every
     // SM streaming rows, which the clusters (idle while their first CTA selects) cannot give: two launches.
     if (!c->layerwise && !c->shift && gather_bytes <= ((size_t)8 << 20)) {
         // one cluster launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-        e = select_compact(sj, cj, c->n_caches, Kc_raw, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen,
-                           c->shift ? &c->rope : nullptr, c->elt, st);
+        e = select_compact(sj.data(), cj.data(), n_jobs, c->Hkv, c->D * c->elt, nullptr, c->elt, st);
         if (e != cudaSuccess) return cuda_rc(e);
     } else {
         {
             LaunchTimer t(c, CITRUS_KERNEL_SELECT, st);
-            e = select_topk(sj, c->n_caches, c->Hkv, c->layerwise ? 1 : 0, st);
+            e = select_topk(sj.data(), n_jobs, c->Hkv, c->layerwise ? 1 : 0, st);
         }
         if (e != cudaSuccess) return cuda_rc(e);
         {
             LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-            e = compact_kv(cj, c->n_caches, Kc_raw, Vc, c->Hkv, c->D * c->elt, (int)u.tokens_seen,
-                           c->shift ? &c->rope : nullptr, c->elt, st);
+            e = compact_kv(cj.data(), n_jobs, c->Hkv, c->D * c->elt, c->shift ? &c->rope : nullptr, c->elt, st);
         }
         if (e != cudaSuccess) return cuda_rc(e);
     }
 
-    for (int ci = 0; ci < c->n_caches; ++ci) {
-        u.cache[ci].cur ^= 1;
-        u.last_n[ci] = nc[ci]; u.last_kept[ci] = kept[ci]; u.last_m[ci] = mc[ci];
-        u.m[ci] = kept[ci];
+    for (int i = 0; i < n; ++i) {
+        Unit& u = c->units[(size_t)layer * c->n_slots + in[i].slot];
+        for (int ci = 0; ci < c->n_caches; ++ci) {
+            u.cache[ci].cur ^= 1;
+            u.last_n[ci] = sz[i].nc[ci]; u.last_kept[ci] = sz[i].kept[ci]; u.last_m[ci] = sz[i].mc[ci];
+            u.m[ci] = sz[i].kept[ci];
+        }
+        u.has_step = true;
+        u.tokens_seen += in[i].L;
     }
-    u.has_step = true;
-    u.tokens_seen += L;
     return CITRUS_OK;
+}
+
+int run_step(citrus_ctx* c, int layer, int slot, const void* Qc, const void* Kc, const void* Vc, int L,
+             const void* Qi, int nI, void* out, cudaStream_t st, int lane = -1, bool inputs_ordered = false) {
+    StepIn in{slot, Qc, Kc, Vc, Qi, L, nI, out};
+    return run_steps(c, layer, 1, &in, nullptr, st, lane, inputs_ordered);
 }
 
 }  // namespace
@@ -543,9 +658,42 @@ int citrus_process_chunk_batch(citrus_handle h, int layer, int n_active, const i
     }
     const size_t qrow = (size_t)h->Hq * h->D * h->elt, krow = (size_t)h->Hkv * h->D * h->elt;   // multiples of 16 bytes
     cudaStream_t caller = reinterpret_cast<cudaStream_t>(stream);
-    // Lanes: only where a step is small (its attention items make a few waves over the SMs at most), which is where a
-    // sequence's kernels wait for each other more than they compute.  Per-launch timing wants one stream, so profiled
-    // runs stay in the caller's stream; a position-shift context needs its per-lane embedding scratch.
+    // One grid over all sequences (tensor-core path, no position shift; unless citrus_set_batch_lanes asked for the
+    // per-sequence launches): every kernel of the step is launched once, its work items are those of all sequences -
+    // each sequence's longest sweeps first, the longest sequence first - and a sequence's rows and caches are
+    // offsets inside the packed tensors and the layer's cache tensors.
+    if (n_active > 1 && h->use_tc && !h->shift && h->lanes_wanted == 0) {
+        std::vector<int> order(n_active);
+        for (int i = 0; i < n_active; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+            return tok_offset[a + 1] - tok_offset[a] > tok_offset[b + 1] - tok_offset[b];
+        });
+        const char* q0 = reinterpret_cast<const char*>(Q) + qrow * tok_offset[0];
+        const char* k0 = reinterpret_cast<const char*>(K) + krow * tok_offset[0];
+        const char* v0 = reinterpret_cast<const char*>(V) + krow * tok_offset[0];
+        const char* qi0 = reinterpret_cast<const char*>(Q_instr) + qrow * instr_offset[0];
+        char* o0 = reinterpret_cast<char*>(out) + qrow * tok_offset[0];
+        PackedIn packed{q0, k0, v0, qi0, o0, tok_offset[n_active] - tok_offset[0], instr_offset[n_active] - instr_offset[0]};
+        for (int first = 0; first < n_active; first += kTcMaxBatch) {
+            const int cnt = std::min(kTcMaxBatch, n_active - first);
+            std::vector<StepIn> in(cnt);
+            for (int j = 0; j < cnt; ++j) {
+                const int i = order[first + j];
+                in[j] = StepIn{seq_slot[i],
+                               reinterpret_cast<const char*>(Q) + qrow * tok_offset[i], reinterpret_cast<const char*>(K) + krow * tok_offset[i],
+                               reinterpret_cast<const char*>(V) + krow * tok_offset[i], reinterpret_cast<const char*>(Q_instr) + qrow * instr_offset[i],
+                               tok_offset[i + 1] - tok_offset[i], instr_offset[i + 1] - instr_offset[i],
+                               reinterpret_cast<char*>(out) + qrow * tok_offset[i]};
+            }
+            int rc = run_steps(h, layer, cnt, in.data(), &packed, caller);
+            if (rc != CITRUS_OK) return rc;                  // only a launch failure can get here; earlier groups have advanced
+        }
+        return CITRUS_OK;
+    }
+    // Lanes (position-shift and fp32 contexts, or on request): only where a step is small (its attention items make a
+    // few waves over the SMs at most), which is where a sequence's kernels wait for each other more than they compute.
+    // Per-launch timing wants one stream, so profiled runs stay in the caller's stream; a position-shift context needs
+    // its per-lane embedding scratch.
     int n_lanes = 1;
     if (n_active > 1 && h->lane_fork != nullptr && !h->profiling &&
         (!h->shift || h->laneRotQi[citrus_ctx::kMaxLanes - 1] != nullptr)) {

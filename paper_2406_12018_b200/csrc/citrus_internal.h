@@ -77,15 +77,37 @@ cudaError_t tc_expire_wait(int* status, unsigned long long limit_ns, cudaStream_
 // Number of key splits for pass 1 of a2-I (1 = the pass writes final log-sum-exp values).
 int tc_lse_splits(int n_rows, int q_heads, int kv_heads, int m, int L, int n_attn_items);
 constexpr int kTcMaxLseSplits = 8;
-// One launch: a1 (qa over ca -> out, optional row log-sum-exp) and pass 1 of a2-I (qi over ci).  Either part
-// may be empty (rows == 0).  With splits > 1 the pass writes (max, sum) pairs to `part`
-// [splits, q_heads, lse_instr_stride] (float2), otherwise log-sum-exp values to lse_instr.
-cudaError_t tc_attention_lse(const QueryRows& qa, const Candidates& ca, void* out, float* lse_chunk, int lse_chunk_stride,
-                             const QueryRows& qi, const Candidates& ci, float* lse_instr, float* part, int lse_instr_stride,
-                             int splits, int* status, cudaStream_t s);
-// Pass 2: column sums; lse_or_part is the matching output of pass 1 (or a1's row log-sum-exp with splits = 1).
-cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse_or_part, int lse_stride, int splits,
-                      float* scores, int score_stride, int* status, cudaStream_t s);
+constexpr int kTcMaxBatch = 32;            // sequences of one batched launch
+
+// The tensors of one launch as its tensor maps see them: the packed token-major tensors of every sequence of the call
+// and the cache tensors of all slots.  A sequence's rows and its cache's heads are offsets inside them.
+struct TcTensors {
+    const void* Q; void* out; int q_rows;          // chunk queries / attention output [q_rows, q_heads, D]
+    const void* K; const void* V; int kv_rows;     // chunk keys / values [kv_rows, kv_heads, D]
+    const void* Qi; int qi_rows;                   // instruction queries [qi_rows, q_heads, D]
+    const void* cacheK[2]; const void* cacheV[2];  // cache id 0 (LM side / shared) and 1 (instruction): [cache_heads, cap, D]
+    int cap[2], cache_heads[2];
+    int q_heads, kv_heads;
+};
+// One sequence's step inside such a launch.
+struct TcSeqStep {
+    int L, q_row0, kv_row0;                // chunk rows; row offset of the sequence in Q / out and in K / V
+    int nI, qi_row0;                       // instruction rows (0: none) and their offset in Qi
+    int m[2], chead[2];                    // rows retained, and head offset inside the cache tensor, per cache id
+    int ic;                                // cache that the instruction scores (0 shared design, 1 individual design)
+    int w;                                 // chunk rows that score the LM-side cache (the last w), 0: none
+    float* lse_chunk;                      // row log-sum-exp of a1 [q_heads, lse_chunk_stride], or null when nothing reads it
+    float* lse_instr; float* part;         // pass 1 of a2-I: [q_heads, lse_instr_stride] / (max, sum) pairs per key split
+    int splits;
+    float* scores[2]; int score_stride;    // per cache id: [kv_heads, score_stride]
+    int produced;                          // 1: wait for the preceding kernels before the first load of Q / K / Qi
+};
+// One launch: a1 (chunk over [cache 0 ; chunk] -> out, optional row log-sum-exp) and pass 1 of a2-I of every sequence.
+cudaError_t tc_attention_lse(const TcTensors& t, const TcSeqStep* seq, int n, int lse_chunk_stride, int lse_instr_stride,
+                             int* status, cudaStream_t s);
+// Pass 2, one launch for all sequences.  which = 0: the chunk's last w rows score cache 0's candidates with a1's
+// probabilities; which = 1: the instruction rows score cache ic's candidates.
+cudaError_t tc_colsum(const TcTensors& t, const TcSeqStep* seq, int n, int which, int lse_stride, int* status, cudaStream_t s);
 
 // ---- select (a3) and compaction (a4) ---------------------------------------
 struct SelectJob {            // one per cache handled by the launch
@@ -116,18 +138,21 @@ struct CompactJob {
     // position shift: the un-rotated keys are what is gathered (old raw cache, caller's chunk K) and kept in
     // dstKraw; dstK receives them embedded by their new slot.  Null when the mode is off.
     const void* srcKraw; void* dstKraw;
+    // the chunk's rows of this job's sequence: token-major [L, kv_heads, D] (un-rotated keys), and the original
+    // position of its first token
+    const void* chunkK; const void* chunkV; int chunk_pos0;
 };
 // Rotary embedding in the half-split layout: element d pairs with d + D/2, the pair turns by pos * theta[d].
 struct RopeTable { double theta[64]; };
 // One tensor of the embedding pre-pass: token-major [rows, heads, D], row i embedded at position pos0 + i.
 struct RopeRows { const void* in; void* out; int rows, heads, pos0; };
 cudaError_t rope_rows(const RopeRows* jobs, int n_jobs, int D, int elt, const RopeTable& table, cudaStream_t s);
-// rope: table of the position shift, or null (the jobs' raw pointers are then null too); elt = bytes per element
-cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
-                       int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s);
+// rope: table of the position shift, or null (the jobs' raw pointers are then null too); elt = bytes per element.
+// Up to 2 * kTcMaxBatch jobs per launch (one per cache of every sequence of a batch).
+cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, int kv_heads, int row_bytes, const RopeTable* rope, int elt, cudaStream_t s);
 // a3 + a4 in one launch (per-head granularity): clusters of CTAs per (cache, KV head).
-cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
-                           int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s);
+cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, int kv_heads, int row_bytes,
+                           const RopeTable* rope, int elt, cudaStream_t s);
 // ratio[g] = |{positions of a} intersect {positions of b}| / rows_b over two ascending position lists per head
 cudaError_t intersection_ratio(const int* pos_a, int stride_a, int rows_a, const int* pos_b, int stride_b, int rows_b,
                                int kv_heads, float* ratio, cudaStream_t s);

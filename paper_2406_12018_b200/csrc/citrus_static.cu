@@ -68,16 +68,26 @@ extern "C" int citrus_importance_static(const void* Q_s, int n_s, const void* K,
         return CITRUS_ERR_CUDA;
     }
     // all candidates are "chunk" rows of a token-major tensor; there is no retained cache (m = 0)
-    Candidates cand{K, K, K, K, 0, n_keys, n_keys, kv_heads};
-    QueryRows q{Q_s, n_s, q_heads, 0, 0, 1};   // produced = 1: wait for earlier stream work before the first load of Q_s or K
     cudaError_t e;
     if (fp32) {
+        Candidates cand{K, K, K, K, 0, n_keys, n_keys, kv_heads};
+        QueryRows q{Q_s, n_s, q_heads, 0, 0, 1};   // produced = 1: wait for earlier stream work before the first load of Q_s or K
         e = simt_attention(true, head_dim, q, cand, nullptr, lse, lse_stride, st);
         if (e == cudaSuccess) e = simt_colsum(true, head_dim, q, cand, lse, lse_stride, scores, score_stride, st);
     } else {
-        const QueryRows none{nullptr, 0, q_heads, 0, 0, 0};
-        e = tc_attention_lse(none, cand, nullptr, nullptr, 0, q, cand, lse, nullptr, lse_stride, 1, status, st);
-        if (e == cudaSuccess) e = tc_colsum(q, cand, lse, lse_stride, 1, scores, score_stride, status, st);
+        TcTensors t{};
+        t.q_heads = q_heads; t.kv_heads = kv_heads;
+        t.Q = nullptr; t.out = nullptr; t.q_rows = 0;
+        t.K = K; t.V = K; t.kv_rows = n_keys;
+        t.Qi = Q_s; t.qi_rows = n_s;
+        for (int ci = 0; ci < 2; ++ci) { t.cacheK[ci] = K; t.cacheV[ci] = K; t.cap[ci] = n_keys; t.cache_heads[ci] = kv_heads; }   // never read: m = 0
+        TcSeqStep q{};
+        q.L = n_keys; q.nI = n_s; q.ic = 0; q.splits = 1; q.w = 0;
+        q.lse_chunk = nullptr; q.lse_instr = lse; q.part = nullptr;
+        q.scores[0] = scores; q.scores[1] = scores; q.score_stride = score_stride;
+        q.produced = 1;                            // wait for earlier stream work before the first load of Q_s or K
+        e = tc_attention_lse(t, &q, 1, 0, lse_stride, status, st);
+        if (e == cudaSuccess) e = tc_colsum(t, &q, 1, 1, lse_stride, status, st);
     }
     if (e != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
     return CITRUS_OK;

@@ -18,10 +18,13 @@ namespace citrus {
 namespace {
 
 constexpr int kSelThreads = 1024;
-constexpr int kMaxJobs = 2;
+// Jobs of one launch: one per cache of every sequence.  Two capacities, so that a single sequence's launch does not
+// carry the parameter block of a whole batch.
+constexpr int kJobsSingle = 2;
+constexpr int kJobsBatch = 2 * kTcMaxBatch;
 
-struct SelectArgs { SelectJob job[kMaxJobs]; };
-struct CompactArgs { CompactJob job[kMaxJobs]; RopeTable rope; int elt; };
+template <int CAP> struct SelectArgs { SelectJob job[CAP]; };
+template <int CAP> struct CompactArgs { CompactJob job[CAP]; RopeTable rope; int elt; };
 
 // A 16-byte piece of a key row embedded at position `pos`: `mine` holds elements [d0, d0 + E) of one half of the head
 // dimension, `other` the same elements of the other half (E = 8 bf16 or 4 fp32); lower: `mine` is the first half.
@@ -244,8 +247,9 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
     CITRUS_TR(15);
 }
 
+template <int CAP>
 __global__ void __launch_bounds__(kSelThreads)
-select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int layerwise) {
+select_topk_kernel(const __grid_constant__ SelectArgs<CAP> args, int kv_heads, int layerwise) {
     extern __shared__ uint32_t keys[];            // [largest n of the jobs]
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the scores are final after this
@@ -254,11 +258,13 @@ select_topk_kernel(const __grid_constant__ SelectArgs args, int kv_heads, int la
 
 // Rows [r_begin, r_end) of one (cache, head) are copied with 128-bit accesses, row_bytes/16 lanes per row.
 template <bool SHIFT>
-__device__ __forceinline__ void compact_rows_t(const CompactJob& job, const uint4* __restrict__ chunkK,
-                                             const uint4* __restrict__ chunkV, const int g, int kv_heads,
-                                             int row_vecs, int r_begin, int r_end, int chunk_pos0, const int* idx,
+__device__ __forceinline__ void compact_rows_t(const CompactJob& job, const int g, int kv_heads,
+                                             int row_vecs, int r_begin, int r_end, const int* idx,
                                              const RopeTable& rope, int elt) {
     const int cap = job.cap;
+    const uint4* __restrict__ chunkK = reinterpret_cast<const uint4*>(job.chunkK);
+    const uint4* __restrict__ chunkV = reinterpret_cast<const uint4*>(job.chunkV);
+    const int chunk_pos0 = job.chunk_pos0;
     constexpr bool shift = SHIFT;                     // position shift: gather un-rotated keys, embed by the new slot
     // idx[r] = candidate kept in row r of this head (global list, or the CTA's slice in shared memory)
     const int rows_per_pass = blockDim.x / row_vecs;
@@ -335,16 +341,16 @@ __device__ __forceinline__ void compact_rows_t(const CompactJob& job, const uint
 constexpr int kCompactThreads = 256;
 constexpr int kCompactRowsPerCta = 64;
 
-template <bool SHIFT>
+template <bool SHIFT, int CAP>
 __global__ void __launch_bounds__(kCompactThreads)
-compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
-                  int kv_heads, int row_vecs, int chunk_pos0) {
+compact_kv_kernel(const __grid_constant__ CompactArgs<CAP> args, int kv_heads, int row_vecs) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the index lists are final after this
     const CompactJob& job = args.job[blockIdx.z];
     const int r0 = blockIdx.x * kCompactRowsPerCta;
-    compact_rows_t<SHIFT>(job, chunkK, chunkV, blockIdx.y, kv_heads, row_vecs,
-                          r0, min(job.kept, r0 + kCompactRowsPerCta), chunk_pos0, job.idx + (size_t)blockIdx.y * job.cap, args.rope, args.elt);
+    if (r0 >= job.kept) return;                              // the grid is sized for the job that keeps most
+    compact_rows_t<SHIFT>(job, blockIdx.y, kv_heads, row_vecs,
+                          r0, min(job.kept, r0 + kCompactRowsPerCta), job.idx + (size_t)blockIdx.y * job.cap, args.rope, args.elt);
 }
 
 // a3 + a4 in one launch: a cluster of kFusedCluster CTAs per (cache, KV head).  The first CTA of the cluster
@@ -354,9 +360,10 @@ compact_kv_kernel(const __grid_constant__ CompactArgs args, const uint4* __restr
 // grid: (kFusedCluster, KV heads, caches), cluster (kFusedCluster, 1, 1)
 constexpr int kFusedCluster = 8;
 
+template <int CAP>
 __global__ void __launch_bounds__(kSelThreads)
-select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_constant__ CompactArgs cmp, const uint4* __restrict__ chunkK, const uint4* __restrict__ chunkV,
-                      int kv_heads, int n_max, int row_vecs, int chunk_pos0) {
+select_compact_kernel(const __grid_constant__ SelectArgs<CAP> sel, const __grid_constant__ CompactArgs<CAP> cmp,
+                      int kv_heads, int n_max, int row_vecs) {
     extern __shared__ uint32_t keys[];            // [n_max] order keys (selecting CTA only), then this CTA's slice of the list
     const int g = blockIdx.y;
     const int kept = cmp.job[blockIdx.z].kept;
@@ -386,8 +393,7 @@ select_compact_kernel(const __grid_constant__ SelectArgs sel, const __grid_const
     CITRUS_TR(16);
     const int r0 = blockIdx.x * per;
     // (the position shift always takes the two-kernel route: its rotation does not fit this kernel's 64 registers)
-    compact_rows_t<false>(cmp.job[blockIdx.z], chunkK, chunkV, g, kv_heads, row_vecs, r0, min(kept, r0 + per), chunk_pos0, s_idx - r0,
-                          cmp.rope, cmp.elt);
+    compact_rows_t<false>(cmp.job[blockIdx.z], g, kv_heads, row_vecs, r0, min(kept, r0 + per), s_idx - r0, cmp.rope, cmp.elt);
     CITRUS_SPAN_MAX(2);
     CITRUS_TR(17);
 }
@@ -458,8 +464,10 @@ cudaError_t raise_smem_limits() {
     if (e != cudaSuccess) return e;
     std::lock_guard<std::mutex> lk(g_attr_mu);
     if (!g_attr_ready.needs_setup(dev)) return cudaSuccess;
-    e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    e = cudaFuncSetAttribute(select_topk_kernel<kJobsSingle>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_topk_kernel<kJobsBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_compact_kernel<kJobsSingle>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_compact_kernel<kJobsBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     g_attr_ready.mark(dev);
     return cudaSuccess;
@@ -496,16 +504,12 @@ cudaError_t intersection_ratio(const int* pos_a, int stride_a, int rows_a, const
     return cudaGetLastError();
 }
 
-cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int layerwise, cudaStream_t s) {
-    if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
-    SelectArgs a;
+template <int CAP>
+static cudaError_t launch_select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int layerwise, cudaStream_t s) {
+    SelectArgs<CAP> a;
     int n = 0;
     for (int i = 0; i < n_jobs; ++i) { a.job[i] = jobs[i]; n = jobs[i].n > n ? jobs[i].n : n; }
     size_t smem = (size_t)n * sizeof(uint32_t);
-    {
-        cudaError_t e = raise_smem_limits();
-        if (e != cudaSuccess) return e;
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(layerwise ? 1 : kv_heads, n_jobs);
     cfg.blockDim = dim3(kSelThreads);
@@ -516,23 +520,27 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int lay
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     before_launch(s);
-    return cudaLaunchKernelEx(&cfg, select_topk_kernel, a, kv_heads, layerwise);
+    return cudaLaunchKernelEx(&cfg, select_topk_kernel<CAP>, a, kv_heads, layerwise);
 }
 
-cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, const void* chunkK, const void* chunkV,
-                           int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s) {
-    if (n_jobs < 1 || n_jobs > kMaxJobs || rope != nullptr) return cudaErrorInvalidValue;
-    SelectArgs sa; CompactArgs ca;
+cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int layerwise, cudaStream_t s) {
+    if (n_jobs < 1 || n_jobs > kJobsBatch) return cudaErrorInvalidValue;
+    cudaError_t e = raise_smem_limits();
+    if (e != cudaSuccess) return e;
+    if (n_jobs <= kJobsSingle) return launch_select_topk<kJobsSingle>(jobs, n_jobs, kv_heads, layerwise, s);
+    return launch_select_topk<kJobsBatch>(jobs, n_jobs, kv_heads, layerwise, s);
+}
+
+template <int CAP>
+static cudaError_t launch_select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, int kv_heads, int row_bytes,
+                                         int elt, cudaStream_t s) {
+    SelectArgs<CAP> sa; CompactArgs<CAP> ca;
     ca.elt = elt;
     int n = 0, kept = 0;
     for (int i = 0; i < n_jobs; ++i) {
         sa.job[i] = sjobs[i]; ca.job[i] = cjobs[i];
         n = sjobs[i].n > n ? sjobs[i].n : n;
         kept = cjobs[i].kept > kept ? cjobs[i].kept : kept;
-    }
-    {
-        cudaError_t e = raise_smem_limits();
-        if (e != cudaSuccess) return e;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kFusedCluster, kv_heads, n_jobs);
@@ -546,14 +554,22 @@ cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int 
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
     before_launch(s);
-    return cudaLaunchKernelEx(&cfg, select_compact_kernel, sa, ca, reinterpret_cast<const uint4*>(chunkK),
-                              reinterpret_cast<const uint4*>(chunkV), kv_heads, n, row_bytes / 16, chunk_pos0);
+    return cudaLaunchKernelEx(&cfg, select_compact_kernel<CAP>, sa, ca, kv_heads, n, row_bytes / 16);
 }
 
-cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, const void* chunkV,
-                       int kv_heads, int row_bytes, int chunk_pos0, const RopeTable* rope, int elt, cudaStream_t s) {
-    if (n_jobs < 1 || n_jobs > kMaxJobs) return cudaErrorInvalidValue;
-    CompactArgs a;
+cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, int kv_heads, int row_bytes,
+                           const RopeTable* rope, int elt, cudaStream_t s) {
+    if (n_jobs < 1 || n_jobs > kJobsBatch || rope != nullptr) return cudaErrorInvalidValue;
+    cudaError_t e = raise_smem_limits();
+    if (e != cudaSuccess) return e;
+    if (n_jobs <= kJobsSingle) return launch_select_compact<kJobsSingle>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, s);
+    return launch_select_compact<kJobsBatch>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, s);
+}
+
+template <int CAP>
+static cudaError_t launch_compact_kv(const CompactJob* jobs, int n_jobs, int kv_heads, int row_bytes, const RopeTable* rope, int elt,
+                                     cudaStream_t s) {
+    CompactArgs<CAP> a;
     a.elt = elt;
     if (rope != nullptr) a.rope = *rope;
     int kept = 0;
@@ -568,11 +584,14 @@ cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, const void* chunkK, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     before_launch(s);
-    if (rope != nullptr)
-        return cudaLaunchKernelEx(&cfg, compact_kv_kernel<true>, a, reinterpret_cast<const uint4*>(chunkK),
-                                  reinterpret_cast<const uint4*>(chunkV), kv_heads, row_vecs, chunk_pos0);
-    return cudaLaunchKernelEx(&cfg, compact_kv_kernel<false>, a, reinterpret_cast<const uint4*>(chunkK),
-                              reinterpret_cast<const uint4*>(chunkV), kv_heads, row_vecs, chunk_pos0);
+    if (rope != nullptr) return cudaLaunchKernelEx(&cfg, compact_kv_kernel<true, CAP>, a, kv_heads, row_vecs);
+    return cudaLaunchKernelEx(&cfg, compact_kv_kernel<false, CAP>, a, kv_heads, row_vecs);
+}
+
+cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, int kv_heads, int row_bytes, const RopeTable* rope, int elt, cudaStream_t s) {
+    if (n_jobs < 1 || n_jobs > kJobsBatch) return cudaErrorInvalidValue;
+    if (n_jobs <= kJobsSingle) return launch_compact_kv<kJobsSingle>(jobs, n_jobs, kv_heads, row_bytes, rope, elt, s);
+    return launch_compact_kv<kJobsBatch>(jobs, n_jobs, kv_heads, row_bytes, rope, elt, s);
 }
 
 }  // namespace citrus

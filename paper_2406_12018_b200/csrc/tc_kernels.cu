@@ -219,7 +219,9 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, int b_mn_major) {
 // ------------------------------------------------------------------ parameters
 struct TcParams {
     int rows;        // query rows in the block
-    int row0;        // row offset of the block inside the Q tensor map
+    int row0;        // row offset of the block inside the Q tensor map (and of its output rows inside the out map)
+    int krow0;       // row offset of this sequence's chunk keys / values inside the chunk K / V maps
+    int chead;       // head offset of this sequence's retained cache inside the cache maps
     int q_heads, kv_heads;
     int m, L;        // retained rows, chunk rows
     int causal, t0;  // row r sees chunk keys u <= t0 + r
@@ -405,8 +407,8 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 const uint32_t bar = smem_u32(&bars->q_full);
                 mbar_expect_tx(bar, (uint32_t)(p.pack * p.pack_rows * 256));
                 for (int hh = 0; hh < p.pack; ++hh) {
-                    tma_load_3d(sQ + hh * p.pack_rows * 128, &mapQ, bar, 0, h + hh, 0);
-                    tma_load_3d(sQ + kHalfBytes + hh * p.pack_rows * 128, &mapQ, bar, 64, h + hh, 0);
+                    tma_load_3d(sQ + hh * p.pack_rows * 128, &mapQ, bar, 0, h + hh, p.row0);
+                    tma_load_3d(sQ + kHalfBytes + hh * p.pack_rows * 128, &mapQ, bar, 64, h + hh, p.row0);
                 }
             }
             __syncwarp();
@@ -416,7 +418,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
         for (int j = 0; j < nt; ++j) {
             const int s = j % kStagesK, jg = sweep_tile(j);
             const bool from_cache = jg < n_cache_tiles;
-            const int row = from_cache ? jg * kTile : (jg - n_cache_tiles) * kTile;
+            const int row = from_cache ? jg * kTile : p.krow0 + (jg - n_cache_tiles) * kTile;
             if (from_cache && !dep_waited) {
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 dep_waited = true;
@@ -425,7 +427,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
 #endif
             }
             if (!mbar_wait_warp(smem_u32(&bars->k_empty[s]), ((j / kStagesK) & 1) ^ 1, p.status)) break;
-            load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, g, !from_cache);
+            load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, from_cache ? p.chead + g : g, !from_cache);
         }
     } else if (warp == 10) {
         // ---------------------------------------------------------------- V TMA producer (converged warp)
@@ -434,10 +436,10 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             for (int j = 0; j < nt; ++j) {
                 const int s = j % kStagesV, jg = sweep_tile(j);
                 const bool from_cache = jg < n_cache_tiles;
-                const int row = from_cache ? jg * kTile : (jg - n_cache_tiles) * kTile;
+                const int row = from_cache ? jg * kTile : p.krow0 + (jg - n_cache_tiles) * kTile;
                 if (from_cache && !dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
                 if (!mbar_wait_warp(smem_u32(&bars->v_empty[s]), ((j / kStagesV) & 1) ^ 1, p.status)) break;
-                load_tile(sV + s * kVStageBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, g, !from_cache);
+                load_tile(sV + s * kVStageBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, from_cache ? p.chead + g : g, !from_cache);
             }
         }
     } else if (warp == 9) {
@@ -518,9 +520,17 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive_warp(smem_u32(&bars->s_free[b]));
-            // ---- row maximum over all 128 columns.  Hidden columns (future tokens of the chunk, rows past the end of
-            // the cache or chunk, which TMA zero-fills) take part: the result only serves as the exponent reference,
-            // any finite value near the visible maximum does, and both threads of the row still agree on it.
+            // ---- row maximum over the visible columns.  A tile that holds hidden columns (future tokens of the chunk,
+            // rows past the end of the cache or chunk - zero fill, stale cache rows, or in a packed batch the next
+            // sequence's rows) has them set to -inf first, in both halves, so both threads of the row still agree.
+            if (lim < kTile) {
+                const int lim_own = lim - half * 64, lim_oth = lim - (half ^ 1) * 64;
+#pragma unroll
+                for (int q = 0; q < 64; ++q) {
+                    if (q >= lim_own) own[q] = 0xff800000u;          // -inf
+                    if (q >= lim_oth) oth[q] = 0xff800000u;
+                }
+            }
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int q = 0; q < 64; q += 2) {
@@ -534,11 +544,14 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 m_ref = m_new;
             } else {
                 // both threads of a row see the same values, so they take the same decision
-                const bool grow = (m_new - m_ref) > kRescaleTau;
+                const bool grow = m_new > m_ref + kRescaleTau;       // also when the row has seen nothing so far (m_ref = -inf)
                 if (__any_sync(0xffffffffu, grow)) {
-                    const float f = ex2(m_ref - m_new);
-                    l_run *= f;
-                    m_ref = m_new;
+                    // Only the rows that grew change their reference; the others scale by exactly one.  A row's
+                    // arithmetic therefore never depends on what the other rows of its warp hold (in a packed batch
+                    // the rows past a sequence's end are the next sequence's), and results are the same bits whether
+                    // a sequence is stepped alone or inside a batch.
+                    const float f = grow ? ex2(m_ref - m_new) : 1.f;
+                    if (grow) { l_run *= f; m_ref = m_new; }
                     if (WITH_PV) {
                         // O must be quiescent: P.V of tile j-1 (and with it every earlier one) has retired
                         ok = pv_done(j - 1);
@@ -570,12 +583,6 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             const uint64_t neg_m2 = pack_f32x2(neg_m, neg_m);
             uint64_t sum2[2] = {0ull, 0ull};
             uint32_t packed[32];
-            if (lim - half * 64 < 64) {                              // hidden columns get probability zero
-                const int lim_own = lim - half * 64;
-#pragma unroll
-                for (int q = 0; q < 64; ++q)
-                    if (q >= lim_own) own[q] = 0xff800000u;          // -inf
-            }
             if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 202 : 52) + 5 * j);
 #pragma unroll
             for (int q = 0; q < 32; ++q) {
@@ -620,6 +627,11 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 tmem_wait_ld();
                 const float inv = 1.f / __uint_as_float(lreg[0]);
                 uint8_t* stage = gQ + half * kHalfBytes + row_in_tile * 128;   // [128 rows][64 bf16], 128-byte swizzle
+                // A tile that reaches past the block's last row is written row by row (a bulk store would run into the
+                // rows of the next sequence of a packed batch); whole tiles go through shared memory and TMA.
+                const bool whole_tile = q_row0 + kTile <= p.rows;
+                uint4* direct = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) +
+                                                         ((size_t)(p.row0 + r) * p.q_heads + h) * kD + half * 64);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t o0[32];
@@ -634,16 +646,17 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                         u.x = pack_bf16(v[0], v[1]); u.y = pack_bf16(v[2], v[3]);
                         u.z = pack_bf16(v[4], v[5]); u.w = pack_bf16(v[6], v[7]);
                         const int chunk = c * 4 + q;                 // 16-byte chunk inside the 128-byte row
-                        *reinterpret_cast<uint4*>(stage + ((chunk ^ (row_in_tile & 7)) << 4)) = u;
+                        if (whole_tile) *reinterpret_cast<uint4*>(stage + ((chunk ^ (row_in_tile & 7)) << 4)) = u;
+                        else if (r < p.rows) direct[chunk] = u;
                     }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_arrive_warp(smem_u32(&bars->out_ready[half]));
-                if ((warp & 3) == 0) {
+                if (whole_tile && (warp & 3) == 0) {
                     // one warp per column half stores its 128 x 64 part of the output tile
                     if (mbar_wait_warp(smem_u32(&bars->out_ready[half]), 0, p.status)) {
                         if (elect_one()) {
-                            tma_store_3d(&mapO, sQ + half * kHalfBytes, half * 64, h, q_row0);
+                            tma_store_3d(&mapO, sQ + half * kHalfBytes, half * 64, h, p.row0 + q_row0);
                             tma_store_wait_read();
                         }
                         __syncwarp();
@@ -673,32 +686,47 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
     if (warp == 9) { __syncwarp(); tmem_dealloc(tmem, kTmemCols); }
 }
 
-// One launch for a1 and for pass 1 of a2-I.  Blocks [0, n_attn) are attention items (query tile, head),
-// longest first; the rest are log-sum-exp items (instruction row tile, head, key split), which fill the SMs
-// that a partial wave of attention items leaves idle.
-//   pa / maps Q, CK, CV, SK, SV, O : attention of the chunk over [cache 0 ; chunk]
-//   pl / maps QI, CKI, SK          : instruction queries over [instruction-side cache ; chunk]
-template <bool NEED_LSE>
+// One launch for a1 and for pass 1 of a2-I of every sequence of a batch (CAP = 1: a single sequence).  The grid is
+// a list of segments: first the attention items (query tile, head) of sequence 0, 1, ... - each sequence's longest
+// sweeps first - then the log-sum-exp items (instruction row tile, head, key split) of sequence 0, 1, ..., which fill
+// the SMs that a partial wave of attention items leaves idle.
+//   pa[s] / maps Q, CK, CV, SK, SV, O : attention of the chunk over [cache 0 ; chunk]
+//   pl[s] / maps QI, CKI, SK          : instruction queries over [instruction-side cache ; chunk]
+// The maps cover the packed tensors of the whole batch; a sequence's rows and cache heads are offsets in them.
+template <int CAP>
+struct AttnBatch {
+    int n;                       // sequences
+    int seg_end[2 * CAP];        // exclusive end of every segment in the 1-D grid
+    TcParams pa[CAP], pl[CAP];
+};
+template <bool NEED_LSE, int CAP>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
                 const __grid_constant__ CUtensorMap mapCV, const __grid_constant__ CUtensorMap mapSK,
                 const __grid_constant__ CUtensorMap mapSV, const __grid_constant__ CUtensorMap mapO,
                 const __grid_constant__ CUtensorMap mapQI, const __grid_constant__ CUtensorMap mapCKI,
-                const TcParams pa, const TcParams pl, const int n_attn) {
+                const __grid_constant__ AttnBatch<CAP> bt) {
     extern __shared__ uint8_t smem_raw[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int id = blockIdx.x;
+    int id = blockIdx.x, seg = 0;
+    if (CAP > 1) {
+        while (seg + 1 < 2 * bt.n && id >= bt.seg_end[seg]) ++seg;
+        if (seg > 0) id -= bt.seg_end[seg - 1];
+    } else if (id >= bt.seg_end[0]) {
+        id -= bt.seg_end[0]; seg = 1;
+    }
 #ifdef CITRUS_TRACE
     unsigned long long t_start = 0;
     if (threadIdx.x == 0) { t_start = global_ns(); atomicMax(&g_citrus_trace[240], ~t_start); }   // complemented: max = earliest
 #endif
-    if (id < n_attn) {
+    if (seg < bt.n) {
+        const TcParams& pa = bt.pa[seg];
         const int n_qt = (pa.rows + kTile - 1) / kTile;
         const int qt = n_qt - 1 - id / pa.q_heads, h = id % pa.q_heads;      // later query tiles see more keys
         attn_body<true, NEED_LSE>(mapQ, mapCK, mapCV, mapSK, mapSV, mapO, pa, qt, h, 0, 1 << 30, 0, smem_raw);
     } else {
-        const int item = id - n_attn;
-        const int split = item % pl.splits, rest = item / pl.splits;
+        const TcParams& pl = bt.pl[seg - bt.n];
+        const int split = id % pl.splits, rest = id / pl.splits;
         const int head_slots = pl.q_heads / pl.pack;
         const int h = (rest % head_slots) * pl.pack, rt = rest / head_slots;
         const int tiles = (pl.m + kTile - 1) / kTile + (pl.L + kTile - 1) / kTile;
@@ -709,7 +737,7 @@ attn_lse_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (threadIdx.x == 0) {
         const unsigned long long t_end = global_ns();
         atomicMax(&g_citrus_trace[241], t_end);
-        atomicMax(&g_citrus_trace[id < n_attn ? 242 : 243], t_end - t_start);   // longest attention / log-sum-exp item
+        atomicMax(&g_citrus_trace[seg < bt.n ? 242 : 243], t_end - t_start);   // longest attention / log-sum-exp item
     }
 #endif
 }
@@ -730,11 +758,25 @@ constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 8192;
 // shorter and shorter under the causal mask; the short ones fill the tail of the last wave.
 // Accumulator rows = 128 candidates, columns = scoring rows of one
 // (head, row block); thread i owns candidate i and adds exp2(logit2 - lse2[row]) over its columns.
+// A batch: blockIdx.y runs over the candidate tiles of sequence 0, 1, ... (tile_end = exclusive prefix ends).
+template <int CAP>
+struct ColBatch {
+    int n;
+    int tile_end[CAP];
+    TcParams p[CAP];
+};
+template <int CAP>
 __global__ void __launch_bounds__(kColThreads, 1)
 colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
-              const __grid_constant__ CUtensorMap mapSK, const TcParams p) {
+              const __grid_constant__ CUtensorMap mapSK, const __grid_constant__ ColBatch<CAP> bt) {
     extern __shared__ uint8_t smem_raw[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    int seq = 0, kt = blockIdx.y;
+    if (CAP > 1) {
+        while (seq + 1 < bt.n && kt >= bt.tile_end[seq]) ++seq;
+        if (seq > 0) kt -= bt.tile_end[seq - 1];
+    }
+    const TcParams& p = bt.p[seq];
 #ifdef CITRUS_TRACE
     if (threadIdx.x == 0) atomicMax(&g_citrus_trace[245], ~global_ns());
 #endif
@@ -744,7 +786,7 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     ColSmem* bars = reinterpret_cast<ColSmem*>(smem_raw + (sQ + kColStages * kTileBytes - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int kt = blockIdx.y, g = blockIdx.x;
+    const int g = blockIdx.x;
     const int G = p.q_heads / p.kv_heads;
     const int n_cache_tiles = (p.m + kTile - 1) / kTile;
     const bool from_cache = kt < n_cache_tiles;
@@ -795,7 +837,8 @@ colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         if (p.dep_first) asm volatile("griddepcontrol.wait;" ::: "memory");
         for (; it < nb && it < kColStages && ok; ++it) ok = load_q(it);
         if (from_cache && !p.dep_first) asm volatile("griddepcontrol.wait;" ::: "memory");
-        load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), key_row0, g, !from_cache);
+        load_tile(sK, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full), from_cache ? key_row0 : p.krow0 + key_row0,
+                  from_cache ? p.chead + g : g, !from_cache);
         for (; it < nb && ok; ++it) ok = load_q(it);
     } else if (warp == kMmaWarp) {
         // MMA issuer (converged warp)
@@ -986,22 +1029,6 @@ bool map_cache(CUtensorMap* map, const void* ptr, int cap, int heads) {
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct Maps { CUtensorMap Q, CK, CV, SK, SV, O; };
-
-// The tensor map's row extent is the number of valid rows, so rows past it read as zero.
-bool build_maps(Maps* mp, const void* Qbase, int q_rows_total, const QueryRows& q, const Candidates& c, bool with_v) {
-    if (!map_token_major(&mp->Q, Qbase, q_rows_total, q.q_heads)) return false;
-    if (!map_cache(&mp->CK, c.cacheK, c.cap, c.kv_heads)) return false;
-    if (!map_token_major(&mp->SK, c.chunkK, c.L, c.kv_heads)) return false;
-    if (with_v) {
-        if (!map_cache(&mp->CV, c.cacheV, c.cap, c.kv_heads)) return false;
-        if (!map_token_major(&mp->SV, c.chunkV, c.L, c.kv_heads)) return false;
-    } else {
-        mp->CV = mp->CK; mp->SV = mp->SK;
-    }
-    return true;
-}
-
 // Launch with programmatic stream serialisation: the kernel may begin (prologue only) before its predecessor
 // in the stream has finished; it reads the predecessor's results after griddepcontrol.wait.
 template <typename... KArgs, typename... Args>
@@ -1014,13 +1041,6 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t 
     cfg.attrs = attr; cfg.numAttrs = 1;
     before_launch(s);
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
-}
-
-TcParams base_params(const QueryRows& q, const Candidates& c, int* status) {
-    TcParams p{};
-    p.rows = q.rows; p.row0 = 0; p.q_heads = q.q_heads; p.kv_heads = c.kv_heads;
-    p.m = c.m; p.L = c.L; p.causal = q.causal; p.t0 = q.t0; p.status = status; p.dep_first = q.produced;
-    return p;
 }
 
 }  // namespace
@@ -1057,11 +1077,12 @@ cudaError_t tc_init() {
         g_encode = reinterpret_cast<EncodeFn>(fn);
     }
     if (!g_device_ready.needs_setup(dev)) return cudaSuccess;
-    e = cudaFuncSetAttribute(attn_lse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_lse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kColSmemBytes);
+    e = cudaFuncSetAttribute(attn_lse_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_lse_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_lse_kernel<true, kTcMaxBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_lse_kernel<false, kTcMaxBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(colsum_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kColSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(colsum_kernel<kTcMaxBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, kColSmemBytes);
     if (e != cudaSuccess) return e;
     g_device_ready.mark(dev);
     return cudaSuccess;
@@ -1092,51 +1113,124 @@ int tc_lse_splits(int n_rows, int q_heads, int kv_heads, int m, int L, int n_att
     return s < 1 ? 1 : s;
 }
 
-cudaError_t tc_attention_lse(const QueryRows& qa, const Candidates& ca, void* out, float* lse_chunk, int lse_chunk_stride,
-                             const QueryRows& qi, const Candidates& ci, float* lse_instr, float* part, int lse_instr_stride,
-                             int splits, int* status, cudaStream_t s) {
-    const bool has_attn = qa.rows > 0, has_lse = qi.rows > 0;
-    if (!has_attn && !has_lse) return cudaSuccess;
-    Maps ma{}, mi{};
-    CUtensorMap mapO{};
-    if (has_attn) {
-        if (!build_maps(&ma, qa.Q, qa.rows, qa, ca, true)) return cudaErrorInvalidValue;
-        if (!map_token_major(&mapO, out, qa.rows, qa.q_heads)) return cudaErrorInvalidValue;
+// Largest pack that every sequence of the batch can use (they share one query map, whose box is pack_rows high).
+static int batch_pack(const TcSeqStep* seq, int n, int q_heads, int kv_heads) {
+    int rows = 0;
+    for (int i = 0; i < n; ++i) {
+        if (seq[i].nI <= 0) continue;
+        if (rows == 0) rows = seq[i].nI;
+        else if (rows != seq[i].nI) return 1;
     }
-    const int pack = has_lse ? lse_pack(qi.rows, qi.q_heads, ci.kv_heads) : 1;
-    if (has_lse) {
-        if (!build_maps(&mi, qi.Q, qi.rows, qi, ci, false)) return cudaErrorInvalidValue;
-        if (pack > 1 && !map_token_major(&mi.Q, qi.Q, qi.rows, qi.q_heads, qi.rows)) return cudaErrorInvalidValue;
-    }
-    if (!has_attn) { ma = mi; mapO = mi.Q; }
-    if (!has_lse) mi = ma;
-    TcParams pa = base_params(has_attn ? qa : qi, has_attn ? ca : ci, status);
-    pa.out = out; pa.lse2 = lse_chunk; pa.lse_stride = lse_chunk_stride; pa.splits = 1;
-    TcParams pl = base_params(has_lse ? qi : qa, has_lse ? ci : ca, status);
-    pl.lse2 = lse_instr; pl.part = reinterpret_cast<float2*>(part); pl.lse_stride = lse_instr_stride; pl.splits = splits;
-    pl.pack = pack; pl.pack_rows = qi.rows;
-    pa.pack = 1; pa.pack_rows = 0;
-    const int n_attn = has_attn ? ((qa.rows + kTile - 1) / kTile) * qa.q_heads : 0;
-    const int n_lse = has_lse ? ((qi.rows + kTile - 1) / kTile) * (qi.q_heads / pack) * splits : 0;
-    dim3 grid(n_attn + n_lse);
-    // both parts read the chunk's K through the same caller tensor, so one chunk-K map serves them
-    if (lse_chunk != nullptr)
-        return launch_pdl(attn_lse_kernel<true>, grid, kAttnThreads, kAttnSmemBytes, s, ma.Q, ma.CK, ma.CV, ma.SK, ma.SV, mapO,
-                          mi.Q, mi.CK, pa, pl, n_attn);
-    return launch_pdl(attn_lse_kernel<false>, grid, kAttnThreads, kAttnSmemBytes, s, ma.Q, ma.CK, ma.CV, ma.SK, ma.SV, mapO,
-                      mi.Q, mi.CK, pa, pl, n_attn);
+    return rows > 0 ? lse_pack(rows, q_heads, kv_heads) : 1;
 }
 
-cudaError_t tc_colsum(const QueryRows& q, const Candidates& c, const float* lse_or_part, int lse_stride, int splits,
-                      float* scores, int score_stride, int* status, cudaStream_t s) {
-    Maps mp;
-    if (!build_maps(&mp, q.Q, q.rows, q, c, false)) return cudaErrorInvalidValue;
-    TcParams p = base_params(q, c, status);
-    p.lse_in = lse_or_part; p.part = reinterpret_cast<float2*>(const_cast<float*>(lse_or_part));
-    p.lse_stride = lse_stride; p.splits = splits; p.scores = scores; p.score_stride = score_stride;
-    const int n_tiles = (c.m + kTile - 1) / kTile + (c.L + kTile - 1) / kTile;
-    dim3 grid(c.kv_heads, n_tiles);
-    return launch_pdl(colsum_kernel, grid, kColThreads, kColSmemBytes, s, mp.Q, mp.CK, mp.SK, p);
+template <int CAP>
+static cudaError_t launch_attention(const TcTensors& t, const TcSeqStep* seq, int n, int lse_chunk_stride, int lse_instr_stride,
+                                    int* status, cudaStream_t s) {
+    bool has_attn = false, has_lse = false, need_lse = false;
+    for (int i = 0; i < n; ++i) {
+        has_attn |= seq[i].L > 0 && t.out != nullptr;
+        has_lse |= seq[i].nI > 0;
+        need_lse |= seq[i].lse_chunk != nullptr;
+    }
+    if (!has_attn && !has_lse) return cudaSuccess;
+    const int ic = seq[0].ic;
+    CUtensorMap mQ{}, mCK{}, mCV{}, mSK{}, mSV{}, mO{}, mQI{}, mCKI{};
+    if (!map_token_major(&mSK, t.K, t.kv_rows, t.kv_heads)) return cudaErrorInvalidValue;
+    if (has_attn) {
+        if (!map_token_major(&mQ, t.Q, t.q_rows, t.q_heads) || !map_token_major(&mO, t.out, t.q_rows, t.q_heads) ||
+            !map_token_major(&mSV, t.V, t.kv_rows, t.kv_heads) ||
+            !map_cache(&mCK, t.cacheK[0], t.cap[0], t.cache_heads[0]) || !map_cache(&mCV, t.cacheV[0], t.cap[0], t.cache_heads[0]))
+            return cudaErrorInvalidValue;
+    }
+    const int pack = has_lse ? batch_pack(seq, n, t.q_heads, t.kv_heads) : 1;
+    int pack_rows = 0;
+    if (has_lse) {
+        for (int i = 0; i < n; ++i) if (seq[i].nI > 0) pack_rows = seq[i].nI;
+        if (!map_token_major(&mQI, t.Qi, t.qi_rows, t.q_heads, pack > 1 ? pack_rows : kTile) ||
+            !map_cache(&mCKI, t.cacheK[ic], t.cap[ic], t.cache_heads[ic]))
+            return cudaErrorInvalidValue;
+    }
+    if (!has_attn) { mQ = mQI; mO = mQI; mCK = mCKI; mCV = mCKI; mSV = mSK; }
+    if (!has_lse) { mQI = mQ; mCKI = mCK; }
+    AttnBatch<CAP> bt{};
+    bt.n = n;
+    int items = 0;
+    for (int i = 0; i < n; ++i) {
+        const TcSeqStep& q = seq[i];
+        TcParams& pa = bt.pa[i];
+        pa.rows = has_attn ? q.L : 0; pa.row0 = q.q_row0; pa.krow0 = q.kv_row0; pa.chead = q.chead[0];
+        pa.q_heads = t.q_heads; pa.kv_heads = t.kv_heads; pa.m = q.m[0]; pa.L = q.L; pa.causal = 1; pa.t0 = 0;
+        pa.out = t.out; pa.lse2 = q.lse_chunk; pa.lse_stride = lse_chunk_stride; pa.splits = 1; pa.pack = 1; pa.pack_rows = 0;
+        pa.status = status; pa.dep_first = q.produced;
+        items += ((pa.rows + kTile - 1) / kTile) * t.q_heads;
+        bt.seg_end[i] = items;
+    }
+    for (int i = 0; i < n; ++i) {
+        const TcSeqStep& q = seq[i];
+        TcParams& pl = bt.pl[i];
+        pl.rows = q.nI; pl.row0 = q.qi_row0; pl.krow0 = q.kv_row0; pl.chead = q.chead[ic];
+        pl.q_heads = t.q_heads; pl.kv_heads = t.kv_heads; pl.m = q.m[ic]; pl.L = q.L; pl.causal = 0; pl.t0 = 0;
+        pl.lse2 = q.lse_instr; pl.part = reinterpret_cast<float2*>(q.part); pl.lse_stride = lse_instr_stride;
+        pl.splits = q.splits < 1 ? 1 : q.splits; pl.pack = pack; pl.pack_rows = q.nI;
+        pl.status = status; pl.dep_first = q.produced;
+        items += ((q.nI + kTile - 1) / kTile) * (t.q_heads / pack) * pl.splits;
+        bt.seg_end[n + i] = items;
+    }
+    if (items == 0) return cudaSuccess;
+    dim3 grid(items);
+    if (need_lse)
+        return launch_pdl(attn_lse_kernel<true, CAP>, grid, kAttnThreads, kAttnSmemBytes, s, mQ, mCK, mCV, mSK, mSV, mO, mQI, mCKI, bt);
+    return launch_pdl(attn_lse_kernel<false, CAP>, grid, kAttnThreads, kAttnSmemBytes, s, mQ, mCK, mCV, mSK, mSV, mO, mQI, mCKI, bt);
+}
+
+cudaError_t tc_attention_lse(const TcTensors& t, const TcSeqStep* seq, int n, int lse_chunk_stride, int lse_instr_stride,
+                             int* status, cudaStream_t s) {
+    if (n < 1 || n > kTcMaxBatch) return cudaErrorInvalidValue;
+    if (n == 1) return launch_attention<1>(t, seq, n, lse_chunk_stride, lse_instr_stride, status, s);
+    return launch_attention<kTcMaxBatch>(t, seq, n, lse_chunk_stride, lse_instr_stride, status, s);
+}
+
+// which = 0: the chunk's last w rows score the LM-side cache's candidates with a1's probabilities (causal);
+// which = 1: the instruction rows score the instruction-side cache's candidates.
+template <int CAP>
+static cudaError_t launch_colsum(const TcTensors& t, const TcSeqStep* seq, int n, int which, int lse_stride, int* status, cudaStream_t s) {
+    const int ci = which == 0 ? 0 : seq[0].ic;
+    CUtensorMap mQ{}, mCK{}, mSK{};
+    if (!map_token_major(&mSK, t.K, t.kv_rows, t.kv_heads) || !map_cache(&mCK, t.cacheK[ci], t.cap[ci], t.cache_heads[ci]))
+        return cudaErrorInvalidValue;
+    if (!(which == 0 ? map_token_major(&mQ, t.Q, t.q_rows, t.q_heads) : map_token_major(&mQ, t.Qi, t.qi_rows, t.q_heads)))
+        return cudaErrorInvalidValue;
+    ColBatch<CAP> bt{};
+    bt.n = n;
+    int tiles = 0;
+    for (int i = 0; i < n; ++i) {
+        const TcSeqStep& q = seq[i];
+        TcParams& p = bt.p[i];
+        const int rows = which == 0 ? q.w : q.nI;
+        p.rows = rows; p.krow0 = q.kv_row0; p.chead = q.chead[ci];
+        p.q_heads = t.q_heads; p.kv_heads = t.kv_heads; p.m = q.m[ci]; p.L = q.L; p.status = status; p.dep_first = q.produced;
+        if (which == 0) {
+            p.row0 = q.q_row0 + (q.L - q.w); p.causal = 1; p.t0 = q.L - q.w;
+            p.lse_in = q.lse_chunk + (q.L - q.w); p.part = nullptr; p.splits = 1;
+        } else {
+            p.row0 = q.qi_row0; p.causal = 0; p.t0 = 0;
+            p.splits = q.splits < 1 ? 1 : q.splits;
+            p.lse_in = q.lse_instr; p.part = reinterpret_cast<float2*>(q.part);
+        }
+        p.lse_stride = lse_stride; p.scores = q.scores[ci]; p.score_stride = q.score_stride;
+        if (rows > 0) tiles += (p.m + kTile - 1) / kTile + (p.L + kTile - 1) / kTile;
+        bt.tile_end[i] = tiles;
+    }
+    if (tiles == 0) return cudaSuccess;
+    dim3 grid(t.kv_heads, tiles);
+    return launch_pdl(colsum_kernel<CAP>, grid, kColThreads, kColSmemBytes, s, mQ, mCK, mSK, bt);
+}
+
+cudaError_t tc_colsum(const TcTensors& t, const TcSeqStep* seq, int n, int which, int lse_stride, int* status, cudaStream_t s) {
+    if (n < 1 || n > kTcMaxBatch) return cudaErrorInvalidValue;
+    if (n == 1) return launch_colsum<1>(t, seq, n, which, lse_stride, status, s);
+    return launch_colsum<kTcMaxBatch>(t, seq, n, which, lse_stride, status, s);
 }
 
 }  // namespace citrus

@@ -449,6 +449,111 @@ def test_ragged_batch_call_matches_per_sequence_calls_and_rejects_bad_batches(la
     a.close(); b.close()
 
 
+def _lock_step_batches(w, docs, lens):
+    """The packed arguments of every lock-step call: finished sequences drop out."""
+    steps, step = [], 0
+    while True:
+        active = [s for s in range(len(lens)) if step * w.chunk_s < lens[s]]
+        if not active:
+            return steps
+        sl = [slice(step * w.chunk_s, min(lens[s], (step + 1) * w.chunk_s)) for s in active]
+        tok = [0]
+        for x in sl:
+            tok.append(tok[-1] + (x.stop - x.start))
+        steps.append((active, tok, sl))
+        step += 1
+
+
+def test_config4_serving_mix_one_grid_batch_all_sequences_in_lock_step():
+    # The ragged serving mix through the packed call: all 16 sequences advance together, one chunk each per call, and
+    # every kernel of a step is launched once over all active sequences.  After every call the caches of every
+    # sequence are property-checked (row count, ascending positions, rows bit-equal to the document's rows); on sampled
+    # steps (first, second, a middle one, and each sequence's last, ragged chunk) every active sequence is compared with
+    # the oracle, which is loaded with the library's cache first.
+    w = C["serving_mix"]
+    lens = wl.sequence_lengths(w)
+    docs = [wl.make_document(w, seq=s) for s in range(w.n_seqs)]
+    dev = [tuple(t.cuda() for t in (d.Q, d.K, d.V, d.Q_instr)) for d in docs]
+    ctx = pu.make_pair(w)
+    ctx.set_inputs_ready(True)
+    steps = _lock_step_batches(w, docs, lens)
+    last_step = {s: -(-lens[s] // w.chunk_s) - 1 for s in range(w.n_seqs)}
+    sampled = {0, 1, len(steps) // 2}
+    G = w.q_heads // w.kv_heads
+    st = {"max_out_err": 0.0, "max_score_err": 0.0, "max_score_rel": 0.0, "flips": 0, "checked_chunks": 0}
+    seen = [0] * w.n_seqs
+    for si, (active, tok, sl) in enumerate(steps):
+        Q = torch.cat([dev[s][0][x] for s, x in zip(active, sl)])
+        K = torch.cat([dev[s][1][x] for s, x in zip(active, sl)])
+        V = torch.cat([dev[s][2][x] for s, x in zip(active, sl)])
+        Qi = torch.cat([dev[s][3] for s in active])
+        ins = [w.n_instr * i for i in range(len(active) + 1)]
+        check = [s for s in active if si in sampled or si == last_step[s]]
+        oracles = {}
+        for s in check:
+            orc = pu.make_oracle(w)
+            if seen[s]:
+                pu.load_oracle_from_library(orc, ctx, 0, s, seen[s])
+            oracles[s] = orc
+        out = ctx.process_chunk_batch(0, active, tok, Q, K, V, ins, Qi)
+        torch.cuda.synchronize()
+        for i, (s, x) in enumerate(zip(active, sl)):
+            seen[s] += x.stop - x.start
+            pu.check_cache_properties(ctx, docs[s], 0, s, seen[s], dev[s][1], dev[s][2])
+            if s not in oracles:
+                continue
+            S_gpu, I_gpu, m_before = ctx.step_view(0, 0, s)
+            forced = {0: I_gpu.cpu().numpy().astype(np.int64)}
+            res = oracles[s].process_chunk(wl.to_f64(docs[s].Q[x]), wl.to_f64(docs[s].K[x]), wl.to_f64(docs[s].V[x]),
+                                           wl.to_f64(docs[s].Q_instr), forced)
+            err = float(np.abs(out[tok[i]:tok[i + 1]].double().cpu().numpy() - res.out).max())
+            assert err <= pu.TOL["bf16"], f"step {si} sequence {s}: attention output error {err}"
+            norm = w.n_instr * G
+            S = S_gpu.double().cpu().numpy()
+            serr = float(np.abs(S - res.scores[0]).max()) / norm
+            assert serr <= pu.TOL["bf16"] and m_before == res.m_before
+            assert np.allclose(S.sum(axis=1), norm, rtol=2e-3)
+            st["flips"] += pu.check_index_rule(res.idx[0], forced[0], res.scores[0], res.m_before + (x.stop - x.start), w.budget_k)
+            Kc, Vc, P = ctx.cache_view(0, 0, s)
+            assert np.array_equal(P.cpu().numpy().astype(np.int64), oracles[s].caches[0].pos)
+            assert np.array_equal(Kc.double().cpu().numpy(), oracles[s].caches[0].K)
+            st["max_out_err"] = max(st["max_out_err"], err); st["max_score_err"] = max(st["max_score_err"], serr)
+            st["checked_chunks"] += 1
+    _report("serving_mix, one grid over 16 sequences", st)
+    assert st["checked_chunks"] >= 16 + 3 and ctx.poll_status() == 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["shared", "individual", "standard"])
+def test_one_grid_batch_equals_per_sequence_calls_bit_for_bit(mode):
+    # five ragged sequences (lengths that leave partial tiles and a one-token chunk) through the packed call in one
+    # grid, against the same steps submitted sequence by sequence: outputs, scores, kept lists and caches identical
+    w = wl.scaled(C["serving_mix"], n_seqs=5, budget_k=300, chunk_s=256, n_instr=40, doc_tokens=1100, min_tokens=100,
+                  mode=mode, lm_window=32)
+    lens = [1100, 257, 640, 100, 999]
+    docs = [wl.make_document(w, seq=s, n_tokens=n) for s, n in enumerate(lens)]
+    a, b = pu.make_pair(w), pu.make_pair(w)
+    n_caches = 2 if mode == "individual" else 1
+    for active, tok, sl in _lock_step_batches(w, docs, lens):
+        Q = torch.cat([docs[s].Q[x] for s, x in zip(active, sl)]).cuda()
+        K = torch.cat([docs[s].K[x] for s, x in zip(active, sl)]).cuda()
+        V = torch.cat([docs[s].V[x] for s, x in zip(active, sl)]).cuda()
+        Qi = torch.cat([docs[s].Q_instr for s in active]).cuda()
+        ins = [w.n_instr * i for i in range(len(active) + 1)]
+        out = a.process_chunk_batch(0, active, tok, Q, K, V, ins, Qi)
+        for i, (s, x) in enumerate(zip(active, sl)):
+            ref = b.process_chunk(0, docs[s].Q[x].cuda(), docs[s].K[x].cuda(), docs[s].V[x].cuda(), docs[s].Q_instr.cuda(), slot=s)
+            torch.cuda.synchronize()
+            assert torch.equal(out[tok[i]:tok[i + 1]], ref)
+            for cid in range(n_caches):
+                for t1, t2 in zip(a.cache_view(0, cid, s), b.cache_view(0, cid, s)):
+                    assert torch.equal(t1, t2)
+                va, vb = a.step_view(0, cid, s), b.step_view(0, cid, s)
+                assert torch.equal(va[0], vb[0]) and torch.equal(va[1], vb[1]) and va[2] == vb[2]
+    assert a.poll_status() == 0
+    a.close(); b.close()
+
+
 @pytest.mark.parametrize("mode,shift", [("shared", False), ("individual", False), ("shared", True), ("individual", True)])
 def test_batch_lanes_in_a_captured_graph_equal_the_single_stream_run(mode, shift):
     # six ragged sequences through the packed call: once on the caller's stream alone, once dealt to four side
