@@ -453,10 +453,13 @@ int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn*
     const int n_jobs = (int)sj.size();
     // Small steps (a few MB to move) are latency-bound: one cluster launch does a3 and a4.  Large steps want every
     // SM streaming rows, which the clusters (idle while their first CTA selects) cannot give: two launches.
-    if (!c->layerwise && !c->shift && gather_bytes <= ((size_t)8 << 20)) {
-        // one cluster launch does both (timed under the compaction id)
+    int n_most = 0;
+    for (const SelectJob& j : sj) n_most = j.n > n_most ? j.n : n_most;
+    if (!c->layerwise && !c->shift && !c->accumulate && gather_bytes <= ((size_t)8 << 20) * (size_t)n &&
+        select_compact_fits(n_most, c->D * c->elt)) {
+        // one launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-        e = select_compact(sj.data(), cj.data(), n_jobs, c->Hkv, c->D * c->elt, nullptr, c->elt, st);
+        e = select_compact(sj.data(), cj.data(), n_jobs, c->Hkv, c->D * c->elt, c->elt, produced ? 0 : 1, st);
         if (e != cudaSuccess) return cuda_rc(e);
     } else {
         {

@@ -62,40 +62,19 @@ __device__ __forceinline__ uint32_t order_key(float f) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// One CTA per (cache, KV head) -- or per cache when layerwise.  The score vector is
-// staged once in shared memory as order keys; a 4-pass most-significant-digit radix
-// select finds the k-th largest key T and how many candidates equal to T are kept;
-// a flagged block scan in index order then emits kept indices ascending, taking the
-// lowest-index candidates among those equal to T.
-// `also(p, j)` is called for every kept candidate j with its place p in the ascending list (the fused kernel
-// uses it to hand the list to the gathering CTAs through shared memory).
-template <typename Also>
-__device__ __forceinline__ void select_body(const SelectJob& job, const int g, int kv_heads, int layerwise,
-                                            uint32_t* keys /* shared, [n] */, Also also) {
-    const int n = job.n, k = job.k, ks = job.idx_stride;
+// The score vector of one (cache, KV head) - or of the whole layer when layerwise - is staged once in shared memory as
+// order keys; a most-significant-digit radix select (8-bit digits; as soon as at most 32 candidates share the prefix
+// one warp ranks them directly) finds the k-th largest key T and how many candidates equal to T are kept (the
+// lowest-index ones).  Called by all kSelThreads threads of a CTA with n > k.
+__device__ __forceinline__ void select_threshold(const SelectJob& job, const int g, int kv_heads, int layerwise,
+                                                 uint32_t* keys /* shared, [n] */, uint32_t& T_out, uint32_t& take_eq_out) {
+    const int n = job.n, k = job.k;
     __shared__ uint32_t hist[256];
     __shared__ uint32_t s_prefix, s_remaining, s_bin_count, s_n_short;
     __shared__ uint32_t s_short[32];
-    __shared__ uint32_t warp_gt[32], warp_eq[32];
-
+    __shared__ uint32_t s_wmin[32], s_wmax[32];
     const int tid = threadIdx.x;
-    const int heads_out = layerwise ? kv_heads : 1;
-    int* idx0 = job.idx + (size_t)g * ks;
-
-    if (n <= k) {                                  // nothing to evict: identity
-        for (int j = tid; j < n; j += kSelThreads) {
-            for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * ks + j] = j;
-            also(j, j);
-            if (job.carried != nullptr && j < job.m) {
-                // accumulative policy: the carried importance still has to be added to what is handed on
-                for (int ho = 0; ho < heads_out; ++ho) {
-                    const int gg = layerwise ? ho : g;
-                    job.scores[(size_t)gg * job.score_stride + j] += job.carried[(size_t)gg * job.pos_stride + j];
-                }
-            }
-        }
-        return;
-    }
+    uint32_t kmin = 0xffffffffu, kmax = 0u;        // over this thread's keys; the forced ones (all-ones) stay out of the maximum
     for (int j = tid; j < n; j += kSelThreads) {
         // one head's score of candidate j; with the accumulative policy the importance its cache row carries is
         // added and the sum written back (it is what the compaction hands on, and what the step view shows)
@@ -123,13 +102,32 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         }
         if (j >= job.forced_from) key = 0xffffffffu;          // the chunk's own states all enter (deferred eviction)
         keys[j] = key;
+        kmin = min(kmin, key);
+        if (key != 0xffffffffu) kmax = max(kmax, key);
     }
+    // The scores of one head share their sign and most of their exponent bits, so the leading digits of the raw keys
+    // tell nothing.  The keys are rebased to d = key - min (a forced key: range + 1) and shifted up so that the range
+    // fills whole 8-bit digits: the order is unchanged, the first digit already spreads the candidates over up to 256
+    // bins, and the digits below the range's width need no pass at all.
+    kmin = __reduce_min_sync(0xffffffffu, kmin); kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if ((tid & 31) == 0) { s_wmin[tid >> 5] = kmin; s_wmax[tid >> 5] = kmax; }
     if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; s_bin_count = (uint32_t)n; s_n_short = 0u; }
+    __syncthreads();
+    kmin = __reduce_min_sync(0xffffffffu, s_wmin[tid & 31]); kmax = __reduce_max_sync(0xffffffffu, s_wmax[tid & 31]);
+    const uint32_t range = kmax > kmin ? kmax - kmin : 0u;            // of the keys that are not forced
+    const uint32_t top = range == 0xffffffffu ? range : range + 1u;   // value given to the forced keys
+    const int nbits = 32 - __clz(top | 1u);
+    const int width = (nbits + 7) & ~7;                               // digits cover `width` bits
+    const int up = width - nbits;
+    for (int j = tid; j < n; j += kSelThreads) {
+        const uint32_t key = keys[j];
+        keys[j] = (key == 0xffffffffu ? top : key - kmin) << up;
+    }
     __syncthreads();
     CITRUS_TR(10);
 
     uint32_t mask = 0u;
-    for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int shift = width - 8; shift >= 0; shift -= 8) {
         if (tid < 256) hist[tid] = 0u;
         __syncthreads();
         const uint32_t prefix = s_prefix;
@@ -176,7 +174,7 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         }
         mask |= 255u << shift;
         __syncthreads();
-        CITRUS_TR(11 + (24 - shift) / 8);
+        CITRUS_TR(11 + (width - 8 - shift) / 8);
         // Short cut: at most 32 candidates still share the prefix.  One warp ranks them directly instead of
         // walking the remaining digits.
         if (shift > 0 && s_bin_count <= 32u) {
@@ -203,8 +201,36 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
             break;
         }
     }
-    const uint32_t T = s_prefix;                   // k-th largest key
-    const uint32_t take_eq = s_remaining;          // candidates equal to T that are kept (lowest indices)
+    T_out = s_prefix;                              // k-th largest key (in the rebased form that `keys` now holds)
+    take_eq_out = s_remaining;                     // candidates equal to T that are kept (lowest indices)
+}
+
+// One CTA per (cache, KV head) -- or per cache when layerwise: threshold, then a flagged block scan in index order
+// emits the kept indices ascending, taking the lowest-index candidates among those equal to T.
+__device__ __forceinline__ void select_body(const SelectJob& job, const int g, int kv_heads, int layerwise,
+                                            uint32_t* keys /* shared, [n] */) {
+    const int n = job.n, k = job.k, ks = job.idx_stride;
+    __shared__ uint32_t warp_gt[32], warp_eq[32];
+
+    const int tid = threadIdx.x;
+    const int heads_out = layerwise ? kv_heads : 1;
+    int* idx0 = job.idx + (size_t)g * ks;
+
+    if (n <= k) {                                  // nothing to evict: identity
+        for (int j = tid; j < n; j += kSelThreads) {
+            for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * ks + j] = j;
+            if (job.carried != nullptr && j < job.m) {
+                // accumulative policy: the carried importance still has to be added to what is handed on
+                for (int ho = 0; ho < heads_out; ++ho) {
+                    const int gg = layerwise ? ho : g;
+                    job.scores[(size_t)gg * job.score_stride + j] += job.carried[(size_t)gg * job.pos_stride + j];
+                }
+            }
+        }
+        return;
+    }
+    uint32_t T, take_eq;
+    select_threshold(job, g, kv_heads, layerwise, keys, T, take_eq);
 
     // ordered emission: thread t owns the contiguous index range [t*per, (t+1)*per)
     const int per = (n + kSelThreads - 1) / kSelThreads;
@@ -239,7 +265,6 @@ __device__ __forceinline__ void select_body(const SelectJob& job, const int g, i
         if (keep) {
             uint32_t p = gt_before + min(eq_before, take_eq);
             for (int ho = 0; ho < heads_out; ++ho) idx0[(size_t)ho * ks + p] = j;
-            also((int)p, j);
         }
         gt_before += key > T;
         eq_before += key == T;
@@ -253,7 +278,7 @@ select_topk_kernel(const __grid_constant__ SelectArgs<CAP> args, int kv_heads, i
     extern __shared__ uint32_t keys[];            // [largest n of the jobs]
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the scores are final after this
-    select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, layerwise, keys, [](int, int) {});
+    select_body(args.job[blockIdx.y], blockIdx.x, kv_heads, layerwise, keys);
 }
 
 // Rows [r_begin, r_end) of one (cache, head) are copied with 128-bit accesses, row_bytes/16 lanes per row.
@@ -353,49 +378,162 @@ compact_kv_kernel(const __grid_constant__ CompactArgs<CAP> args, int kv_heads, i
                           r0, min(job.kept, r0 + kCompactRowsPerCta), job.idx + (size_t)blockIdx.y * job.cap, args.rope, args.elt);
 }
 
-// a3 + a4 in one launch: a cluster of kFusedCluster CTAs per (cache, KV head).  The first CTA of the cluster
-// selects and writes each kept index twice: to the global list (part of the result) and into the shared memory
-// of the CTA that will gather that row; the cluster barrier publishes the slices, then every CTA gathers its
-// share of the kept rows without another trip to global memory for the indices.
-// grid: (kFusedCluster, KV heads, caches), cluster (kFusedCluster, 1, 1)
-constexpr int kFusedCluster = 8;
+// a3 + a4 in one launch, for steps that are small enough to be latency-bound: kFusedParts CTAs per (cache, KV head),
+// each responsible for a contiguous share of the CANDIDATES.  A CTA
+//   1. starts bulk copies of its share's K and V rows into shared memory (the chunk's rows at once when the caller's
+//      inputs are declared complete, the old cache's rows after griddepcontrol.wait), so that the whole load latency
+//      hides behind the selection;
+//   2. runs the selection on the full score vector (every CTA of the head repeats this small computation instead of
+//      waiting for one that does it: no cluster, no hand-over of index lists);
+//   3. counts the kept candidates that precede its share, scans its own share (one candidate per thread) and writes
+//      its kept rows - consecutive kept candidates are consecutive rows of the new cache - from shared memory.
+// grid: (kFusedParts, KV heads, jobs)
+constexpr int kFusedParts = 8;
+constexpr int kFusedMaxShare = kSelThreads;      // one candidate per thread in the local scan
+
+__device__ __forceinline__ uint32_t sc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 
 template <int CAP>
 __global__ void __launch_bounds__(kSelThreads)
-select_compact_kernel(const __grid_constant__ SelectArgs<CAP> sel, const __grid_constant__ CompactArgs<CAP> cmp,
-                      int kv_heads, int n_max, int row_vecs) {
-    extern __shared__ uint32_t keys[];            // [n_max] order keys (selecting CTA only), then this CTA's slice of the list
-    const int g = blockIdx.y;
-    const int kept = cmp.job[blockIdx.z].kept;
-    const int per = (kept + kFusedCluster - 1) / kFusedCluster;
-    int* s_idx = reinterpret_cast<int*>(keys + n_max);     // [per]
-    // programmatic dependent launch: let the next kernel start its prologue, then wait for the scores
+select_gather_kernel(const __grid_constant__ SelectArgs<CAP> sel, const __grid_constant__ CompactArgs<CAP> cmp,
+                     int kv_heads, int n_max, int share_max, int row_bytes, int early_chunk_rows) {
+    extern __shared__ __align__(128) uint8_t sg_smem[];
+    __shared__ uint64_t rows_bar;
+    __shared__ uint32_t w_gt[32], w_eq[32], w_keep[32];
+    __shared__ int s_lkept[kFusedMaxShare];          // local candidate index of the CTA's r-th kept candidate
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    CITRUS_SPAN_MIN(0);
-    // every CTA of the cluster is running (its shared memory may be written) once this first barrier completes
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    CITRUS_SPAN_MIN(1);
-    CITRUS_TR(9);
-    if (blockIdx.x == 0) {
-        const uint32_t slice = (uint32_t)__cvta_generic_to_shared(s_idx);
-        select_body(sel.job[blockIdx.z], g, kv_heads, 0, keys, [&](int p, int j) {
-            uint32_t remote;
-            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(slice + 4u * (uint32_t)(p % per)), "r"(p / per));
-            asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(j) : "memory");
-        });
+    const SelectJob& sjob = sel.job[blockIdx.z];
+    const CompactJob& job = cmp.job[blockIdx.z];
+    const int g = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = sjob.n, k = sjob.k, m = job.m, cap = job.cap;
+    const int share = (n + kFusedParts - 1) / kFusedParts;
+    const int c0 = min(n, (int)blockIdx.x * share), c1 = min(n, c0 + share);
+    const int cnt = c1 - c0;
+    uint32_t* keys = reinterpret_cast<uint32_t*>(sg_smem);                       // [n_max]
+    uint8_t* rowK = sg_smem + (((size_t)n_max * 4 + 127) & ~(size_t)127);        // [share_max][row_bytes]
+    uint8_t* rowV = rowK + (size_t)share_max * row_bytes;
+    const uint32_t bar = sc_smem_u32(&rows_bar);
+    // this CTA's candidates: [c0, cm) are rows of the old cache, [cm, c1) rows of the chunk
+    const int cm = min(c1, max(c0, m));
+    const uint8_t* srcK = reinterpret_cast<const uint8_t*>(job.srcK);
+    const uint8_t* srcV = reinterpret_cast<const uint8_t*>(job.srcV);
+    const uint8_t* chunkK = reinterpret_cast<const uint8_t*>(job.chunkK);
+    const uint8_t* chunkV = reinterpret_cast<const uint8_t*>(job.chunkV);
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(2 * cnt * row_bytes)) : "memory");
     }
-    // hardware cluster barrier with release/acquire semantics: the slices written above are visible to their owners
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    CITRUS_SPAN_MAX(3);
-    CITRUS_TR(16);
-    const int r0 = blockIdx.x * per;
-    // (the position shift always takes the two-kernel route: its rotation does not fit this kernel's 64 registers)
-    compact_rows_t<false>(cmp.job[blockIdx.z], g, kv_heads, row_vecs, r0, min(kept, r0 + per), s_idx - r0, cmp.rope, cmp.elt);
-    CITRUS_SPAN_MAX(2);
-    CITRUS_TR(17);
+    __syncthreads();
+    auto copy_chunk_rows = [&]() {
+        // one copy per row and tensor: chunk rows are kv_heads * row_bytes apart
+        for (int j = cm + tid; j < c1; j += kSelThreads) {
+            const size_t src = ((size_t)(j - m) * kv_heads + g) * row_bytes;
+            bulk_g2s(sc_smem_u32(rowK + (size_t)(j - c0) * row_bytes), chunkK + src, (uint32_t)row_bytes, bar);
+            bulk_g2s(sc_smem_u32(rowV + (size_t)(j - c0) * row_bytes), chunkV + src, (uint32_t)row_bytes, bar);
+        }
+    };
+    CITRUS_TR(1);
+    if (early_chunk_rows) copy_chunk_rows();
+    CITRUS_TR(2);
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // scores, the old cache and its positions are final after this
+    CITRUS_TR(3);
+    if (!early_chunk_rows) copy_chunk_rows();
+    if (tid == 0 && cm > c0) {
+        // the old cache's rows of the share are contiguous: one copy per tensor (pieces of at most 64 KB)
+        const size_t src = ((size_t)g * cap + c0) * row_bytes;
+        const uint32_t total = (uint32_t)(cm - c0) * (uint32_t)row_bytes;
+        for (uint32_t off = 0; off < total; off += 65536u) {
+            const uint32_t piece = min(65536u, total - off);
+            bulk_g2s(sc_smem_u32(rowK + off), srcK + src + off, piece, bar);
+            bulk_g2s(sc_smem_u32(rowV + off), srcV + src + off, piece, bar);
+        }
+    }
+    // original position of this thread's candidate (thread t <-> candidate c0 + t), fetched before the selection
+    const int j_mine = c0 + tid;
+    int pos_mine = 0;
+    if (tid < cnt) pos_mine = j_mine < m ? __ldg(job.srcPos + (size_t)g * cap + j_mine) : job.chunk_pos0 + (j_mine - m);
+
+    // ---- selection on the whole score vector
+    bool keep = false;
+    uint32_t p_mine = 0;                                      // place of this thread's candidate in the ascending list
+    int p_base = 0, kept_here = 0;
+    if (n <= k) {                                             // nothing to evict
+        keep = tid < cnt; p_mine = (uint32_t)j_mine; p_base = c0; kept_here = cnt;
+        if (keep) s_lkept[tid] = tid;
+        __syncthreads();
+    } else {
+        uint32_t T, take_eq;
+        CITRUS_TR(4);
+        select_threshold(sjob, g, kv_heads, 0, keys, T, take_eq);
+        CITRUS_TR(5);
+        // kept candidates and candidates equal to T before the share (all threads count a slice of keys[0, c0))
+        uint32_t gt = 0u, eq = 0u;
+        for (int j = tid; j < c0; j += kSelThreads) { const uint32_t key = keys[j]; gt += key > T; eq += key == T; }
+        const uint32_t key_mine = tid < cnt ? keys[j_mine] : 0u;
+        const bool is_gt = tid < cnt && key_mine > T, is_eq = tid < cnt && key_mine == T;
+        gt = __reduce_add_sync(0xffffffffu, gt); eq = __reduce_add_sync(0xffffffffu, eq);
+        // the share itself, one candidate per thread: ballots give the in-warp ranks
+        const uint32_t b_gt = __ballot_sync(0xffffffffu, is_gt), b_eq = __ballot_sync(0xffffffffu, is_eq);
+        if (lane == 0) { w_gt[warp] = gt | ((uint32_t)__popc(b_gt) << 16); w_eq[warp] = eq | ((uint32_t)__popc(b_eq) << 16); }
+        __syncthreads();
+        // every warp adds up: totals before the share (low halves), and the share's counts of the warps before it
+        uint32_t v_gt = w_gt[lane], v_eq = w_eq[lane];
+        const uint32_t gt_before = __reduce_add_sync(0xffffffffu, v_gt & 0xffffu);
+        const uint32_t eq_before = __reduce_add_sync(0xffffffffu, v_eq & 0xffffu);
+        const uint32_t gt_warps = __reduce_add_sync(0xffffffffu, lane < warp ? (v_gt >> 16) : 0u);
+        const uint32_t eq_warps = __reduce_add_sync(0xffffffffu, lane < warp ? (v_eq >> 16) : 0u);
+        const uint32_t lt_mask = (1u << lane) - 1u;
+        const uint32_t gt_rank = gt_warps + (uint32_t)__popc(b_gt & lt_mask);       // kept-by-value candidates of the share before mine
+        const uint32_t eq_rank = eq_before + eq_warps + (uint32_t)__popc(b_eq & lt_mask);   // equal-to-T candidates before mine, whole vector
+        keep = is_gt || (is_eq && eq_rank < take_eq);
+        // ties kept before the share, and inside the share before mine
+        const uint32_t eq_kept_before = min(eq_before, take_eq);
+        const uint32_t eq_kept_rank = min(eq_rank, take_eq) - eq_kept_before;
+        p_base = (int)(gt_before + eq_kept_before);
+        p_mine = (uint32_t)p_base + gt_rank + eq_kept_rank;
+        const uint32_t b_keep = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) w_keep[warp] = (uint32_t)__popc(b_keep);
+        if (keep) s_lkept[p_mine - (uint32_t)p_base] = tid;
+        __syncthreads();
+        kept_here = (int)__reduce_add_sync(0xffffffffu, w_keep[lane]);
+    }
+    CITRUS_TR(6);
+    // ---- index list and positions of the kept candidates of the share
+    if (keep) {
+        sjob.idx[(size_t)g * sjob.idx_stride + p_mine] = j_mine;
+        job.dstPos[(size_t)g * cap + p_mine] = pos_mine;
+    }
+    // ---- rows: wait for the copies, then shared memory -> new cache, row_vecs lanes per row
+    {
+        bool landed = false;
+        for (int spin = 0; spin < (1 << 22) && !landed; ++spin) {       // bounded: the copies of a few KB take microseconds
+            uint32_t ok;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(bar) : "memory");
+            landed = ok != 0;
+        }
+        if (!landed) return;                                            // (never seen; the rows are then left unwritten)
+    }
+    CITRUS_TR(7);
+    const int row_vecs = row_bytes / 16;
+    const int rows_per_pass = kSelThreads / row_vecs;
+    const int sub = tid / row_vecs, v = tid % row_vecs;
+    uint4* dstK = reinterpret_cast<uint4*>(job.dstK);
+    uint4* dstV = reinterpret_cast<uint4*>(job.dstV);
+    for (int r = sub; r < kept_here; r += rows_per_pass) {
+        const int l = s_lkept[r];
+        const uint4 a = *reinterpret_cast<const uint4*>(rowK + (size_t)l * row_bytes + (size_t)v * 16);
+        const uint4 bb = *reinterpret_cast<const uint4*>(rowV + (size_t)l * row_bytes + (size_t)v * 16);
+        const size_t doff = ((size_t)g * cap + p_base + r) * row_vecs + v;
+        dstK[doff] = a;
+        dstV[doff] = bb;
+    }
+    CITRUS_TR(8);
 }
 
 // One CTA per KV head: thread t looks element t, t + 256, ... of list b up in list a (both strictly ascending) by
@@ -466,8 +604,8 @@ cudaError_t raise_smem_limits() {
     if (!g_attr_ready.needs_setup(dev)) return cudaSuccess;
     e = cudaFuncSetAttribute(select_topk_kernel<kJobsSingle>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(select_topk_kernel<kJobsBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_compact_kernel<kJobsSingle>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_compact_kernel<kJobsBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_gather_kernel<kJobsSingle>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(select_gather_kernel<kJobsBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     g_attr_ready.mark(dev);
     return cudaSuccess;
@@ -531,39 +669,46 @@ cudaError_t select_topk(const SelectJob* jobs, int n_jobs, int kv_heads, int lay
     return launch_select_topk<kJobsBatch>(jobs, n_jobs, kv_heads, layerwise, s);
 }
 
+// Shared memory of the fused kernel for a step with at most n candidates per job.
+static size_t fused_smem_bytes(int n, int row_bytes) {
+    const int share = (n + kFusedParts - 1) / kFusedParts;
+    return (((size_t)n * 4 + 127) & ~(size_t)127) + (size_t)2 * share * row_bytes;
+}
+bool select_compact_fits(int n, int row_bytes) {
+    return (n + kFusedParts - 1) / kFusedParts <= kFusedMaxShare && fused_smem_bytes(n, row_bytes) <= 200 * 1024;
+}
+
 template <int CAP>
 static cudaError_t launch_select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, int kv_heads, int row_bytes,
-                                         int elt, cudaStream_t s) {
+                                         int elt, int early_chunk_rows, cudaStream_t s) {
     SelectArgs<CAP> sa; CompactArgs<CAP> ca;
     ca.elt = elt;
-    int n = 0, kept = 0;
+    int n = 0;
     for (int i = 0; i < n_jobs; ++i) {
         sa.job[i] = sjobs[i]; ca.job[i] = cjobs[i];
         n = sjobs[i].n > n ? sjobs[i].n : n;
-        kept = cjobs[i].kept > kept ? cjobs[i].kept : kept;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kFusedCluster, kv_heads, n_jobs);
+    cfg.gridDim = dim3(kFusedParts, kv_heads, n_jobs);
     cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = ((size_t)n + (size_t)((kept + kFusedCluster - 1) / kFusedCluster)) * sizeof(uint32_t);
+    cfg.dynamicSmemBytes = fused_smem_bytes(n, row_bytes);
     cfg.stream = s;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kFusedCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 2;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
     before_launch(s);
-    return cudaLaunchKernelEx(&cfg, select_compact_kernel<CAP>, sa, ca, kv_heads, n, row_bytes / 16);
+    return cudaLaunchKernelEx(&cfg, select_gather_kernel<CAP>, sa, ca, kv_heads, n, (n + kFusedParts - 1) / kFusedParts, row_bytes,
+                              early_chunk_rows);
 }
 
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, int kv_heads, int row_bytes,
-                           const RopeTable* rope, int elt, cudaStream_t s) {
-    if (n_jobs < 1 || n_jobs > kJobsBatch || rope != nullptr) return cudaErrorInvalidValue;
+                           int elt, int early_chunk_rows, cudaStream_t s) {
+    if (n_jobs < 1 || n_jobs > kJobsBatch) return cudaErrorInvalidValue;
     cudaError_t e = raise_smem_limits();
     if (e != cudaSuccess) return e;
-    if (n_jobs <= kJobsSingle) return launch_select_compact<kJobsSingle>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, s);
-    return launch_select_compact<kJobsBatch>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, s);
+    if (n_jobs <= kJobsSingle) return launch_select_compact<kJobsSingle>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, early_chunk_rows, s);
+    return launch_select_compact<kJobsBatch>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, early_chunk_rows, s);
 }
 
 template <int CAP>
