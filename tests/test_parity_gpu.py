@@ -554,6 +554,38 @@ def test_one_grid_batch_equals_per_sequence_calls_bit_for_bit(mode):
     a.close(); b.close()
 
 
+def test_one_grid_batch_of_more_sequences_than_one_launch_holds():
+    # 40 short sequences in one call: the library cuts the batch into groups of 32 sequences per launch; tiny chunks
+    # (1 to 70 tokens: far less than a tile, so every tile of the packed tensors mixes several sequences' rows)
+    w = wl.scaled(C["serving_mix"], n_seqs=40, budget_k=48, chunk_s=70, n_instr=8, doc_tokens=140, min_tokens=1,
+                  q_heads=8, kv_heads=2)
+    lens = [1 + (37 * s) % 140 for s in range(40)]
+    docs = [wl.make_document(w, seq=s, n_tokens=n) for s, n in enumerate(lens)]
+    a, b = pu.make_pair(w), pu.make_pair(w)
+    for active, tok, sl in _lock_step_batches(w, docs, lens):
+        Q = torch.cat([docs[s].Q[x] for s, x in zip(active, sl)]).cuda()
+        K = torch.cat([docs[s].K[x] for s, x in zip(active, sl)]).cuda()
+        V = torch.cat([docs[s].V[x] for s, x in zip(active, sl)]).cuda()
+        Qi = torch.cat([docs[s].Q_instr for s in active]).cuda()
+        ins = [w.n_instr * i for i in range(len(active) + 1)]
+        out = a.process_chunk_batch(0, active, tok, Q, K, V, ins, Qi)
+        for i, (s, x) in enumerate(zip(active, sl)):
+            ref = b.process_chunk(0, docs[s].Q[x].cuda(), docs[s].K[x].cuda(), docs[s].V[x].cuda(), docs[s].Q_instr.cuda(), slot=s)
+            torch.cuda.synchronize()
+            assert torch.equal(out[tok[i]:tok[i + 1]], ref)
+            for t1, t2 in zip(a.cache_view(0, 0, s), b.cache_view(0, 0, s)):
+                assert torch.equal(t1, t2)
+    # and against the oracle: the longest sequence's last state
+    s = max(range(40), key=lambda i: lens[i])
+    orc = pu.make_oracle(w)
+    for c in range(0, lens[s], w.chunk_s):
+        x = slice(c, min(lens[s], c + w.chunk_s))
+        orc.process_chunk(wl.to_f64(docs[s].Q[x]), wl.to_f64(docs[s].K[x]), wl.to_f64(docs[s].V[x]), wl.to_f64(docs[s].Q_instr))
+    assert np.array_equal(a.cache_view(0, 0, s)[2].cpu().numpy().astype(np.int64), orc.caches[0].pos)
+    assert a.poll_status() == 0
+    a.close(); b.close()
+
+
 @pytest.mark.parametrize("mode,shift", [("shared", False), ("individual", False), ("shared", True), ("individual", True)])
 def test_batch_lanes_in_a_captured_graph_equal_the_single_stream_run(mode, shift):
     # six ragged sequences through the packed call: once on the caller's stream alone, once dealt to four side
