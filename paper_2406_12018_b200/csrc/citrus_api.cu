@@ -381,16 +381,12 @@ int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn*
             e = tc_attention_lse(t, seq.data(), n, c->ls, CITRUS_MAX_INSTR, c->status, st);
         }
         if (e != cudaSuccess) return cuda_rc(e);
-        // a2-L (individual design, standard chunked eviction): votes of the chunk's last w queries on cache 0's candidates
-        if (any_lm) {
+        // a2-L (individual design, standard chunked eviction: votes of the chunk's last w queries on cache 0's
+        // candidates) and pass 2 of a2-I (Eq. 1 column sums of the instruction queries over the instruction-side cache's
+        // candidates) in one launch: the two are independent, and the short instruction sweeps fill the tail of the LM ones
+        if (any_lm || any_instr) {
             LaunchTimer tm(c, CITRUS_KERNEL_COLSUM, st);
-            e = tc_colsum(t, seq.data(), n, 0, c->ls, c->status, st);
-            if (e != cudaSuccess) return cuda_rc(e);
-        }
-        // a2-I pass 2: Eq. 1 column sums of the instruction queries over the instruction-side cache's candidates
-        if (any_instr) {
-            LaunchTimer tm(c, CITRUS_KERNEL_COLSUM, st);
-            e = tc_colsum(t, seq.data(), n, 1, CITRUS_MAX_INSTR, c->status, st);
+            e = tc_colsum(t, seq.data(), n, any_lm, any_instr, c->ls, CITRUS_MAX_INSTR, c->status, st);
             if (e != cudaSuccess) return cuda_rc(e);
         }
     } else {

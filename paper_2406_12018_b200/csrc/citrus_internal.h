@@ -105,9 +105,10 @@ struct TcSeqStep {
 // One launch: a1 (chunk over [cache 0 ; chunk] -> out, optional row log-sum-exp) and pass 1 of a2-I of every sequence.
 cudaError_t tc_attention_lse(const TcTensors& t, const TcSeqStep* seq, int n, int lse_chunk_stride, int lse_instr_stride,
                              int* status, cudaStream_t s);
-// Pass 2, one launch for all sequences.  which = 0: the chunk's last w rows score cache 0's candidates with a1's
-// probabilities; which = 1: the instruction rows score cache ic's candidates.
-cudaError_t tc_colsum(const TcTensors& t, const TcSeqStep* seq, int n, int which, int lse_stride, int* status, cudaStream_t s);
+// The column sums, one launch for both scorings and all sequences.  do_lm: the chunk's last w rows score cache 0's
+// candidates with a1's probabilities; do_instr: the instruction rows score cache ic's candidates.
+cudaError_t tc_colsum(const TcTensors& t, const TcSeqStep* seq, int n, bool do_lm, bool do_instr, int lse_chunk_stride,
+                      int lse_instr_stride, int* status, cudaStream_t s);
 
 // ---- select (a3) and compaction (a4) ---------------------------------------
 struct SelectJob {            // one per cache handled by the launch

@@ -87,7 +87,7 @@ extern "C" int citrus_importance_static(const void* Q_s, int n_s, const void* K,
         q.scores[0] = scores; q.scores[1] = scores; q.score_stride = score_stride;
         q.produced = 1;                            // wait for earlier stream work before the first load of Q_s or K
         e = tc_attention_lse(t, &q, 1, 0, lse_stride, status, st);
-        if (e == cudaSuccess) e = tc_colsum(t, &q, 1, 1, lse_stride, status, st);
+        if (e == cudaSuccess) e = tc_colsum(t, &q, 1, false, true, 0, lse_stride, status, st);
     }
     if (e != cudaSuccess) { cudaGetLastError(); return CITRUS_ERR_CUDA; }
     return CITRUS_OK;

@@ -758,25 +758,29 @@ constexpr int kColSmemBytes = 1024 + kTileBytes * (1 + kColStages) + 8192;
 // shorter and shorter under the causal mask; the short ones fill the tail of the last wave.
 // Accumulator rows = 128 candidates, columns = scoring rows of one
 // (head, row block); thread i owns candidate i and adds exp2(logit2 - lse2[row]) over its columns.
-// A batch: blockIdx.y runs over the candidate tiles of sequence 0, 1, ... (tile_end = exclusive prefix ends).
+// One launch serves both scoring passes of a step and every sequence of a batch: blockIdx.y runs over the candidate
+// tiles of entry 0, 1, ... (tile_end = exclusive prefix ends).  Entries [0, n_first) are LM scorings (the chunk's last
+// w rows over cache 0's candidates: query map Q0, cache map CK0), the others instruction scorings (instruction rows
+// over the instruction-side cache's candidates: Q1, CK1).  The LM entries come first: their sweeps are the long ones.
 template <int CAP>
 struct ColBatch {
-    int n;
-    int tile_end[CAP];
-    TcParams p[CAP];
+    int n_entries, n_first;
+    int tile_end[2 * CAP];
+    TcParams p[2 * CAP];
 };
 template <int CAP>
 __global__ void __launch_bounds__(kColThreads, 1)
-colsum_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapCK,
+colsum_kernel(const __grid_constant__ CUtensorMap mapQ0, const __grid_constant__ CUtensorMap mapCK0,
+              const __grid_constant__ CUtensorMap mapQ1, const __grid_constant__ CUtensorMap mapCK1,
               const __grid_constant__ CUtensorMap mapSK, const __grid_constant__ ColBatch<CAP> bt) {
     extern __shared__ uint8_t smem_raw[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    int seq = 0, kt = blockIdx.y;
-    if (CAP > 1) {
-        while (seq + 1 < bt.n && kt >= bt.tile_end[seq]) ++seq;
-        if (seq > 0) kt -= bt.tile_end[seq - 1];
-    }
-    const TcParams& p = bt.p[seq];
+    int entry = 0, kt = blockIdx.y;
+    while (entry + 1 < bt.n_entries && kt >= bt.tile_end[entry]) ++entry;
+    if (entry > 0) kt -= bt.tile_end[entry - 1];
+    const TcParams& p = bt.p[entry];
+    const CUtensorMap& mapQ = entry < bt.n_first ? mapQ0 : mapQ1;
+    const CUtensorMap& mapCK = entry < bt.n_first ? mapCK0 : mapCK1;
 #ifdef CITRUS_TRACE
     if (threadIdx.x == 0) atomicMax(&g_citrus_trace[245], ~global_ns());
 #endif
@@ -1191,46 +1195,58 @@ cudaError_t tc_attention_lse(const TcTensors& t, const TcSeqStep* seq, int n, in
     return launch_attention<kTcMaxBatch>(t, seq, n, lse_chunk_stride, lse_instr_stride, status, s);
 }
 
-// which = 0: the chunk's last w rows score the LM-side cache's candidates with a1's probabilities (causal);
-// which = 1: the instruction rows score the instruction-side cache's candidates.
+// The column sums of a step in one launch: with do_lm the chunk's last w rows score cache 0's candidates with a1's
+// probabilities (causal); with do_instr the instruction rows score the instruction-side cache's candidates.
 template <int CAP>
-static cudaError_t launch_colsum(const TcTensors& t, const TcSeqStep* seq, int n, int which, int lse_stride, int* status, cudaStream_t s) {
-    const int ci = which == 0 ? 0 : seq[0].ic;
-    CUtensorMap mQ{}, mCK{}, mSK{};
-    if (!map_token_major(&mSK, t.K, t.kv_rows, t.kv_heads) || !map_cache(&mCK, t.cacheK[ci], t.cap[ci], t.cache_heads[ci]))
+static cudaError_t launch_colsum(const TcTensors& t, const TcSeqStep* seq, int n, bool do_lm, bool do_instr,
+                                 int lse_chunk_stride, int lse_instr_stride, int* status, cudaStream_t s) {
+    const int ic = seq[0].ic;
+    CUtensorMap mQ0{}, mCK0{}, mQ1{}, mCK1{}, mSK{};
+    if (!map_token_major(&mSK, t.K, t.kv_rows, t.kv_heads)) return cudaErrorInvalidValue;
+    if (do_lm && (!map_token_major(&mQ0, t.Q, t.q_rows, t.q_heads) || !map_cache(&mCK0, t.cacheK[0], t.cap[0], t.cache_heads[0])))
         return cudaErrorInvalidValue;
-    if (!(which == 0 ? map_token_major(&mQ, t.Q, t.q_rows, t.q_heads) : map_token_major(&mQ, t.Qi, t.qi_rows, t.q_heads)))
+    if (do_instr && (!map_token_major(&mQ1, t.Qi, t.qi_rows, t.q_heads) || !map_cache(&mCK1, t.cacheK[ic], t.cap[ic], t.cache_heads[ic])))
         return cudaErrorInvalidValue;
+    if (!do_lm) { mQ0 = mQ1; mCK0 = mCK1; }
+    if (!do_instr) { mQ1 = mQ0; mCK1 = mCK0; }
     ColBatch<CAP> bt{};
-    bt.n = n;
-    int tiles = 0;
-    for (int i = 0; i < n; ++i) {
-        const TcSeqStep& q = seq[i];
-        TcParams& p = bt.p[i];
-        const int rows = which == 0 ? q.w : q.nI;
-        p.rows = rows; p.krow0 = q.kv_row0; p.chead = q.chead[ci];
-        p.q_heads = t.q_heads; p.kv_heads = t.kv_heads; p.m = q.m[ci]; p.L = q.L; p.status = status; p.dep_first = q.produced;
-        if (which == 0) {
-            p.row0 = q.q_row0 + (q.L - q.w); p.causal = 1; p.t0 = q.L - q.w;
-            p.lse_in = q.lse_chunk + (q.L - q.w); p.part = nullptr; p.splits = 1;
-        } else {
-            p.row0 = q.qi_row0; p.causal = 0; p.t0 = 0;
-            p.splits = q.splits < 1 ? 1 : q.splits;
-            p.lse_in = q.lse_instr; p.part = reinterpret_cast<float2*>(q.part);
+    int tiles = 0, e = 0;
+    for (int which = 0; which < 2; ++which) {
+        if (which == 0 ? !do_lm : !do_instr) continue;
+        const int ci = which == 0 ? 0 : ic;
+        for (int i = 0; i < n; ++i) {
+            const TcSeqStep& q = seq[i];
+            const int rows = which == 0 ? q.w : q.nI;
+            if (rows <= 0) continue;
+            TcParams& p = bt.p[e];
+            p.rows = rows; p.krow0 = q.kv_row0; p.chead = q.chead[ci];
+            p.q_heads = t.q_heads; p.kv_heads = t.kv_heads; p.m = q.m[ci]; p.L = q.L; p.status = status; p.dep_first = q.produced;
+            if (which == 0) {
+                p.row0 = q.q_row0 + (q.L - q.w); p.causal = 1; p.t0 = q.L - q.w;
+                p.lse_in = q.lse_chunk + (q.L - q.w); p.part = nullptr; p.splits = 1; p.lse_stride = lse_chunk_stride;
+            } else {
+                p.row0 = q.qi_row0; p.causal = 0; p.t0 = 0;
+                p.splits = q.splits < 1 ? 1 : q.splits;
+                p.lse_in = q.lse_instr; p.part = reinterpret_cast<float2*>(q.part); p.lse_stride = lse_instr_stride;
+            }
+            p.scores = q.scores[ci]; p.score_stride = q.score_stride;
+            tiles += (p.m + kTile - 1) / kTile + (p.L + kTile - 1) / kTile;
+            bt.tile_end[e++] = tiles;
         }
-        p.lse_stride = lse_stride; p.scores = q.scores[ci]; p.score_stride = q.score_stride;
-        if (rows > 0) tiles += (p.m + kTile - 1) / kTile + (p.L + kTile - 1) / kTile;
-        bt.tile_end[i] = tiles;
+        if (which == 0) bt.n_first = e;
     }
+    bt.n_entries = e;
     if (tiles == 0) return cudaSuccess;
     dim3 grid(t.kv_heads, tiles);
-    return launch_pdl(colsum_kernel<CAP>, grid, kColThreads, kColSmemBytes, s, mQ, mCK, mSK, bt);
+    return launch_pdl(colsum_kernel<CAP>, grid, kColThreads, kColSmemBytes, s, mQ0, mCK0, mQ1, mCK1, mSK, bt);
 }
 
-cudaError_t tc_colsum(const TcTensors& t, const TcSeqStep* seq, int n, int which, int lse_stride, int* status, cudaStream_t s) {
+cudaError_t tc_colsum(const TcTensors& t, const TcSeqStep* seq, int n, bool do_lm, bool do_instr, int lse_chunk_stride,
+                      int lse_instr_stride, int* status, cudaStream_t s) {
     if (n < 1 || n > kTcMaxBatch) return cudaErrorInvalidValue;
-    if (n == 1) return launch_colsum<1>(t, seq, n, which, lse_stride, status, s);
-    return launch_colsum<kTcMaxBatch>(t, seq, n, which, lse_stride, status, s);
+    if (!do_lm && !do_instr) return cudaSuccess;
+    if (n == 1) return launch_colsum<1>(t, seq, n, do_lm, do_instr, lse_chunk_stride, lse_instr_stride, status, s);
+    return launch_colsum<kTcMaxBatch>(t, seq, n, do_lm, do_instr, lse_chunk_stride, lse_instr_stride, status, s);
 }
 
 }  // namespace citrus
