@@ -137,6 +137,18 @@ int citrus_set_batch_lanes(citrus_handle h, int n_lanes);
  */
 int citrus_set_inputs_ready(citrus_handle h, int ready);
 
+/*
+ * Attention beside the scoring chain (no counterpart in the paper; a property of how the kernels are launched).  With a
+ * shared cache scored by the instruction text (section 4.2, shared cache design) nothing in a2-a4 reads a1's result.
+ * For a step with at most max_ctas attention items (128 query rows of one head each: one CTA) the library then runs a1
+ * on a stream of its own while the caller's stream runs log-sum-exp -> column sums -> select / gather on the SMs that
+ * leaves free; the two fork at the start of the call and join before it returns, so `out`, the caches and stream
+ * order look the same to the caller.  max_ctas = 0 switches this off (one launch for a1 and the log-sum-exp pass);
+ * the default is 64 (measured on 148 SMs: +20 % for 64 items; 128 items lose 10 % in any split, so they stay in one
+ * stream).  Results do not depend on the setting.  Errors: INVALID_ARG.
+ */
+int citrus_set_attention_beside(citrus_handle h, int max_ctas);
+
 /* Forget every cache of every layer and slot (start a new document). Host-only
  * bookkeeping; enqueues nothing. */
 int citrus_reset(citrus_handle h);

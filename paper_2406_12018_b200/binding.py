@@ -32,7 +32,7 @@ EXPORTS = [
     "citrus_create", "citrus_set_batch", "citrus_set_batch_lanes", "citrus_reset", "citrus_process_chunk", "citrus_process_chunk_slot",
     "citrus_process_chunk_host", "citrus_process_document_host", "citrus_process_chunk_batch", "citrus_cache_view", "citrus_step_view", "citrus_profile",
     "citrus_profile_read", "citrus_importance_static", "citrus_intersection_ratio", "citrus_set_rope_base",
-    "citrus_poll_status", "citrus_set_inputs_ready", "citrus_debug_expire_wait",
+    "citrus_poll_status", "citrus_set_inputs_ready", "citrus_set_attention_beside", "citrus_debug_expire_wait",
     "citrus_destroy", "citrus_strerror",
 ]
 
@@ -74,6 +74,7 @@ def load() -> C.CDLL:
     lib.citrus_importance_static.argtypes = [vp, i, vp, i, i, i, i, C.c_uint, vp, i, vp, vp]
     lib.citrus_poll_status.argtypes = [vp]
     lib.citrus_set_inputs_ready.argtypes = [vp, i]
+    lib.citrus_set_attention_beside.argtypes = [vp, i]
     lib.citrus_debug_expire_wait.argtypes = [vp, C.c_ulonglong, vp]
     lib.citrus_destroy.argtypes = [vp]
     lib.citrus_strerror.argtypes = [i]
@@ -281,6 +282,12 @@ class Citrus:
         rc = load().citrus_set_inputs_ready(self._h, 1 if ready else 0)
         if rc != 0:
             raise CitrusError(rc, "citrus_set_inputs_ready")
+
+    def set_attention_beside(self, max_ctas: int):
+        """Steps of at most max_ctas attention items run a1 on a side stream beside the scoring chain (0 = off; see citrus.h)."""
+        rc = load().citrus_set_attention_beside(self._h, int(max_ctas))
+        if rc != 0:
+            raise CitrusError(rc, "citrus_set_attention_beside")
 
     def debug_expire_wait(self, limit_ns: int = 1_000_000, stream=None):
         """Test aid: let one bounded device wait run out (see citrus.h)."""

@@ -77,6 +77,13 @@ struct citrus_ctx {
     cudaStream_t shift_stream = nullptr;
     bool shift_stream_set = false;
     cudaEvent_t shift_done = nullptr;
+    // a1 beside a2-a4: when nothing in a2-a4 reads a1's result (shared cache scored by the instruction text), the
+    // attention of a step of at most a1_cap items (CTAs) runs on a side stream while the caller's stream runs the
+    // chain log-sum-exp -> column sums -> select / gather on the SMs it leaves free; the streams fork at the start of
+    // a call and join before it returns.  0 = off.
+    int a1_cap = 64;
+    cudaStream_t a1_stream = nullptr;
+    cudaEvent_t a1_fork = nullptr, a1_done = nullptr;
     // optional per-launch timing: (kernel id, start, stop) event pairs recorded on the launching stream
     bool profiling = false;
     struct Timed { int id; cudaEvent_t a, b; };
@@ -146,6 +153,10 @@ void free_copy_streams(citrus_ctx* c) {
     c->lane_fork = nullptr;
     if (c->shift_done) cudaEventDestroy(c->shift_done);
     c->shift_done = nullptr;
+    if (c->a1_fork) cudaEventDestroy(c->a1_fork);
+    if (c->a1_done) cudaEventDestroy(c->a1_done);
+    if (c->a1_stream) cudaStreamDestroy(c->a1_stream);
+    c->a1_fork = c->a1_done = nullptr; c->a1_stream = nullptr;
 }
 // Side streams and events of the batch lanes (created once, by citrus_set_batch for more than one slot).
 int make_lanes(citrus_ctx* c) {
@@ -267,6 +278,12 @@ struct PackedIn {
 
 // The launch sequence of one chunk step for n sequences of one layer (n > 1: the tensor-core path without position
 // shift; every launch then covers all sequences).  The steps of different sequences are independent.
+cudaError_t join_a1(citrus_ctx* c, cudaStream_t st) {
+    cudaError_t e = cudaEventRecord(c->a1_done, c->a1_stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->a1_done, 0);
+    return e;
+}
+
 int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn* packed, cudaStream_t st, int lane = -1,
               bool inputs_ordered = false) {
     c->used = true;
@@ -347,6 +364,7 @@ int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn*
         if (sz[i].lm_scoring != sz[0].lm_scoring || sz[i].instr_scoring != sz[0].instr_scoring) return CITRUS_ERR_INVALID_ARG;
 
     cudaError_t e = cudaSuccess;
+    bool beside = false;                                           // a1 runs on the side stream: join before returning
     const void *Qc = in[0].Q, *Kc = in[0].K, *Qi = in[0].Qi;       // single-sequence paths below (n == 1)
     if (c->shift) {
         // position shift: embed the chunk's queries and keys at rows m .. m+L-1 and the instruction queries behind them
@@ -375,7 +393,35 @@ int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn*
             const LayerCache& lc = c->layer_cache[(size_t)layer * 2 + cc];
             t.cacheK[ci] = lc.K; t.cacheV[ci] = lc.V; t.cap[ci] = c->cap[cc]; t.cache_heads[ci] = 2 * c->n_slots * c->Hkv;
         }
-        {
+        // a1 beside a2-a4 (see a1_cap): one sequence on the caller's stream, nothing downstream reads a1's result,
+        // and the attention items leave SMs free for the chain
+        const int a1_items = ((in[0].L + 127) / 128) * c->Hq;
+        beside = n == 1 && lane < 0 && c->a1_stream != nullptr && !any_lm && any_instr &&
+                 in[0].out != nullptr && a1_items <= c->a1_cap;
+        if (beside) {
+            e = cudaEventRecord(c->a1_fork, st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(c->a1_stream, c->a1_fork, 0);
+            if (e != cudaSuccess) return cuda_rc(e);
+            cudaError_t e1, e2;
+            {
+                // a1 alone, behind everything the caller's stream held at the fork (so its inputs are complete)
+                TcSeqStep qa = seq[0];
+                qa.nI = 0; qa.produced = 0;
+                LaunchTimer tm(c, CITRUS_KERNEL_ATTENTION, c->a1_stream);
+                e1 = tc_attention_lse(t, &qa, 1, c->ls, CITRUS_MAX_INSTR, c->status, c->a1_stream);
+            }
+            {
+                // pass 1 of a2-I alone
+                TcTensors tl = t;
+                tl.out = nullptr;
+                LaunchTimer tm(c, CITRUS_KERNEL_SCORE_LSE, st);
+                e2 = tc_attention_lse(tl, seq.data(), 1, c->ls, CITRUS_MAX_INSTR, c->status, st);
+            }
+            if (e1 != cudaSuccess || e2 != cudaSuccess) {
+                join_a1(c, st);
+                return cuda_rc(e1 != cudaSuccess ? e1 : e2);
+            }
+        } else {
             // a1 and pass 1 of a2-I (row log-sum-exp of the instruction queries, possibly split over key ranges): one launch
             LaunchTimer tm(c, CITRUS_KERNEL_ATTENTION, st);
             e = tc_attention_lse(t, seq.data(), n, c->ls, CITRUS_MAX_INSTR, c->status, st);
@@ -387,7 +433,7 @@ int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn*
         if (any_lm || any_instr) {
             LaunchTimer tm(c, CITRUS_KERNEL_COLSUM, st);
             e = tc_colsum(t, seq.data(), n, any_lm, any_instr, c->ls, CITRUS_MAX_INSTR, c->status, st);
-            if (e != cudaSuccess) return cuda_rc(e);
+            if (e != cudaSuccess) { if (beside) join_a1(c, st); return cuda_rc(e); }
         }
     } else {
         Unit& u = c->units[(size_t)layer * c->n_slots + in[0].slot];
@@ -456,19 +502,22 @@ int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn*
         // one launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
         e = select_compact(sj.data(), cj.data(), n_jobs, c->Hkv, c->D * c->elt, c->elt, produced ? 0 : 1, st);
-        if (e != cudaSuccess) return cuda_rc(e);
+        if (e != cudaSuccess) { if (beside) join_a1(c, st); return cuda_rc(e); }
     } else {
         {
             LaunchTimer t(c, CITRUS_KERNEL_SELECT, st);
             e = select_topk(sj.data(), n_jobs, c->Hkv, c->layerwise ? 1 : 0, st);
         }
-        if (e != cudaSuccess) return cuda_rc(e);
+        if (e != cudaSuccess) { if (beside) join_a1(c, st); return cuda_rc(e); }
         {
             LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
             e = compact_kv(cj.data(), n_jobs, c->Hkv, c->D * c->elt, c->shift ? &c->rope : nullptr, c->elt, st);
         }
-        if (e != cudaSuccess) return cuda_rc(e);
+        if (e != cudaSuccess) { if (beside) join_a1(c, st); return cuda_rc(e); }
     }
+    // the caller's stream continues behind a1: `out` is complete in stream order, and the next step's compaction, which
+    // overwrites the cache buffer this a1 reads, comes after it
+    if (beside && (e = join_a1(c, st)) != cudaSuccess) return cuda_rc(e);
 
     for (int i = 0; i < n; ++i) {
         Unit& u = c->units[(size_t)layer * c->n_slots + in[i].slot];
@@ -556,6 +605,13 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
         cudaGetLastError();
         rc = CITRUS_ERR_CUDA;
     }
+    if (rc == CITRUS_OK && c->use_tc && !c->individual && !c->shift &&
+        (cudaStreamCreateWithFlags(&c->a1_stream, cudaStreamNonBlocking) != cudaSuccess ||
+         cudaEventCreateWithFlags(&c->a1_fork, cudaEventDisableTiming) != cudaSuccess ||
+         cudaEventCreateWithFlags(&c->a1_done, cudaEventDisableTiming) != cudaSuccess)) {
+        cudaGetLastError();
+        rc = CITRUS_ERR_CUDA;
+    }
     if (rc == CITRUS_OK && c->shift) {
         const size_t row = (size_t)head_dim * c->elt;
         rc = dev_alloc(c, &c->rotQ, (size_t)chunk_s * q_heads * row, false, true);
@@ -597,6 +653,12 @@ int citrus_set_batch_lanes(citrus_handle h, int n_lanes) {
     if (h == nullptr || !is_live(h)) return CITRUS_ERR_INVALID_ARG;
     if (n_lanes < 0 || n_lanes > citrus_ctx::kMaxLanes) return CITRUS_ERR_INVALID_ARG;
     h->lanes_wanted = n_lanes;
+    return CITRUS_OK;
+}
+
+int citrus_set_attention_beside(citrus_handle h, int max_ctas) {
+    if (h == nullptr || !is_live(h) || max_ctas < 0) return CITRUS_ERR_INVALID_ARG;
+    h->a1_cap = max_ctas;
     return CITRUS_OK;
 }
 

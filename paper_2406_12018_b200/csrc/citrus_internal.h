@@ -103,6 +103,7 @@ struct TcSeqStep {
     int produced;                          // 1: wait for the preceding kernels before the first load of Q / K / Qi
 };
 // One launch: a1 (chunk over [cache 0 ; chunk] -> out, optional row log-sum-exp) and pass 1 of a2-I of every sequence.
+// t.out == nullptr: pass 1 of a2-I alone; nI == 0 everywhere: a1 alone.
 cudaError_t tc_attention_lse(const TcTensors& t, const TcSeqStep* seq, int n, int lse_chunk_stride, int lse_instr_stride,
                              int* status, cudaStream_t s);
 // The column sums, one launch for both scorings and all sequences.  do_lm: the chunk's last w rows score cache 0's

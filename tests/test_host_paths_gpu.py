@@ -93,3 +93,52 @@ def test_inputs_ready_route_equals_the_default_route(mode):
     _, st = pu.run_document(w, ctx)
     assert st["checked_chunks"] == 9
     ctx.close()
+
+
+def test_attention_beside_the_scoring_chain_gives_the_same_bits_as_one_stream():
+    # Shared cache scored by the instruction text: nothing in a2-a4 reads a1's result, and a step of at most 64 attention
+    # items (here 2 row tiles x 32 heads) runs a1 on a side stream beside log-sum-exp -> column sums -> select / gather.
+    # Off (0), the default and a larger limit must agree bit for bit, with the calls enqueued back to back; the
+    # caller's stream alone orders `out` and the caches.
+    w = wl.scaled(C["mistral7b_layer"], chunk_s=256, doc_tokens=4096 + 100, n_planted=6)
+    doc = wl.make_document(w)
+    Q, K, V, Qi = (t.cuda() for t in (doc.Q, doc.K, doc.V, doc.Q_instr))
+    res = []
+    for cap in (0, None, 148):
+        ctx = pu.make_pair(w)
+        ctx.set_inputs_ready(True)
+        if cap is not None:
+            ctx.set_attention_beside(cap)
+        out = torch.empty_like(Q)
+        st = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(st):
+            for c in range(0, Q.shape[0], w.chunk_s):
+                sl = slice(c, min(Q.shape[0], c + w.chunk_s))
+                ctx.process_chunk(0, Q[sl], K[sl], V[sl], Qi, out=out[sl], stream=st)
+            seen = out.float().abs().sum()                 # stream-ordered read of `out` right behind the last call
+        torch.cuda.synchronize()
+        assert float(seen) == float(out.float().abs().sum())
+        res.append((out, tuple(t.clone() for t in ctx.cache_view(0, 0))))
+        assert ctx.poll_status() == 0
+        ctx.close()
+    for out, view in res[1:]:
+        assert torch.equal(res[0][0], out)
+        for x, y in zip(res[0][1], view):
+            assert torch.equal(x, y)
+    # and through a CUDA graph: the side stream joins the capture and leaves it again inside every call
+    ctx = pu.make_pair(w)
+    ctx.set_inputs_ready(True)
+    out = torch.empty_like(Q)
+    st = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g, stream=st):
+        for c in range(0, Q.shape[0], w.chunk_s):
+            sl = slice(c, min(Q.shape[0], c + w.chunk_s))
+            ctx.process_chunk(0, Q[sl], K[sl], V[sl], Qi, out=out[sl], stream=st)
+    ctx.reset()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(res[0][0], out) and ctx.poll_status() == 0
+    ctx.close()
