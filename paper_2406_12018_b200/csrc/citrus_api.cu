@@ -605,7 +605,7 @@ int citrus_create(citrus_handle* out, int layers, int q_heads, int kv_heads, int
         cudaGetLastError();
         rc = CITRUS_ERR_CUDA;
     }
-    if (rc == CITRUS_OK && c->use_tc && !c->individual && !c->shift &&
+    if (rc == CITRUS_OK && c->use_tc && !c->individual &&
         (cudaStreamCreateWithFlags(&c->a1_stream, cudaStreamNonBlocking) != cudaSuccess ||
          cudaEventCreateWithFlags(&c->a1_fork, cudaEventDisableTiming) != cudaSuccess ||
          cudaEventCreateWithFlags(&c->a1_done, cudaEventDisableTiming) != cudaSuccess)) {
