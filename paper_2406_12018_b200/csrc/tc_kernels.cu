@@ -164,81 +164,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
 }
-// 16 lanes x 128 consecutive 32-bit columns in the matrix-fragment layout: thread t holds, for every group of eight
-// columns i, columns 8 i + 2 (t % 4) + {0, 1} of lane (t / 4) in r[4 i], r[4 i + 1] and of lane (t / 4 + 8) in r[4 i + 2], r[4 i + 3].
-__device__ __forceinline__ void tmem_ld_frag64(uint32_t taddr, uint32_t* r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
-        "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
-        "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]),
-          "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]),
-          "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]),
-          "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]),
-          "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
-        : "r"(taddr) : "memory");
-}
-
-// 16 lanes x 64 consecutive 32-bit columns (32 registers) in the matrix-fragment layout: thread t holds, for every group of eight
-// columns i, columns 8 i + 2 (t % 4) + {0, 1} of lane (t / 4) in r[4 i], r[4 i + 1] and of lane (t / 4 + 8) in r[4 i + 2], r[4 i + 3].
-__device__ __forceinline__ void tmem_ld_frag32(uint32_t taddr, uint32_t* r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st_frag32(uint32_t taddr, const uint32_t* r) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.16x256b.x8.b32 [%32], "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
-        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
-          "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-          "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
-          "r"(taddr) : "memory");
-}
-
-// 16 lanes x 16 consecutive 32-bit columns in the matrix-fragment layout: thread t holds, for every group of eight
-// columns i, columns 8 i + 2 (t % 4) + {0, 1} of lane (t / 4) in r[4 i], r[4 i + 1] and of lane (t / 4 + 8) in r[4 i + 2], r[4 i + 3].
-__device__ __forceinline__ void tmem_ld_frag8(uint32_t taddr, uint32_t* r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x2.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st_frag8(uint32_t taddr, const uint32_t* r) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.16x256b.x2.b32 [%8], "
-        "{%0, %1, %2, %3, %4, %5, %6, %7};"
-        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-          "r"(taddr) : "memory");
-}
-
-// 16 lanes x 64 consecutive 32-bit columns (bf16 pairs): thread t holds column 4 i + (t % 4) of lane (t / 4) in r[2 i] and of
-// lane (t / 4 + 8) in r[2 i + 1] - the pair of adjacent fp32 columns it holds in the fragment layout above, packed.
-__device__ __forceinline__ void tmem_st_pairs32(uint32_t taddr, const uint32_t* r) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.16x128b.x16.b32 [%32], "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
-        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
-          "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-          "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
-          "r"(taddr) : "memory");
-}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -360,7 +285,7 @@ __device__ __forceinline__ void issue_pv(uint32_t tmem_o, uint32_t tmem_p, uint3
 constexpr int kStagesK = 2;             // K ring
 constexpr int kStagesV = 2;             // V ring
 constexpr int kVStageBytes = kTileBytes + kHalfBytes;   // a V tile and, right behind it, a [128 keys][64] block of ones
-constexpr int kAttnThreads = 384;       // 8 softmax warps, K-TMA warp, Q.K^T issuer, V-TMA warp, P.V issuer
+constexpr int kAttnThreads = 352;       // 8 softmax warps, K-TMA warp, MMA warp, V-TMA warp
 constexpr int kColGroups = 4;           // column-sum warp groups (four warps each), one S^T accumulator per group
 constexpr int kColThreads = (kColGroups * 4 + 2) * 32;   // the groups, 1 TMA warp, 1 MMA warp
 constexpr int kTmemCols = 512;
@@ -380,10 +305,10 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 struct AttnSmem {
-    uint64_t q_full, qk_ready[2], pv_ready[2];
-    uint64_t s_full[2], o_done[2], xch, out_ready[2], drain;
+    uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
+    uint64_t s_full[2], s_free[2], p_full, o_done[2], xch, out_ready[2], drain;
     uint32_t tmem_base;
-    float lsum[kTile], mfin[kTile];     // fp32 row sum and exponent reference of every row, for the thread that finishes it
+    float lsum[2][kTile];               // fp32 row sums of the two column halves, exchanged once at the end
 };
 constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + kStagesK) + kVStageBytes * kStagesV + 4096;
 
@@ -395,10 +320,10 @@ constexpr int kAttnSmemBytes = 1024 /*align slack*/ + kTileBytes * (1 + kStagesK
 // as soon as the softmax warps have read S of tile j into registers; the tensor pipe never waits for the
 // exponentials of the tile it is about to overwrite, only P.V of tile j waits for P of tile j.
 //
-// Softmax: eight warps; warp w owns rows 32 (w & 3) + 16 (w >> 2) .. +15 and all 128 columns, which it reads once per
-// tile in the matrix-fragment layout (16 lanes x 256 bits: four threads share a row, each holding two adjacent columns
-// of every group of eight, for two rows), so the row maximum costs two shuffles and nothing is read twice or
-// exchanged through shared memory.  The row sum of the bf16-rounded probabilities - the normaliser that makes
+// Softmax: eight warps; warps w and w+4 share rows 32 (w & 3) .. +31, thread (w, lane) owns columns
+// 64 (w >> 2) .. +63 of its row.  Both threads of a row read all 128 columns once to take the same row maximum
+// (so they agree on the exponent reference and on every rescale without exchanging anything) and keep only their
+// own half for the exponentials.  The row sum of the bf16-rounded probabilities - the normaliser that makes
 // out = sum(p~ v) / sum(p~) a convex combination of V rows - comes from the tensor core itself: the V operand of
 // P.V is 144 columns wide, the last 16 read from a block of ones, so columns 128..143 of O accumulate sum(p~)
 // in the same fp32 arithmetic as the output columns, and are rescaled with them.
@@ -430,16 +355,16 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
     const int nt = max(0, tile_end - tile_begin);
 
     if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars->q_full), 1);
+        for (int s = 0; s < kStagesK; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
+        for (int s = 0; s < kStagesV; ++s) { mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1); }
         for (int b = 0; b < 2; ++b) {
-            // qk_ready[b]: K of tile j = b (mod 2) is staged (one arrival that carries the bytes) and S[b] is free (eight
-            // arrivals, one per softmax warp); pv_ready[b]: V of that tile is staged (one) and its P is stored (eight)
-            mbar_init(smem_u32(&bars->qk_ready[b]), 9); mbar_init(smem_u32(&bars->pv_ready[b]), 9);
-            mbar_init(smem_u32(&bars->s_full[b]), 1);
+            mbar_init(smem_u32(&bars->s_full[b]), 1); mbar_init(smem_u32(&bars->s_free[b]), 8);
             mbar_init(smem_u32(&bars->o_done[b]), 1); mbar_init(smem_u32(&bars->out_ready[b]), 4);
         }
-        mbar_init(smem_u32(&bars->q_full), 1);
+        mbar_init(smem_u32(&bars->p_full), 8);
         mbar_init(smem_u32(&bars->xch), 8);
-        mbar_init(smem_u32(&bars->drain), WITH_PV ? 2 : 1);
+        mbar_init(smem_u32(&bars->drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (WITH_PV) {
@@ -501,9 +426,8 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 if (WITH_PV && lane == 0) atomicMax(&g_citrus_trace[244], ~global_ns());
 #endif
             }
-            // stage s = j & 1 is free once Q.K^T of tile j - 2 has retired, which is what s_full of that tile says
-            if (j >= 2 && !mbar_wait_warp(smem_u32(&bars->s_full[s]), ((j >> 1) - 1) & 1, p.status)) break;
-            load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->qk_ready[s]), row, from_cache ? p.chead + g : g, !from_cache);
+            if (!mbar_wait_warp(smem_u32(&bars->k_empty[s]), ((j / kStagesK) & 1) ^ 1, p.status)) break;
+            load_tile(sK + s * kTileBytes, from_cache ? &mapCK : &mapSK, smem_u32(&bars->k_full[s]), row, from_cache ? p.chead + g : g, !from_cache);
         }
     } else if (warp == 10) {
         // ---------------------------------------------------------------- V TMA producer (converged warp)
@@ -514,225 +438,182 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
                 const bool from_cache = jg < n_cache_tiles;
                 const int row = from_cache ? jg * kTile : p.krow0 + (jg - n_cache_tiles) * kTile;
                 if (from_cache && !dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
-                if (j >= 2 && !mbar_wait_warp(smem_u32(&bars->o_done[s]), ((j >> 1) - 1) & 1, p.status)) break;   // P.V of tile j - 2
-                load_tile(sV + s * kVStageBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->pv_ready[s]), row, from_cache ? p.chead + g : g, !from_cache);
+                if (!mbar_wait_warp(smem_u32(&bars->v_empty[s]), ((j / kStagesV) & 1) ^ 1, p.status)) break;
+                load_tile(sV + s * kVStageBytes, from_cache ? &mapCV : &mapSV, smem_u32(&bars->v_full[s]), row, from_cache ? p.chead + g : g, !from_cache);
             }
         }
     } else if (warp == 9) {
-        // ---------------------------------------------------------------- Q.K^T issuer: one thread.
-        // An MMA occupies its issuing thread for as long as the tensor pipe works on it (64 cycles at 128 x 128 x 16),
-        // and every wait of an issuer costs a few hundred cycles of dependent instructions that compete for issue slots
-        // with the softmax warps; with one issuer for both products that chain (17 MMAs and four waits per key tile) was
-        // as long as the softmax warps' own.  So each product has its issuer, with one wait and one commit per tile.
-        if (lane == 0) {
-            constexpr uint32_t idesc_qk = make_idesc(128, 0);
-            const uint64_t dQ = desc_kmajor(sQ);
-            bool ok = mbar_wait(smem_u32(&bars->q_full), 0, p.status);
-            if (WITH_PV) CITRUS_TR(2);
-            auto step = [&](int j, const int b) {
-                ok = mbar_wait(smem_u32(&bars->qk_ready[b]), (j >> 1) & 1, p.status);
-                if (!ok) return;
-                tc_fence_after();
-                const uint64_t dK = desc_kmajor(sK + b * kTileBytes);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);   // start-address field units
-                    mma_ss(tmS(b), dQ + off, dK + off, idesc_qk, kk > 0);
-                }
-                mma_commit(smem_u32(&bars->s_full[b]));
-                if (WITH_PV && j >= 2 && j < 12) CITRUS_TR(10 + j);
-            };
-            for (int j = 0; j < nt && ok; j += 2) {
-                step(j, 0);
-                if (ok && j + 1 < nt) step(j + 1, 1);
-            }
-            // all tensor-core work retired before tensor memory is released
-            mma_commit(smem_u32(&bars->drain));
-            mbar_wait(smem_u32(&bars->drain), 0, p.status);
+        // ---------------------------------------------------------------- MMA issuer (converged warp)
+        constexpr uint32_t idesc_qk = make_idesc(128, 0);
+        constexpr uint32_t idesc_pv = make_idesc(kOCols, 1);
+        bool ok = mbar_wait_warp(smem_u32(&bars->q_full), 0, p.status);
+        if (WITH_PV) CITRUS_TR(2);
+        auto k_ready = [&](int j) { return mbar_wait_warp(smem_u32(&bars->k_full[j % kStagesK]), (j / kStagesK) & 1, p.status); };
+        auto qk = [&](int j) {
+            const int s = j % kStagesK;
+            issue_qk(tmS(j & 1), sQ, sK + s * kTileBytes, idesc_qk, smem_u32(&bars->s_full[j & 1]), smem_u32(&bars->k_empty[s]));
+        };
+        for (int j = 0; j < 2 && j < nt && ok; ++j) {
+            ok = k_ready(j);
+            if (ok) { tc_fence_after(); qk(j); }
         }
-        __syncwarp();
-    } else if (warp == 11) {
-        // ---------------------------------------------------------------- P.V issuer: one thread
-        if (WITH_PV && lane == 0) {
-            constexpr uint32_t idesc_pv = make_idesc(kOCols, 1);
-            bool ok = true;
-            auto step = [&](int j, const int b) {
-                ok = mbar_wait(smem_u32(&bars->pv_ready[b]), (j >> 1) & 1, p.status);
-                if (!ok) return;
+        for (int j = 0; j < nt && ok; ++j) {
+            if (j + 2 < nt) {
+                // S[j & 1] is free as soon as every softmax thread holds tile j in registers
+                ok = k_ready(j + 2) && mbar_wait_warp(smem_u32(&bars->s_free[j & 1]), (j >> 1) & 1, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                qk(j + 2);
+                if (WITH_PV && j + 2 < 12) CITRUS_TR(10 + j + 2);
+            }
+            if (WITH_PV) {
+                const int s = j % kStagesV;
+                ok = mbar_wait_warp(smem_u32(&bars->v_full[s]), (j / kStagesV) & 1, p.status) &&
+                     mbar_wait_warp(smem_u32(&bars->p_full), j & 1, p.status);
+                if (!ok) break;
                 tc_fence_after();
                 if (j < 10) CITRUS_TR(90 + j);
-                const uint64_t dV = desc_mnmajor(sV + b * kVStageBytes);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)     // 16 keys per step: P columns 8*kk.., V rows 16*kk.. (2048 B apart)
-                    mma_ts(tmem + kTmemO, tmem + kTmemP + kk * 8, dV + (uint64_t)((kk * 2048) >> 4), idesc_pv, !(j == 0 && kk == 0));
-                mma_commit(smem_u32(&bars->o_done[b]));
+                issue_pv(tmem + kTmemO, tmem + kTmemP, sV + s * kVStageBytes, idesc_pv, j == 0,
+                         smem_u32(&bars->v_empty[s]), smem_u32(&bars->o_done[j & 1]));
                 if (j < 10) CITRUS_TR(30 + j);
-            };
-            for (int j = 0; j < nt && ok; j += 2) {
-                step(j, 0);
-                if (ok && j + 1 < nt) step(j + 1, 1);
             }
-            mma_commit(smem_u32(&bars->drain));
         }
+        // all tensor-core work retired before tensor memory is released
+        if (elect_one()) mma_commit(smem_u32(&bars->drain));
         __syncwarp();
+        mbar_wait_warp(smem_u32(&bars->drain), 0, p.status);
     } else {
         // ---------------------------------------------------------------- softmax warps 0-7
-        // Warp w owns rows 32 (w & 3) + 16 (w >> 2) .. + 15 of the tile and all 128 columns, in the matrix-fragment
-        // layout of tensor memory: a thread holds, for two rows (A and B = A + 8), two adjacent columns of every group of
-        // eight.  One read of S per tile, the row maximum by two shuffles inside the four threads that share a row, and
-        // each adjacent pair of probabilities is one packed bf16 column of P.
-        const int rbase = (warp & 3) * 32 + (warp >> 2) * 16;
-        const int rowA = rbase + (lane >> 2);                        // rows of this thread inside the tile: rowA, rowA + 8
-        const int cq = (lane & 3) * 2;                               // its columns: 8 i + cq, 8 i + cq + 1
-        const uint32_t frag_base = (uint32_t)rbase << 16;
+        const int half = warp >> 2;                                  // which 64 columns of the row this thread keeps
+        const int row_in_tile = (warp & 3) * 32 + lane;
+        const int r = q_row0 + row_in_tile;                          // row inside the block
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t o_addr = tmem + kTmemO + lane_base;
+        const uint32_t p_addr = tmem + kTmemP + lane_base + (uint32_t)half * 32u;
         const float scale2 = kLog2e * rsqrtf((float)kD);
         const uint64_t scale2x2 = pack_f32x2(scale2, scale2);
-        float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        float m_ref = -INFINITY, l_run = 0.f;
         bool ok = true;
-        mbar_arrive_warp(smem_u32(&bars->qk_ready[0]));             // both S buffers start out free
-        mbar_arrive_warp(smem_u32(&bars->qk_ready[1]));
 #pragma unroll 1
         for (int j = 0; j < nt; ++j) {
             const int b = j & 1;
             ok = mbar_wait_warp(smem_u32(&bars->s_full[b]), (j >> 1) & 1, p.status);
             if (!ok) break;
-            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR(((warp >> 2) ? 200 : 50) + 5 * j);
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 200 : 50) + 5 * j);
             tc_fence_after();
-            // number of visible columns of this tile for each of the two rows
-            int lim[2] = {kTile, kTile};
+            // number of visible columns of this tile for this row
+            int lim = kTile;
             const int jg = sweep_tile(j);
             if (jg < n_cache_tiles) {
-                lim[0] = lim[1] = min(kTile, p.m - jg * kTile);
+                lim = min(kTile, p.m - jg * kTile);
             } else {
                 const int u0 = (jg - n_cache_tiles) * kTile;
-                lim[0] = lim[1] = min(kTile, p.L - u0);
-                if (p.causal) {
-                    lim[0] = min(lim[0], p.t0 + q_row0 + rowA - u0 + 1);
-                    lim[1] = min(lim[1], p.t0 + q_row0 + rowA + 8 - u0 + 1);
-                }
+                lim = min(kTile, p.L - u0);
+                if (p.causal) lim = min(lim, p.t0 + r - u0 + 1);
             }
-            uint32_t v[64];                                          // v[4 i + 2 x + e]: row x, column 8 i + cq + e
-            tmem_ld_frag64(tmS(b) + frag_base, v);
+            const uint32_t s_addr = tmS(b) + lane_base;
+            uint32_t own[64], oth[64];
+            tmem_ld32(s_addr + (half ^ 1) * 64, oth);
+            tmem_ld32(s_addr + (half ^ 1) * 64 + 32, oth + 32);
+            tmem_ld32(s_addr + half * 64, own);
+            tmem_ld32(s_addr + half * 64 + 32, own + 32);
             tmem_wait_ld();
             tc_fence_before();
-            mbar_arrive_warp(smem_u32(&bars->qk_ready[b]));
+            mbar_arrive_warp(smem_u32(&bars->s_free[b]));
             // ---- row maximum over the visible columns.  A tile that holds hidden columns (future tokens of the chunk,
             // rows past the end of the cache or chunk - zero fill, stale cache rows, or in a packed batch the next
-            // sequence's rows) has them set to -inf first.
-            if (lim[0] < kTile || lim[1] < kTile) {
+            // sequence's rows) has them set to -inf first, in both halves, so both threads of the row still agree.
+            if (lim < kTile) {
+                const int lim_own = lim - half * 64, lim_oth = lim - (half ^ 1) * 64;
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        if (8 * i + cq + e >= lim[0]) v[4 * i + e] = 0xff800000u;          // -inf
-                        if (8 * i + cq + e >= lim[1]) v[4 * i + 2 + e] = 0xff800000u;
-                    }
+                for (int q = 0; q < 64; ++q) {
+                    if (q >= lim_own) own[q] = 0xff800000u;          // -inf
+                    if (q >= lim_oth) oth[q] = 0xff800000u;
+                }
             }
-            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};                  // [row][two chains]
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                mx4[i & 1] = max3(mx4[i & 1], __uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]));
-                mx4[2 + (i & 1)] = max3(mx4[2 + (i & 1)], __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+            for (int q = 0; q < 64; q += 2) {
+                mx4[(q >> 1) & 1] = max3(mx4[(q >> 1) & 1], __uint_as_float(oth[q]), __uint_as_float(oth[q + 1]));
+                mx4[2 + ((q >> 1) & 1)] = max3(mx4[2 + ((q >> 1) & 1)], __uint_as_float(own[q]), __uint_as_float(own[q + 1]));
             }
-            float mx[2] = {fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])};
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                mx[x] = fmaxf(mx[x], __shfl_xor_sync(0xffffffffu, mx[x], 1));
-                mx[x] = fmaxf(mx[x], __shfl_xor_sync(0xffffffffu, mx[x], 2));
-            }
-            const float m_new[2] = {fmaxf(m_ref[0], mx[0] * scale2), fmaxf(m_ref[1], mx[1] * scale2)};
-            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR(((warp >> 2) ? 201 : 51) + 5 * j);
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            const float m_new = fmaxf(m_ref, mx * scale2);
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 201 : 51) + 5 * j);
             if (j == 0) {
-                m_ref[0] = m_new[0]; m_ref[1] = m_new[1];
+                m_ref = m_new;
             } else {
-                // the four threads of a row see the same maximum, so they take the same decision
-                const bool grow[2] = {m_new[0] > m_ref[0] + kRescaleTau,      // also when the row has seen nothing so far
-                                      m_new[1] > m_ref[1] + kRescaleTau};     // (m_ref = -inf)
-                if (__any_sync(0xffffffffu, grow[0] || grow[1])) {
+                // both threads of a row see the same values, so they take the same decision
+                const bool grow = m_new > m_ref + kRescaleTau;       // also when the row has seen nothing so far (m_ref = -inf)
+                if (__any_sync(0xffffffffu, grow)) {
                     // Only the rows that grew change their reference; the others scale by exactly one.  A row's
                     // arithmetic therefore never depends on what the other rows of its warp hold (in a packed batch
                     // the rows past a sequence's end are the next sequence's), and results are the same bits whether
                     // a sequence is stepped alone or inside a batch.
-                    float f[2];
-#pragma unroll
-                    for (int x = 0; x < 2; ++x) {
-                        f[x] = grow[x] ? ex2(m_ref[x] - m_new[x]) : 1.f;
-                        if (grow[x]) { l_run[x] *= f[x]; m_ref[x] = m_new[x]; }
-                    }
+                    const float f = grow ? ex2(m_ref - m_new) : 1.f;
+                    if (grow) { l_run *= f; m_ref = m_new; }
                     if (WITH_PV) {
                         // O must be quiescent: P.V of tile j-1 (and with it every earlier one) has retired
                         ok = pv_done(j - 1);
                         if (!ok) break;
                         tc_fence_after();
 #pragma unroll 1
-                        for (int c = 0; c < 2; ++c) {                // 64 columns (32 registers) at a time
+                        for (int c = 0; c < 2; ++c) {
                             uint32_t oreg[32];
-                            tmem_ld_frag32(tmem + kTmemO + frag_base + c * 64, oreg);
+                            tmem_ld32(o_addr + half * 64 + c * 32, oreg);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int q = 0; q < 32; ++q) oreg[q] = __float_as_uint(__uint_as_float(oreg[q]) * f[(q >> 1) & 1]);
-                            tmem_st_frag32(tmem + kTmemO + frag_base + c * 64, oreg);
+                            for (int q = 0; q < 32; ++q) oreg[q] = __float_as_uint(__uint_as_float(oreg[q]) * f);
+                            tmem_st32(o_addr + half * 64 + c * 32, oreg);
                         }
-                        uint32_t lreg[8];
-                        tmem_ld_frag8(tmem + kTmemL + frag_base, lreg);
-                        tmem_wait_ld();
+                        if (half == 0) {
+                            uint32_t lreg[16];
+                            tmem_ld16(tmem + kTmemL + lane_base, lreg);
+                            tmem_wait_ld();
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) lreg[q] = __float_as_uint(__uint_as_float(lreg[q]) * f[(q >> 1) & 1]);
-                        tmem_st_frag8(tmem + kTmemL + frag_base, lreg);
+                            for (int q = 0; q < 16; ++q) lreg[q] = __float_as_uint(__uint_as_float(lreg[q]) * f);
+                            tmem_st16(tmem + kTmemL + lane_base, lreg);
+                        }
                     }
                 }
             }
-            // ---- probabilities; with NEED_LSE the fp32 values are summed too (that sum feeds the log-sum-exp that
-            // the LM scoring pass reuses)
-            const float neg_m[2] = {m_ref[0] == -INFINITY ? 0.f : -m_ref[0], m_ref[1] == -INFINITY ? 0.f : -m_ref[1]};
-            const uint64_t neg_m2[2] = {pack_f32x2(neg_m[0], neg_m[0]), pack_f32x2(neg_m[1], neg_m[1])};
+            // ---- probabilities of this thread's 64 columns; with NEED_LSE the fp32 values are summed too (that sum
+            // feeds the log-sum-exp that the LM scoring pass reuses)
+            const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
+            const uint64_t neg_m2 = pack_f32x2(neg_m, neg_m);
             uint64_t sum2[2] = {0ull, 0ull};
-            uint32_t packed[32];                                     // packed[2 i + x]: row x, P column 4 i + (lane & 3)
-            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR(((warp >> 2) ? 202 : 52) + 5 * j);
+            uint32_t packed[32];
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 202 : 52) + 5 * j);
 #pragma unroll
-            for (int i = 0; i < 16; ++i)
-#pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    float x0, x1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[4 * i + 2 * x]), __uint_as_float(v[4 * i + 2 * x + 1])),
-                                           scale2x2, neg_m2[x]), x0, x1);
-                    const float p0 = ex2(x0), p1 = ex2(x1);
-                    if (NEED_LSE) sum2[x] = add_f32x2(sum2[x], pack_f32x2(p0, p1));
-                    packed[2 * i + x] = pack_bf16(p0, p1);
-                }
-            if (NEED_LSE) {
-                float a0, a1;
-                unpack_f32x2(sum2[0], a0, a1); l_run[0] += a0 + a1;
-                unpack_f32x2(sum2[1], a0, a1); l_run[1] += a0 + a1;
+            for (int q = 0; q < 32; ++q) {
+                float x0, x1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(own[2 * q]), __uint_as_float(own[2 * q + 1])), scale2x2, neg_m2), x0, x1);
+                const float p0 = ex2(x0), p1 = ex2(x1);
+                if (NEED_LSE) sum2[q & 1] = add_f32x2(sum2[q & 1], pack_f32x2(p0, p1));
+                packed[q] = pack_bf16(p0, p1);
             }
-            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR(((warp >> 2) ? 203 : 53) + 5 * j);
+            if (NEED_LSE) {
+                float a0, a1, b0, b1;
+                unpack_f32x2(sum2[0], a0, a1); unpack_f32x2(sum2[1], b0, b1);
+                l_run += (a0 + a1) + (b0 + b1);
+            }
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 203 : 53) + 5 * j);
             if (WITH_PV) {
                 // the single P buffer is free once P.V of the previous tile has read it
                 if (j > 0) { ok = pv_done(j - 1); if (!ok) break; }
                 tc_fence_after();
-                tmem_st_pairs32(tmem + kTmemP + frag_base, packed);
+                tmem_st16(p_addr, packed);
+                tmem_st16(p_addr + 16, packed + 16);
                 tmem_wait_st();                                      // also covers a rescale's stores to O
                 tc_fence_before();
-                mbar_arrive_warp(smem_u32(&bars->pv_ready[b]));
+                mbar_arrive_warp(smem_u32(&bars->p_full));
             }
-            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR(((warp >> 2) ? 204 : 54) + 5 * j);
+            if (WITH_PV && (warp & 3) == 0 && j < 8) CITRUS_TR((half ? 204 : 54) + 5 * j);
         }
-        // ---- epilogue: rows are finished in the plain layout (thread = row, 64 columns each: warps w and w + 4 share
-        // rows 32 (w & 3) .. + 31), so a row's reference and fp32 sum travel through shared memory
-        const int half = warp >> 2;                                  // which 64 output columns this thread finishes
-        const int row_in_tile = (warp & 3) * 32 + lane;
-        const int r = q_row0 + row_in_tile;                          // row inside the block
-        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t o_addr = tmem + kTmemO + lane_base;
+        // ---- epilogue
         if (ok && WITH_PV && nt > 0) ok = pv_done(nt - 1);
         if (NEED_LSE) {
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                float l = l_run[x];
-                l += __shfl_xor_sync(0xffffffffu, l, 1);
-                l += __shfl_xor_sync(0xffffffffu, l, 2);
-                if ((lane & 3) == 0) { bars->lsum[rowA + 8 * x] = l; bars->mfin[rowA + 8 * x] = m_ref[x]; }
-            }
+            bars->lsum[half][row_in_tile] = l_run;
             mbar_arrive_warp(smem_u32(&bars->xch));
             ok = mbar_wait_warp(smem_u32(&bars->xch), 0, p.status) && ok;
         }
@@ -792,9 +673,9 @@ __device__ __forceinline__ void attn_body(const CUtensorMap& mapQ, const CUtenso
             }
             if (NEED_LSE && half == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // see the note on the sweep order
             if (NEED_LSE && half == 0 && row_ok) {
-                const float l = bars->lsum[row_in_tile], m_row = bars->mfin[row_in_tile];
-                if (p.splits > 1) p.part[((size_t)split * p.q_heads + oh) * p.lse_stride + orow] = make_float2(m_row, l);
-                else if (p.lse2 != nullptr) p.lse2[(size_t)oh * p.lse_stride + orow] = m_row + log2f(l);
+                const float l = bars->lsum[0][row_in_tile] + bars->lsum[1][row_in_tile];
+                if (p.splits > 1) p.part[((size_t)split * p.q_heads + oh) * p.lse_stride + orow] = make_float2(m_ref, l);
+                else if (p.lse2 != nullptr) p.lse2[(size_t)oh * p.lse_stride + orow] = m_ref + log2f(l);
             }
         }
     }
