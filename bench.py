@@ -40,6 +40,7 @@ WORKLOAD = "long_doc_stress"
 # workload, from the ncu summary under profiles/; None whenever that kernel has changed since the capture.
 ATTN_DRAM_TRAFFIC_BYTES = 102.4e6
 ATTENTION_BESIDE = None          # --attention-beside: passed to every context (None = the library's default)
+BATCH_LANES = 0                  # --lanes: passed to the contexts of batch workloads (0 = the library's choice)
 METRIC = "document tokens/s through chunked eviction per layer"
 UNIT = "tokens/s"
 TARGET_TIMED_SECONDS = 2.2
@@ -308,6 +309,8 @@ class Job:
         self.ctx.set_inputs_ready(True)
         if ATTENTION_BESIDE is not None:
             self.ctx.set_attention_beside(ATTENTION_BESIDE)
+        if self.batch and BATCH_LANES:
+            self.ctx.set_batch_lanes(BATCH_LANES)
 
     def one_pass(self):
         """Every chunk of every (layer | sequence) once, in the order a model would submit them."""
@@ -620,14 +623,15 @@ def main():
                     help="stop after the rank set-up (prints rank, world size and this rank's share of the work)")
     ap.add_argument("--sequences", type=int, default=1,
                     help="side measurement: this many documents advance together through the ragged-batch call (1 GPU)")
-    ap.add_argument("--lanes", type=int, default=0, help="with --sequences: side streams of the batch call (0 = automatic)")
+    ap.add_argument("--lanes", type=int, default=0, help="batch workloads and --sequences: citrus_set_batch_lanes (0 = the library's choice: one grid over all sequences)")
     ap.add_argument("--attention-beside", type=int, default=None,
                     help="largest step (attention items) whose a1 runs beside the scoring chain (citrus_set_attention_beside; 0 = off; default: the library's)")
     ap.add_argument("--traffic", type=float, default=ATTN_DRAM_TRAFFIC_BYTES,
                     help="DRAM bytes per attention launch from the committed ncu summary (null if stale)")
     args = ap.parse_args()
-    global ATTENTION_BESIDE
+    global ATTENTION_BESIDE, BATCH_LANES
     ATTENTION_BESIDE = args.attention_beside
+    BATCH_LANES = args.lanes
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if "WORLD_SIZE" not in os.environ and args.gpus > 1:
         raise SystemExit(respawn_under_torchrun(args))
