@@ -497,11 +497,11 @@ int run_steps(citrus_ctx* c, int layer, int n, const StepIn* in, const PackedIn*
     // SM streaming rows, which the clusters (idle while their first CTA selects) cannot give: two launches.
     int n_most = 0;
     for (const SelectJob& j : sj) n_most = j.n > n_most ? j.n : n_most;
-    if (!c->layerwise && !c->shift && !c->accumulate && gather_bytes <= ((size_t)8 << 20) * (size_t)n &&
+    if (!c->shift && !c->accumulate && gather_bytes <= ((size_t)8 << 20) * (size_t)n &&
         select_compact_fits(n_most, c->D * c->elt)) {
         // one launch does both (timed under the compaction id)
         LaunchTimer t(c, CITRUS_KERNEL_COMPACT, st);
-        e = select_compact(sj.data(), cj.data(), n_jobs, c->Hkv, c->D * c->elt, c->elt, produced ? 0 : 1, st);
+        e = select_compact(sj.data(), cj.data(), n_jobs, c->Hkv, c->D * c->elt, c->elt, produced ? 0 : 1, c->layerwise ? 1 : 0, st);
         if (e != cudaSuccess) { if (beside) join_a1(c, st); return cuda_rc(e); }
     } else {
         {

@@ -155,10 +155,11 @@ cudaError_t compact_kv(const CompactJob* jobs, int n_jobs, int kv_heads, int row
 // a3 + a4 in one launch (per-head granularity, no carried importance, no position shift) for small steps: several
 // CTAs per (cache, KV head), each staging its share of the candidate rows in shared memory while it selects.
 // early_chunk_rows: the chunk's K / V may be read before the preceding kernels have ended (caller inputs, complete).
+// layerwise: every head keeps the candidates that the sum of the heads' scores ranks highest.
 // select_compact_fits: whether a step of n candidates with rows of row_bytes fits that kernel's shared memory.
 bool select_compact_fits(int n, int row_bytes);
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, int kv_heads, int row_bytes,
-                           int elt, int early_chunk_rows, cudaStream_t s);
+                           int elt, int early_chunk_rows, int layerwise, cudaStream_t s);
 // ratio[g] = |{positions of a} intersect {positions of b}| / rows_b over two ascending position lists per head
 cudaError_t intersection_ratio(const int* pos_a, int stride_a, int rows_a, const int* pos_b, int stride_b, int rows_b,
                                int kv_heads, float* ratio, cudaStream_t s);

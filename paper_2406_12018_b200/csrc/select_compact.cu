@@ -400,7 +400,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 template <int CAP>
 __global__ void __launch_bounds__(kSelThreads)
 select_gather_kernel(const __grid_constant__ SelectArgs<CAP> sel, const __grid_constant__ CompactArgs<CAP> cmp,
-                     int kv_heads, int n_max, int share_max, int row_bytes, int early_chunk_rows) {
+                     int kv_heads, int n_max, int share_max, int row_bytes, int early_chunk_rows, int layerwise) {
     extern __shared__ __align__(128) uint8_t sg_smem[];
     __shared__ uint64_t rows_bar;
     __shared__ uint32_t w_gt[32], w_eq[32], w_keep[32];
@@ -469,7 +469,8 @@ select_gather_kernel(const __grid_constant__ SelectArgs<CAP> sel, const __grid_c
     } else {
         uint32_t T, take_eq;
         CITRUS_TR(4);
-        select_threshold(sjob, g, kv_heads, 0, keys, T, take_eq);
+        // (layer-wise granularity: every CTA ranks the sum of the heads' scores, so all heads keep the same candidates)
+        select_threshold(sjob, g, kv_heads, layerwise, keys, T, take_eq);
         CITRUS_TR(5);
         // kept candidates and candidates equal to T before the share (all threads count a slice of keys[0, c0))
         uint32_t gt = 0u, eq = 0u;
@@ -680,7 +681,7 @@ bool select_compact_fits(int n, int row_bytes) {
 
 template <int CAP>
 static cudaError_t launch_select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, int kv_heads, int row_bytes,
-                                         int elt, int early_chunk_rows, cudaStream_t s) {
+                                         int elt, int early_chunk_rows, int layerwise, cudaStream_t s) {
     SelectArgs<CAP> sa; CompactArgs<CAP> ca;
     ca.elt = elt;
     int n = 0;
@@ -699,16 +700,16 @@ static cudaError_t launch_select_compact(const SelectJob* sjobs, const CompactJo
     cfg.attrs = attr; cfg.numAttrs = 1;
     before_launch(s);
     return cudaLaunchKernelEx(&cfg, select_gather_kernel<CAP>, sa, ca, kv_heads, n, (n + kFusedParts - 1) / kFusedParts, row_bytes,
-                              early_chunk_rows);
+                              early_chunk_rows, layerwise);
 }
 
 cudaError_t select_compact(const SelectJob* sjobs, const CompactJob* cjobs, int n_jobs, int kv_heads, int row_bytes,
-                           int elt, int early_chunk_rows, cudaStream_t s) {
+                           int elt, int early_chunk_rows, int layerwise, cudaStream_t s) {
     if (n_jobs < 1 || n_jobs > kJobsBatch) return cudaErrorInvalidValue;
     cudaError_t e = raise_smem_limits();
     if (e != cudaSuccess) return e;
-    if (n_jobs <= kJobsSingle) return launch_select_compact<kJobsSingle>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, early_chunk_rows, s);
-    return launch_select_compact<kJobsBatch>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, early_chunk_rows, s);
+    if (n_jobs <= kJobsSingle) return launch_select_compact<kJobsSingle>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, early_chunk_rows, layerwise, s);
+    return launch_select_compact<kJobsBatch>(sjobs, cjobs, n_jobs, kv_heads, row_bytes, elt, early_chunk_rows, layerwise, s);
 }
 
 template <int CAP>
